@@ -1,0 +1,398 @@
+#!/usr/bin/env python
+"""Benchmark of the ScaleKV per-scale hot path on B200.
+
+One "step" = one full pass of the workload: after a reset, for every scale k and every layer,
+append -> attend -> compress (no compress after the last scale).  The metric is scale-steps per
+second (one scale-step = append + attend + compress of every layer at one scale); passes per
+second is printed beside it.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload pass2b] [--impl reference]
+
+Prints one JSON line.  Inputs are seeded synthetic tensors (see paper_2505_19602_b200/synth.py),
+generated on the device before the timed region.  With --gpus N > 1 (under torchrun) every rank
+runs an independent replica on its own batch: the path shards by batch with no collective.
+"""
+import argparse
+import dataclasses
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "scale_steps_per_sec"
+UNIT = "scale-steps/s"
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="scalekv", choices=["scalekv", "reference"])
+    ap.add_argument("--workload", default="pass2b")
+    ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling on a small case)")
+    ap.add_argument("--full-cache", action="store_true", help="KEEP_ALL budgets instead of drafter/refiner budgets")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-side-stream", action="store_true")
+    ap.add_argument("--cpu-sample-slices", type=int, default=16)
+    return ap.parse_args()
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.25)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons, power = [], [], set(), []
+        for r in self.rows:
+            if len(r) < 7:
+                continue
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1])); power.append(float(r[2]))
+            except ValueError:
+                continue
+            for name, v in zip(["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"], r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_burst": p["bf16_tflops"], "bf16_sustained": p["bf16_tflops_sustained"],
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_burst": 1590.0, "bf16_sustained": 1400.0, "source": "fallback"}
+
+
+def workload_from_args(args):
+    from paper_2505_19602_b200 import synth
+
+    wl = synth.WORKLOADS[args.workload]
+    if args.layers:
+        nd = max(1, round(wl.n_drafters * args.layers / wl.n_layers)) if wl.n_drafters else 0
+        wl = dataclasses.replace(wl, n_layers=args.layers, n_drafters=nd)
+    return wl
+
+
+# --------------------------------------------------------------------------------------------
+# CPU oracle legs (cpu_baseline of the main line; the whole of --impl reference)
+# --------------------------------------------------------------------------------------------
+def oracle_threads():
+    try:
+        from threadpoolctl import threadpool_info
+
+        n = [i.get("num_threads", 1) for i in threadpool_info()]
+        return max(n) if n else 1
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def oracle_slice_pass(wl, layer, b, h, budgets, windows):
+    """One slice's full pass on the CPU oracle.  Returns seconds."""
+    import numpy as np
+
+    from oracle import scalekv_oracle as orc
+    from paper_2505_19602_b200 import synth
+
+    one = dataclasses.replace(wl)
+    cache = orc.SliceCache(wl.n_tokens, wl.head_dim)
+    data = []
+    for k in range(wl.n_scales):
+        Q, K, V = synth.scale_inputs(one, layer, k)
+        data.append(tuple(t[b, h].double().numpy() for t in (Q, K, V)))
+    t0 = time.perf_counter()
+    for k in range(wl.n_scales):
+        Q, K, V = data[k]
+        cache.append(K, V)
+        cache.attend(Q)
+        if k + 1 < wl.n_scales:
+            w = windows[k] if windows[k] is not None else list(range(wl.n_tokens[k]))
+            cache.compress(Q[w], w, budgets[layer][k])
+    return time.perf_counter() - t0
+
+
+def oracle_rate(wl, budgets, windows, n_sample):
+    """scale-steps/s of the oracle extrapolated from a sample of slices (slices are independent)."""
+    small = dataclasses.replace(wl, batch=1, n_heads=1)        # same per-slice shapes, cheap to generate
+    layers = sorted(set(round(i * (wl.n_layers - 1) / max(n_sample - 1, 1)) for i in range(n_sample)))
+    secs = [oracle_slice_pass(small, l, 0, 0, budgets, windows) for l in layers]
+    per_slice = sum(secs) / len(secs)
+    total = per_slice * wl.n_slices
+    return wl.n_scales / total, f"{len(layers)} slices (layers {layers}, batch 0, head 0), full {wl.n_scales}-scale pass each, " \
+                                f"{per_slice:.2f} s per slice-pass, extrapolated to {wl.n_slices} slices"
+
+
+def host_policy(wl, args):
+    """Budgets and windows.  Roles of the timed workloads come from scalekv_layer_stats when a GPU
+    is present; the reference arm (CPU only) uses the planted drafter layers directly."""
+    from oracle import scalekv_oracle as orc
+
+    windows = [orc.window_centroids(a, a, wl.window) for a in wl.sides]
+    return windows
+
+
+def reference_budgets(wl, full_cache):
+    from oracle import scalekv_oracle as orc
+    from paper_2505_19602_b200 import synth
+
+    if full_cache or wl.n_drafters == 0 and wl.name != "layer2b":
+        return [[orc.KEEP_ALL] * wl.n_scales for _ in range(wl.n_layers)]
+    n = wl.n_tokens
+    if wl.n_drafters == 0:
+        b = orc.budget_tokens(0.10, n)
+        return [[b] * wl.n_scales for _ in range(wl.n_layers)]
+    planted = set(synth.drafter_layers(wl))
+    bd, br = orc.budget_tokens(0.30, n), orc.budget_tokens(0.03, n)
+    return [[bd if l in planted else br] * wl.n_scales for l in range(wl.n_layers)]
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    wl = workload_from_args(args)
+    windows = host_policy(wl, args)
+    budgets = reference_budgets(wl, args.full_cache)
+    rates = []
+    note = ""
+    t_all = time.perf_counter()
+    for i in range(args.warmup + args.steps):
+        r, note = oracle_rate(wl, budgets, windows, 4)
+        if i >= args.warmup:
+            rates.append(r)
+    value = statistics.mean(rates)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1000.0 * wl.n_scales / value, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "layers": wl.n_layers, "batch": wl.batch, "heads": wl.n_heads, "head_dim": wl.head_dim,
+                   "scales": wl.n_scales, "budget": "full" if args.full_cache else "drafter 30% / refiner 3%"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
+                         "sample": "per step: " + note},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0, "wall_s": time.perf_counter() - t_all,
+    }
+    print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------------------------
+# CUDA arm
+# --------------------------------------------------------------------------------------------
+def run_scalekv(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2505_19602_b200 import binding, pipeline, synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU path")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    wl = workload_from_args(args)
+    if world > 1:
+        wl = dataclasses.replace(wl, seed=wl.seed + 1000 * rank)      # every rank owns a different batch
+    peaks = load_peaks()
+    windows = pipeline.windows_for(wl.sides, wl.window)
+
+    # budgets: drafter / refiner roles per scale from the offline statistics on seeded inputs
+    t0 = time.perf_counter()
+    if args.full_cache:
+        budgets = [[binding.KEEP_ALL] * wl.n_scales for _ in range(wl.n_layers)]
+        role_note = "full cache"
+    elif wl.n_drafters > 0:
+        asi, roles = pipeline.calibrate_roles(wl, wl.n_drafters, device=local_rank)
+        budgets = pipeline.budget_table(wl, roles)
+        planted = synth.drafter_layers(wl)
+        hits = sum(int(roles[l][k]) for k in range(1, wl.n_scales - 1) for l in planted)
+        role_note = f"{wl.n_drafters} drafters per scale from scalekv_layer_stats; {hits}/{len(planted) * (wl.n_scales - 2)} planted recovered"
+    else:
+        b = pipeline.pct_budget(10, 100, sum(wl.n_tokens[:-1]))
+        budgets = [[b] * wl.n_scales for _ in range(wl.n_layers)]
+        role_note = "uniform 10%"
+    calib_s = time.perf_counter() - t0
+
+    kv = binding.ScaleKV(wl.n_layers, wl.batch, wl.n_heads, wl.head_dim, wl.dtype, wl.sides, wl.sides, budgets,
+                         max_window=min(wl.window, binding.MAX_WINDOW), device=local_rank,
+                         side_stream=not args.no_side_stream)
+    inputs = pipeline.PassInputs(wl, device=local_rank)
+    work = pipeline.pass_work(wl, budgets, windows)
+    torch.cuda.synchronize()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed_passes(n_pass):
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(kv.stream_main):
+            ev0.record()
+        for _ in range(n_pass):
+            pipeline.run_pass(kv, inputs, windows)
+        kv.stream_main.wait_stream(kv.stream_side)
+        with torch.cuda.stream(kv.stream_main):
+            ev1.record()
+        kv.scalekv_sync()
+        return ev0.elapsed_time(ev1)
+
+    for _ in range(args.warmup):
+        pipeline.run_pass(kv, inputs, windows)
+    kv.scalekv_sync()
+    launches0 = kv.scalekv_launch_count()
+    sampler = ClockSampler(local_rank)
+    barrier()
+    sampler.start()
+    ms = timed_passes(args.steps)
+    barrier()
+    clocks = sampler.stop()
+    launches = kv.scalekv_launch_count() - launches0
+    if world > 1:
+        t = torch.tensor([ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    value = wl.n_scales * args.steps * world / (ms / 1000.0)
+
+    # per-kernel-class device time over the same number of passes, CUDA events on the launching streams
+    kv.scalekv_profile_enable(True)
+    for _ in range(args.steps):
+        pipeline.run_pass(kv, inputs, windows)
+    prof = kv.scalekv_profile_read()
+    kv.scalekv_profile_enable(False)
+    att_ms, att_n = prof["attend"]
+    att_tflops = work["attend_flop"] * args.steps / (att_ms / 1000.0) / 1e12 if att_ms > 0 else 0.0
+    peak_tf = peaks["bf16_sustained"] if wl.dtype == "bf16" else None
+    kernels = {}
+    for name, key in (("append", "append_bytes"), ("score", "score_bytes"), ("select", "select_bytes"), ("compact", "compact_bytes")):
+        kms, kn = prof[name]
+        gbs = work[key] * args.steps / (kms / 1000.0) / 1e9 if kms > 0 else 0.0
+        kernels[name] = {"ms_per_pass": kms / args.steps, "launches_per_pass": kn / args.steps, "algorithmic_GBps": gbs,
+                         "frac_of_hbm_peak": gbs / peaks["hbm_gbs"]}
+    kernels["attend"] = {"ms_per_pass": att_ms / args.steps, "launches_per_pass": att_n / args.steps, "TFLOPps": att_tflops}
+    roofline = {"bound": "tensor", "kernel": "attend", "achieved": att_tflops, "peak": peak_tf, "unit": "TFLOP/s",
+                "frac": (att_tflops / peak_tf) if peak_tf else None, "traffic": None,
+                "peak_source": f"{peaks['source']} bf16 sustained (kernel timed inside a long step)",
+                "avg_launch_ms": att_ms / max(att_n, 1)}
+    ser_ms = (work["attend_flop"] / (peaks["bf16_sustained"] * 1e12) +
+              (work["score_bytes"] + work["compact_bytes"] + work["append_bytes"] + work["select_bytes"]) / (peaks["hbm_gbs"] * 1e9)) * 1e3
+    pass_ms = ms / args.steps
+    roofline["pass_roofline_ms_serial"] = ser_ms
+    roofline["pass_frac_serial"] = ser_ms / pass_ms
+
+    # end to end from pinned host buffers through scalekv_step_host
+    e2e = None
+    if not args.no_e2e:
+        n_max = max(wl.n_tokens)
+        dt = synth.torch_dtype(wl.dtype)
+        host = {}
+        for k in range(wl.n_scales):
+            host[k] = tuple(t.cpu().pin_memory() for t in inputs.data[(0, k)])
+        Oh = torch.empty(wl.batch, wl.n_heads, n_max, wl.head_dim, dtype=dt).pin_memory()
+        staging = torch.empty(4 * wl.batch * wl.n_heads * n_max * wl.head_dim, dtype=dt, device="cuda")
+        torch.cuda.synchronize()
+
+        def e2e_pass():
+            kv.scalekv_reset()
+            for k in range(wl.n_scales):
+                nk = wl.n_tokens[k]
+                Qh, Kh, Vh = host[k]
+                last = k + 1 == wl.n_scales
+                for l in range(wl.n_layers):
+                    kv.scalekv_step_host(l, k, Qh, Kh, Vh, Oh, staging, window_pos=None if last else windows[k])
+                    kv.scalekv_sync()          # the host reads the step's output before the next layer
+        e2e_steps = max(1, min(args.steps, 3))
+        e2e_pass()
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            e2e_pass()
+        barrier()
+        e2e_s = time.perf_counter() - t0
+        if world > 1:
+            t = torch.tensor([e2e_s], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_s = float(t.item())
+        esz = 2 if wl.dtype == "bf16" else 4
+        tok_bytes = sum(wl.n_tokens) * wl.batch * wl.n_heads * wl.head_dim * esz * wl.n_layers
+        e2e = {"value": wl.n_scales * e2e_steps * world / e2e_s, "unit": UNIT, "h2d_bytes_per_step": 3 * tok_bytes,
+               "d2h_bytes_per_step": tok_bytes, "steps": e2e_steps,
+               "note": "pinned host Q/K/V -> device, append+attend+compress, O -> host, per layer and scale; "
+                       "layer 0's host tensors are reused for every layer"}
+        del staging
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        v, note = oracle_rate(wl, budgets, windows, args.cpu_sample_slices)
+        cpu = {"value": v, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle", "sample": note}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": pass_ms, "passes_per_sec": args.steps * world / (ms / 1000.0), "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
+            "config": {"workload": wl.name, "layers": wl.n_layers, "batch": wl.batch, "heads": wl.n_heads,
+                       "head_dim": wl.head_dim, "scales": wl.n_scales, "tokens": sum(wl.n_tokens),
+                       "budget": role_note, "window": wl.window, "parallelism": f"replica x{world} (batch-sharded, no collective)",
+                       "l2_policy": f"inputs larger than L2: {inputs.bytes() / 1e9:.1f} GB of Q/K/V per pass",
+                       "side_stream": not args.no_side_stream, "calibration_s": round(calib_s, 1),
+                       "attend_kernel": "tcgen05" if os.environ.get("SCALEKV_ATTEND", "") != "simt" else "simt"},
+            "roofline": roofline, "kernels": kernels, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches,
+            "clocks": clocks, "work_per_pass": {k: v for k, v in work.items() if k != "per_scale_flop"},
+        }
+        print(json.dumps(line))
+    kv.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_scalekv(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,212 @@
+/*
+ * scalekv.h - C ABI of the ScaleKV per-scale hot path for NVIDIA B200 (sm_100a).
+ *
+ * The library implements, with hand-written CUDA kernels, the step that scale-aware KV-cache
+ * compression (arXiv 2505.19602) adds to next-scale-prediction inference: for every scale k of
+ * the coarse-to-fine schedule and every transformer layer l,
+ *
+ *     append   : the K/V rows of the current token map r_k join the layer's cache, so that the
+ *                keys are P_{k-1} U C_k                                  (Sec. 1; Sec. 3.3, ASI paragraph)
+ *     attend   : O = softmax(Q K^T / sqrt(d)) V over every cache entry   (Sec. 3.3, Eq. 5)
+ *     compress : observation-window scores, top-k^l selection, pruning   (Sec. 3.3, "KV Cache Selection")
+ *
+ * plus the offline statistics that split layers into drafters and refiners (Sec. 3.3, Eq. 2-4).
+ *
+ * Conventions
+ *  - A "slice" is one (layer, batch, head) triple; slices never exchange data.
+ *  - Every function returns a scalekv_status.  Argument and call-order errors are reported
+ *    synchronously and leave the device untouched.  Device-side errors (a bounded wait that gave
+ *    up, a failed bounds check) are recorded in a sticky status word and returned by scalekv_sync.
+ *  - append / attend / compress only enqueue work on the caller's CUDA streams and return.
+ *  - Ownership: the caller owns the pool, the workspace, the streams and every tensor it passes.
+ *    The library owns only the host-side context.  It never allocates device memory after
+ *    scalekv_init and never falls back to the CPU: an unsupported (dtype, head_dim) pair is an error.
+ *  - Pointers are DEVICE pointers unless a parameter is documented as HOST.
+ *  - One context must be used by one host thread at a time.
+ */
+#ifndef SCALEKV_H
+#define SCALEKV_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct scalekv_ctx scalekv_ctx; /* opaque, host-side, library-owned */
+
+typedef enum {
+  SCALEKV_OK = 0,
+  SCALEKV_ERR_INVALID_ARG = 1,  /* null pointer, size out of range, misaligned tensor            */
+  SCALEKV_ERR_BAD_STATE = 2,    /* call out of order for this layer (append -> attend -> compress) */
+  SCALEKV_ERR_CAPACITY = 3,     /* pool or workspace smaller than scalekv_query_sizes reports     */
+  SCALEKV_ERR_UNSUPPORTED = 4,  /* (dtype, head_dim) not built: bf16 x 128 and f32 x 64 are        */
+  SCALEKV_ERR_CUDA = 5,         /* a CUDA runtime/driver call failed; text in scalekv_error_string */
+  SCALEKV_ERR_TIMEOUT = 6,      /* a bounded device-side wait gave up (reported by scalekv_sync)   */
+  SCALEKV_ERR_DEVICE_CHECK = 7  /* a device-side bounds check tripped (reported by scalekv_sync)   */
+} scalekv_status;
+
+typedef enum { SCALEKV_BF16 = 0, SCALEKV_F32 = 1 } scalekv_dtype;
+
+#define SCALEKV_KEEP_ALL (-1)   /* budget value: never evict                                       */
+#define SCALEKV_MAX_WINDOW 64   /* largest explicit observation window (a whole-map window is free) */
+#define SCALEKV_MAX_SCALES 32
+
+typedef struct {
+  int32_t n_layers, batch, n_heads, head_dim;
+  int32_t dtype;                 /* scalekv_dtype of Q, K, V, O and of the cache                    */
+  int32_t n_scales;
+  const int32_t *scale_h;        /* HOST [n_scales]: token-map heights h_k (copied)                 */
+  const int32_t *scale_w;        /* HOST [n_scales]: token-map widths  w_k (copied)                 */
+  const int32_t *budgets;        /* HOST [n_layers][n_scales]: k^l of the compress issued during    */
+                                 /* scale k = number of NON-window entries kept; SCALEKV_KEEP_ALL   */
+                                 /* or any value >= the candidates means no eviction (copied)       */
+  int32_t max_window;            /* upper bound on the explicit window size w, <= SCALEKV_MAX_WINDOW */
+  float softmax_scale;           /* 0 => 1/sqrt(head_dim) (Eq. 5)                                   */
+  int32_t page_tokens;           /* tokens per page; 0 => 128; must be a power of two >= 16         */
+  void *pool;                    /* device memory for pages, page tables and lengths (borrowed)     */
+  size_t pool_bytes;
+  void *workspace;               /* device scratch for scores, keep lists, statistics (borrowed)    */
+  size_t workspace_bytes;
+  void *stream_main;             /* cudaStream_t: append and attend run here                        */
+  void *stream_side;             /* cudaStream_t: compress runs here (may equal stream_main)        */
+  int32_t device;                /* CUDA device ordinal that owns pool, workspace and streams       */
+} scalekv_config;
+
+/* A [batch][n_heads][tokens][head_dim] tensor view: device pointer + ELEMENT strides; the
+ * innermost (head_dim) axis is contiguous and every row must start on a 16-byte boundary. */
+typedef struct {
+  const void *ptr;
+  int64_t stride_b, stride_h, stride_t;
+} scalekv_tensor;
+
+/* ---- life cycle ------------------------------------------------------------------------- */
+
+/* Bytes of pool and workspace that scalekv_init needs for this configuration (pointers in cfg
+ * are ignored).  The pool holds, per layer, ceil(cap_l / page_tokens) persistent pages per slice,
+ * cap_l being the largest cache a compress leaves behind, plus two transient page sets (even /
+ * odd layers) that hold the part of the current map that exceeds cap_l until that layer's
+ * compress; page tables; per-slice lengths.  No CUDA call is made. */
+scalekv_status scalekv_query_sizes(const scalekv_config *cfg, size_t *pool_bytes, size_t *workspace_bytes);
+
+/* Creates a context: copies schedule and budgets, carves the pool, uploads the page tables and
+ * zeroes the lengths (synchronous).  *out is NULL on failure. */
+scalekv_status scalekv_init(const scalekv_config *cfg, scalekv_ctx **out);
+
+/* Empties every slice (start of a new image batch).  Enqueued on stream_main after both streams'
+ * pending work. */
+scalekv_status scalekv_reset(scalekv_ctx *ctx);
+
+/* Waits for both streams and frees the host context.  Device memory stays with the caller. */
+scalekv_status scalekv_destroy(scalekv_ctx *ctx);
+
+/* ---- the hot path ------------------------------------------------------------------------ */
+
+/* Sec. 1 / Sec. 3.3: the current map joins the cache.  K and V are [B][H][n_k][d] views of the
+ * n_k = h_k * w_k rows of scale `scale` (0-based; scales must arrive in ascending order, once per
+ * layer).  Row i receives original position N_{k-1} + i.  The rows are copied; the caller may
+ * reuse its buffers once stream_main has passed this point.  Runs on stream_main after waiting
+ * for this layer's previous compress. */
+scalekv_status scalekv_append(scalekv_ctx *ctx, int32_t layer, int32_t scale, scalekv_tensor K, scalekv_tensor V);
+
+/* Eq. 5: O[b][h][i] = sum_j softmax_j(scale * <Q[b][h][i], K_j>) V_j over all L entries of the
+ * slice (history that survived earlier compressions, then the current map).  Q and O are
+ * [B][H][n_k][d] views in the configured dtype; lse (nullable) is a dense float [B][H][n_k]
+ * that receives max + log-sum-exp of the scaled logits.  bf16: products are exact, sums are
+ * fp32, P is rounded to bf16 before the PV product.  f32: plain fp32 FMA.  Runs on stream_main. */
+scalekv_status scalekv_attend(scalekv_ctx *ctx, int32_t layer, scalekv_tensor Q, scalekv_tensor O, float *lse);
+
+/* Sec. 3.3 "KV Cache Selection": with A = softmax(Q_W K^T * scale) over all L entries,
+ * s_i = (1/w) sum_{j in W} A_ji (Eq. 5, mean over the window rows, per head, fp32); the
+ * candidates are all entries that are not window entries; the k' = min(k^l, #candidates) best are
+ * kept (equal scores: lowest original position first) together with the w window entries; the
+ * survivors are moved to the front of the slice in ascending original position, in place.
+ *   Qw          window queries.  qw_is_full_map == 0: a [B][H][w][d] view whose row j is the query
+ *               at window_pos[j].  qw_is_full_map != 0: the [B][H][n_k][d] query tensor of the
+ *               current map; the library reads rows window_pos[j] itself.
+ *   w           window size, 1 <= w <= max_window; ignored when window_pos is NULL.
+ *   window_pos  HOST array [w] of distinct raster indices (r * w_k + c) inside the current map,
+ *               ascending, identical for every slice.  NULL means the window is the whole current
+ *               map (w = n_k; requires n_k <= SCALEKV_MAX_WINDOW and a dense Qw of n_k rows).
+ * k^l is budgets[layer][scale] of the scale last appended.  If nothing can be evicted the call
+ * only commits the lengths.  Runs on stream_side after this layer's attend. */
+scalekv_status scalekv_compress(scalekv_ctx *ctx, int32_t layer, scalekv_tensor Qw, int32_t w,
+                                const int32_t *window_pos, int32_t qw_is_full_map);
+
+/* One whole step for one layer from HOST memory (pinned memory recommended): copies Q, K, V
+ * (dense [B][H][n_k][d]) to `staging`, runs append, attend and compress with the window rows
+ * taken from Q (w > 0: explicit window_pos; w < 0: the whole map is the window; w == 0: no
+ * compress), and copies O back to O_host.  staging is device memory of at least
+ * 4 * B*H*n_k*d elements.  Everything is enqueued on the context's streams; the host buffers must
+ * stay valid until scalekv_sync. */
+scalekv_status scalekv_step_host(scalekv_ctx *ctx, int32_t layer, int32_t scale, const void *Q_host,
+                                 const void *K_host, const void *V_host, void *O_host, void *staging,
+                                 size_t staging_bytes, int32_t w, const int32_t *window_pos);
+
+/* ---- offline statistics and host-side policy (Sec. 3.3, Eq. 2-4) --------------------------- */
+
+/* Eq. 2 for the scale last appended to `layer` (call after append, cache uncompressed): for every
+ * query row i = 0, query_stride, 2*query_stride, ... of Q and every slice, alpha_i = softmax row
+ * over all entries; c_i = mass on the current map; t_i = sum of the min(K', |history|) largest
+ * alpha_ij over the history.  *car and *htk (HOST) receive the means of c_i and t_i over rows and
+ * slices; ASI = car * htk.  Synchronous; not part of the timed path.  topk_prime <= 64. */
+scalekv_status scalekv_layer_stats(scalekv_ctx *ctx, int32_t layer, scalekv_tensor Q, int32_t topk_prime,
+                                   int32_t query_stride, double *car, double *htk);
+
+/* Sec. 3.3: the observation window = centroid token of each of N patches of an h x w map.
+ * g = floor(sqrt(N)) patches per side, patch (a,b) = rows [a*h/g, (a+1)*h/g) x cols alike, centroid =
+ * lower-middle cell; a map with at most N tokens is its own window.  pos (HOST, room for N entries)
+ * receives ascending raster indices, *count their number.  Host only. */
+scalekv_status scalekv_window_centroids(int32_t h, int32_t w, int32_t n_patches, int32_t *pos, int32_t *count);
+
+/* Eq. 3: Z = (ASI - mu_k) / (sigma_k + eps) per scale over layers (population sigma); drafters are
+ * the pairs with the lowest Z.  asi HOST [L][K] row-major.  mode 0: the n_drafters lowest pairs over
+ * all ranked (layer, scale) pairs; mode 1: the n_drafters lowest layers at every ranked scale.
+ * Scales 0 and K-1 are not ranked (no history / nothing follows).  Ties: lower scale, then lower
+ * layer.  is_drafter HOST [L][K] receives 0/1.  Host only. */
+scalekv_status scalekv_assign_roles(const double *asi, int32_t L, int32_t K, int32_t n_drafters, int32_t mode,
+                                    double eps, uint8_t *is_drafter);
+
+/* Eq. 4: B_r(k) = max(B_r(0) - delta * k, 0) for k = 1..K; per scale N_d^k B_d(k) + N_r^k B_r(k) =
+ * B_uniform * L, which sums to the printed constraint; a scale without drafters gets B_uniform
+ * everywhere; values rounded half up.  budgets_out HOST [L][K].  Host only. */
+scalekv_status scalekv_make_budgets(const uint8_t *is_drafter, int32_t L, int32_t K, double b_uniform, double b_r0,
+                                    double delta, int32_t *budgets_out);
+
+/* ---- introspection ------------------------------------------------------------------------ */
+
+/* Current number of entries of every slice of a layer -> len_host HOST [B][H].  Synchronous. */
+scalekv_status scalekv_lengths(scalekv_ctx *ctx, int32_t layer, int32_t *len_host);
+
+/* Copies one slice to the host: original positions (pos_host [cap]), and, if non-NULL, its K and V
+ * rows ([cap][d] in the configured dtype).  *len receives the entry count; fails with CAPACITY if it
+ * exceeds cap.  Synchronous.  Rows beyond the layer's persistent capacity live in pages shared with
+ * other layers and are only meaningful until the layer after next appends. */
+scalekv_status scalekv_export_slice(scalekv_ctx *ctx, int32_t layer, int32_t b, int32_t h, int32_t *pos_host,
+                                    void *K_host, void *V_host, int32_t cap, int32_t *len);
+
+/* Importance scores of one slice as left by the most recent evicting compress (any layer):
+ * s_host HOST [cap] floats indexed by the slot order BEFORE that compress.  Synchronous. */
+scalekv_status scalekv_export_scores(scalekv_ctx *ctx, int32_t b, int32_t h, float *s_host, int32_t cap, int32_t *len);
+
+/* Waits for both streams; returns the sticky device status (OK, TIMEOUT or DEVICE_CHECK). */
+scalekv_status scalekv_sync(scalekv_ctx *ctx);
+
+/* Number of kernels this context has launched since scalekv_init (HOST out). */
+scalekv_status scalekv_launch_count(scalekv_ctx *ctx, int64_t *count);
+
+/* Per-kernel-class device timing.  While enabled, every launch is bracketed by CUDA events on the
+ * stream it runs on.  scalekv_profile_read waits for both streams and returns, for class `which`
+ * (0 append, 1 attend, 2 score, 3 select, 4 compact, 5 other), the summed milliseconds and the
+ * number of launches since profiling was last enabled. */
+scalekv_status scalekv_profile_enable(scalekv_ctx *ctx, int32_t on);
+scalekv_status scalekv_profile_read(scalekv_ctx *ctx, int32_t which, double *ms_total, int64_t *launches);
+
+/* Text of the last error of this context (never NULL; valid until the next call). */
+const char *scalekv_error_string(scalekv_ctx *ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SCALEKV_H */

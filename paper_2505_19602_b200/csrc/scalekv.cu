@@ -1,0 +1,760 @@
+// Host runtime and C ABI of the ScaleKV hot path (see include/scalekv.h for the contract).
+// The context plans the paged store, tracks the per-layer call order and lengths, orders the two
+// streams with events and launches the kernels.  Nothing here computes on the CPU.
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <string>
+#include <vector>
+
+#include "../../include/scalekv.h"
+#include "attend_tc.cuh"
+#include "kernels_simt.cuh"
+
+using namespace scalekv;
+
+namespace {
+
+constexpr int kNumClasses = 6;
+enum KernelClass { kAppend = 0, kAttend = 1, kScore = 2, kSelect = 3, kCompact = 4, kOther = 5 };
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct LayerPlan {
+  int cap = 0;            // largest cache a compress can leave behind
+  int max_len = 0;        // largest cache during any step
+  int persist_pages = 0;  // pages owned by each slice of this layer
+  int total_pages = 0;    // logical pages per slice (persistent + transient)
+  size_t page_table_off = 0;  // element offset into the page-table area
+  int first_page = 0;         // first persistent page id
+};
+
+struct Plan {
+  int n_layers, B, H, d, esize, K, P, page_shift, n_slices, max_window;
+  std::vector<int> n, N;            // tokens per scale, cumulative (N[0] = 0)
+  std::vector<int> budgets;         // [layers][K]
+  std::vector<LayerPlan> layers;
+  int trans_pages_per_slice = 0;    // size of one transient set per slice
+  int trans_first[2] = {0, 0};
+  long long n_pages = 0;
+  int ld_s = 0;                     // padded max length (leading dimension of per-slice scratch)
+  int n_max = 0;
+  // pool layout (byte offsets)
+  size_t off_k, off_v, off_pos, off_pt, off_len, off_status, pool_bytes;
+  size_t pt_elems;
+  // workspace layout
+  size_t off_logits, off_scores, off_keys, off_keep, off_kept, off_acc, off_qw, ws_bytes;
+};
+
+scalekv_status make_plan(const scalekv_config *c, Plan &p, std::string &err) {
+  if (!c || !c->scale_h || !c->scale_w || !c->budgets) { err = "null config field"; return SCALEKV_ERR_INVALID_ARG; }
+  if (c->n_layers < 1 || c->batch < 1 || c->n_heads < 1 || c->n_scales < 1 || c->n_scales > SCALEKV_MAX_SCALES) {
+    err = "n_layers, batch, n_heads >= 1 and 1 <= n_scales <= 32 required"; return SCALEKV_ERR_INVALID_ARG;
+  }
+  if (c->max_window < 1 || c->max_window > SCALEKV_MAX_WINDOW) { err = "max_window out of range"; return SCALEKV_ERR_INVALID_ARG; }
+  if (!((c->dtype == SCALEKV_BF16 && c->head_dim == 128) || (c->dtype == SCALEKV_F32 && c->head_dim == 64))) {
+    err = "unsupported (dtype, head_dim): bf16 x 128 and f32 x 64 are built"; return SCALEKV_ERR_UNSUPPORTED;
+  }
+  p.n_layers = c->n_layers; p.B = c->batch; p.H = c->n_heads; p.d = c->head_dim;
+  p.esize = c->dtype == SCALEKV_BF16 ? 2 : 4;
+  p.K = c->n_scales; p.max_window = c->max_window;
+  p.P = c->page_tokens == 0 ? 128 : c->page_tokens;
+  if (p.P < 16 || (p.P & (p.P - 1))) { err = "page_tokens must be a power of two >= 16"; return SCALEKV_ERR_INVALID_ARG; }
+  p.page_shift = 0; while ((1 << p.page_shift) < p.P) ++p.page_shift;
+  p.n_slices = p.B * p.H;
+  p.n.resize(p.K); p.N.assign(p.K + 1, 0);
+  p.n_max = 0;
+  for (int k = 0; k < p.K; ++k) {
+    if (c->scale_h[k] < 1 || c->scale_w[k] < 1) { err = "scale sides must be >= 1"; return SCALEKV_ERR_INVALID_ARG; }
+    p.n[k] = c->scale_h[k] * c->scale_w[k];
+    p.N[k + 1] = p.N[k] + p.n[k];
+    p.n_max = std::max(p.n_max, p.n[k]);
+  }
+  p.budgets.assign(c->budgets, c->budgets + (size_t)p.n_layers * p.K);
+  p.layers.resize(p.n_layers);
+  int trans_max = 0, len_max = 0;
+  size_t pt = 0;
+  long long page = 0;
+  for (int l = 0; l < p.n_layers; ++l) {
+    LayerPlan &lp = p.layers[l];
+    int hist = 0;
+    for (int k = 0; k < p.K; ++k) {
+      const int L = hist + p.n[k];
+      lp.max_len = std::max(lp.max_len, L);
+      const int bud = p.budgets[(size_t)l * p.K + k];
+      if (bud < SCALEKV_KEEP_ALL) { err = "budget < -1"; return SCALEKV_ERR_INVALID_ARG; }
+      const int wmax = std::min(p.max_window, p.n[k]);
+      const long long kept = bud == SCALEKV_KEEP_ALL ? L : std::min<long long>(L, (long long)bud + wmax);
+      hist = (int)kept;
+      lp.cap = std::max(lp.cap, hist);
+    }
+    lp.total_pages = (lp.max_len + p.P - 1) / p.P;
+    lp.persist_pages = std::min(lp.total_pages, (lp.cap + p.P - 1) / p.P);
+    lp.page_table_off = pt;
+    pt += (size_t)p.n_slices * lp.total_pages;
+    lp.first_page = (int)page;
+    page += (long long)p.n_slices * lp.persist_pages;
+    trans_max = std::max(trans_max, lp.total_pages - lp.persist_pages);
+    len_max = std::max(len_max, lp.max_len);
+  }
+  p.trans_pages_per_slice = trans_max;
+  p.trans_first[0] = (int)page; page += (long long)p.n_slices * trans_max;
+  p.trans_first[1] = (int)page; page += (long long)p.n_slices * trans_max;
+  if (page > 0x7fffffffLL / p.P) { err = "store too large for 32-bit row indices"; return SCALEKV_ERR_CAPACITY; }
+  p.n_pages = page;
+  p.pt_elems = pt;
+  p.ld_s = (int)align_up((size_t)len_max, 64);
+  const size_t row_bytes = (size_t)p.d * p.esize;
+  size_t o = 0;
+  p.off_k = o; o = align_up(o + (size_t)p.n_pages * p.P * row_bytes, 1024);
+  p.off_v = o; o = align_up(o + (size_t)p.n_pages * p.P * row_bytes, 1024);
+  p.off_pos = o; o = align_up(o + (size_t)p.n_pages * p.P * 4, 1024);
+  p.off_pt = o; o = align_up(o + pt * 4, 1024);
+  p.off_len = o; o = align_up(o + (size_t)p.n_layers * p.n_slices * 4, 1024);
+  p.off_status = o; o = align_up(o + 256, 1024);
+  p.pool_bytes = o;
+  o = 0;
+  p.off_logits = o; o = align_up(o + (size_t)p.n_slices * p.max_window * p.ld_s * 4, 1024);
+  p.off_scores = o; o = align_up(o + (size_t)p.n_slices * p.ld_s * 4, 1024);
+  p.off_keys = o; o = align_up(o + (size_t)p.n_slices * p.ld_s * 4, 1024);
+  p.off_keep = o; o = align_up(o + (size_t)p.n_slices * p.ld_s * 4, 1024);
+  p.off_kept = o; o = align_up(o + (size_t)p.n_slices * 4, 1024);
+  p.off_acc = o; o = align_up(o + 64, 1024);
+  p.off_qw = o; o = align_up(o + (size_t)p.n_slices * p.max_window * row_bytes, 1024);
+  p.ws_bytes = o;
+  return SCALEKV_OK;
+}
+
+}  // namespace
+
+struct scalekv_ctx {
+  Plan plan;
+  int device = 0;
+  int dtype = 0;
+  float scale = 0.f;
+  char *pool = nullptr, *ws = nullptr;
+  cudaStream_t s_main = nullptr, s_side = nullptr;
+  std::vector<int> page_table_host;
+  // per layer state
+  std::vector<int> next_scale;     // scale expected by the next append
+  std::vector<int> hist;           // entries before the current map (uniform over slices)
+  std::vector<int> pending;        // n_k of an appended, not yet committed current map (0 = none)
+  std::vector<int> attended;       // attend ran for the pending map
+  std::vector<cudaEvent_t> ev_attend, ev_compress;
+  std::vector<char> ev_compress_live;
+  int64_t launches = 0;
+  int scores_len = 0;              // length of the score vectors left by the last evicting compress
+  bool profile = false;
+  struct Timed { cudaEvent_t a, b; int cls; };
+  std::vector<Timed> timed;
+  std::vector<cudaEvent_t> event_pool;
+  double prof_ms[kNumClasses] = {0};
+  int64_t prof_n[kNumClasses] = {0};
+  std::string err = "ok";
+  AttendTc tc;
+};
+
+namespace {
+
+scalekv_status fail(scalekv_ctx *c, scalekv_status st, const char *fmt, ...) {
+  char buf[512];
+  va_list ap; va_start(ap, fmt); vsnprintf(buf, sizeof buf, fmt, ap); va_end(ap);
+  if (c) c->err = buf;
+  return st;
+}
+
+#define CU(call)                                                                                   \
+  do {                                                                                             \
+    cudaError_t e_ = (call);                                                                       \
+    if (e_ != cudaSuccess) return fail(ctx, SCALEKV_ERR_CUDA, "%s: %s", #call, cudaGetErrorString(e_)); \
+  } while (0)
+
+LayerView layer_view(scalekv_ctx *c, int l) {
+  const Plan &p = c->plan;
+  LayerView lv;
+  lv.k_pool = c->pool + p.off_k;
+  lv.v_pool = c->pool + p.off_v;
+  lv.pos_pool = reinterpret_cast<int *>(c->pool + p.off_pos);
+  lv.page_table = reinterpret_cast<const int *>(c->pool + p.off_pt) + p.layers[l].page_table_off;
+  lv.hist_len = reinterpret_cast<int *>(c->pool + p.off_len) + (size_t)l * p.n_slices;
+  lv.status = reinterpret_cast<int *>(c->pool + p.off_status);
+  lv.pages_per_slice = p.layers[l].total_pages;
+  lv.page_shift = p.page_shift;
+  lv.page_mask = p.P - 1;
+  lv.row_bytes = p.d * p.esize;
+  lv.n_slices = p.n_slices;
+  lv.n_heads = p.H;
+  return lv;
+}
+
+TensorView tview(const scalekv_tensor &t) {
+  TensorView v; v.ptr = static_cast<const char *>(t.ptr); v.sb = t.stride_b; v.sh = t.stride_h; v.st = t.stride_t;
+  return v;
+}
+
+bool tensor_ok(const scalekv_tensor &t, int esize) {
+  if (!t.ptr) return false;
+  if (reinterpret_cast<uintptr_t>(t.ptr) & 15) return false;
+  return ((t.stride_b * esize) % 16 == 0) && ((t.stride_h * esize) % 16 == 0) && ((t.stride_t * esize) % 16 == 0);
+}
+
+struct Scope {  // brackets one launch with events when profiling; counts launches
+  scalekv_ctx *c; cudaStream_t s; int cls; cudaEvent_t a = nullptr, b = nullptr;
+  Scope(scalekv_ctx *c_, cudaStream_t s_, int cls_) : c(c_), s(s_), cls(cls_) {
+    if (c->profile) {
+      a = take(); b = take();
+      cudaEventRecord(a, s);
+    }
+  }
+  cudaEvent_t take() {
+    if (!c->event_pool.empty()) { cudaEvent_t e = c->event_pool.back(); c->event_pool.pop_back(); return e; }
+    cudaEvent_t e; cudaEventCreate(&e); return e;
+  }
+  ~Scope() {
+    c->launches++;
+    if (c->profile) { cudaEventRecord(b, s); c->timed.push_back({a, b, cls}); }
+  }
+};
+
+void drain_profile(scalekv_ctx *c) {
+  for (auto &t : c->timed) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, t.a, t.b) == cudaSuccess) { c->prof_ms[t.cls] += ms; c->prof_n[t.cls]++; }
+    c->event_pool.push_back(t.a); c->event_pool.push_back(t.b);
+  }
+  c->timed.clear();
+}
+
+template <typename F> void set_smem(F *f, size_t bytes) {
+  cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+}
+
+scalekv_status check_launch(scalekv_ctx *ctx, const char *what) {
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(ctx, SCALEKV_ERR_CUDA, "launch of %s failed: %s", what, cudaGetErrorString(e));
+  return SCALEKV_OK;
+}
+
+scalekv_status commit_pending(scalekv_ctx *ctx, int l, cudaStream_t s) {
+  if (ctx->pending[l] == 0) return SCALEKV_OK;
+  const Plan &p = ctx->plan;
+  const int L = ctx->hist[l] + ctx->pending[l];
+  if (L > p.layers[l].persist_pages * p.P && p.layers[l].persist_pages < p.layers[l].total_pages)
+    return fail(ctx, SCALEKV_ERR_CAPACITY, "layer %d: %d entries kept without compress exceed the persistent capacity %d",
+                l, L, p.layers[l].persist_pages * p.P);
+  {
+    Scope sc(ctx, s, kOther);
+    commit_kernel<<<(p.n_slices + 255) / 256, 256, 0, s>>>(layer_view(ctx, l), ctx->pending[l]);
+  }
+  ctx->hist[l] = L;
+  ctx->pending[l] = 0;
+  ctx->attended[l] = 0;
+  return check_launch(ctx, "commit");
+}
+
+scalekv_status fill_window(scalekv_ctx *ctx, int l, int w, const int32_t *window_pos, WindowArg &wa) {
+  const Plan &p = ctx->plan;
+  const int k = ctx->next_scale[l] - 1;
+  wa.n_prev = p.N[k];
+  wa.n_k = p.n[k];
+  if (window_pos == nullptr) {
+    if (wa.n_k > p.max_window) return fail(ctx, SCALEKV_ERR_INVALID_ARG, "whole-map window needs n_k <= max_window");
+    wa.w = wa.n_k; wa.all = 1;
+    for (int j = 0; j < wa.w; ++j) wa.pos[j] = j;
+  } else {
+    if (w < 1 || w > p.max_window || w > wa.n_k) return fail(ctx, SCALEKV_ERR_INVALID_ARG, "window size %d out of range", w);
+    wa.w = w; wa.all = 0;
+    for (int j = 0; j < w; ++j) {
+      if (window_pos[j] < 0 || window_pos[j] >= wa.n_k || (j > 0 && window_pos[j] <= window_pos[j - 1]))
+        return fail(ctx, SCALEKV_ERR_INVALID_ARG, "window_pos must be ascending, distinct and inside the current map");
+      wa.pos[j] = window_pos[j];
+    }
+  }
+  for (int j = wa.w; j < kMaxWindow; ++j) wa.pos[j] = 0x7fffffff;
+  return SCALEKV_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+scalekv_status scalekv_query_sizes(const scalekv_config *cfg, size_t *pool_bytes, size_t *workspace_bytes) {
+  Plan p; std::string err;
+  scalekv_status st = make_plan(cfg, p, err);
+  if (st != SCALEKV_OK) return st;
+  if (pool_bytes) *pool_bytes = p.pool_bytes;
+  if (workspace_bytes) *workspace_bytes = p.ws_bytes;
+  return SCALEKV_OK;
+}
+
+scalekv_status scalekv_init(const scalekv_config *cfg, scalekv_ctx **out) {
+  if (!out) return SCALEKV_ERR_INVALID_ARG;
+  *out = nullptr;
+  scalekv_ctx *ctx = new scalekv_ctx();
+  std::string err;
+  scalekv_status st = make_plan(cfg, ctx->plan, err);
+  if (st != SCALEKV_OK) { delete ctx; return st; }
+  const Plan &p = ctx->plan;
+  if (!cfg->pool || !cfg->workspace) { delete ctx; return SCALEKV_ERR_INVALID_ARG; }
+  if (cfg->pool_bytes < p.pool_bytes || cfg->workspace_bytes < p.ws_bytes) { delete ctx; return SCALEKV_ERR_CAPACITY; }
+  if ((reinterpret_cast<uintptr_t>(cfg->pool) & 1023) || (reinterpret_cast<uintptr_t>(cfg->workspace) & 255)) {
+    delete ctx; return SCALEKV_ERR_INVALID_ARG;
+  }
+  ctx->device = cfg->device; ctx->dtype = cfg->dtype;
+  ctx->scale = cfg->softmax_scale != 0.f ? cfg->softmax_scale : 1.0f / std::sqrt((float)cfg->head_dim);
+  ctx->pool = static_cast<char *>(cfg->pool); ctx->ws = static_cast<char *>(cfg->workspace);
+  ctx->s_main = static_cast<cudaStream_t>(cfg->stream_main);
+  ctx->s_side = cfg->stream_side ? static_cast<cudaStream_t>(cfg->stream_side) : ctx->s_main;
+  auto bail = [&](scalekv_status s) { delete ctx; return s; };
+  if (cudaSetDevice(cfg->device) != cudaSuccess) return bail(SCALEKV_ERR_CUDA);
+  int major = 0, minor = 0;
+  cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, cfg->device);
+  cudaDeviceGetAttribute(&minor, cudaDevAttrComputeCapabilityMinor, cfg->device);
+  if (major != 10) return bail(SCALEKV_ERR_UNSUPPORTED);
+  // page tables: persistent pages first, then the transient set of the layer's parity
+  ctx->page_table_host.resize(p.pt_elems);
+  for (int l = 0; l < p.n_layers; ++l) {
+    const LayerPlan &lp = p.layers[l];
+    for (int s = 0; s < p.n_slices; ++s)
+      for (int j = 0; j < lp.total_pages; ++j) {
+        int page = j < lp.persist_pages
+                       ? lp.first_page + s * lp.persist_pages + j
+                       : p.trans_first[l & 1] + s * p.trans_pages_per_slice + (j - lp.persist_pages);
+        ctx->page_table_host[lp.page_table_off + (size_t)s * lp.total_pages + j] = page;
+      }
+  }
+  if (cudaMemcpy(ctx->pool + p.off_pt, ctx->page_table_host.data(), p.pt_elems * 4, cudaMemcpyHostToDevice) != cudaSuccess)
+    return bail(SCALEKV_ERR_CUDA);
+  if (cudaMemset(ctx->pool + p.off_len, 0, (size_t)p.n_layers * p.n_slices * 4) != cudaSuccess) return bail(SCALEKV_ERR_CUDA);
+  if (cudaMemset(ctx->pool + p.off_status, 0, 256) != cudaSuccess) return bail(SCALEKV_ERR_CUDA);
+  ctx->next_scale.assign(p.n_layers, 0);
+  ctx->hist.assign(p.n_layers, 0);
+  ctx->pending.assign(p.n_layers, 0);
+  ctx->attended.assign(p.n_layers, 0);
+  ctx->ev_attend.resize(p.n_layers); ctx->ev_compress.resize(p.n_layers);
+  ctx->ev_compress_live.assign(p.n_layers, 0);
+  for (int l = 0; l < p.n_layers; ++l) {
+    if (cudaEventCreateWithFlags(&ctx->ev_attend[l], cudaEventDisableTiming) != cudaSuccess) return bail(SCALEKV_ERR_CUDA);
+    if (cudaEventCreateWithFlags(&ctx->ev_compress[l], cudaEventDisableTiming) != cudaSuccess) return bail(SCALEKV_ERR_CUDA);
+  }
+  if (cfg->dtype == SCALEKV_BF16) {
+    set_smem(attend_simt_kernel<__nv_bfloat16, 128>, (64 * 132 * 2 + 64 * 65 + 192) * 4);
+    set_smem(score_logits_kernel<__nv_bfloat16, 128>, 2 * 64 * 132 * 4);
+    set_smem(layer_stats_kernel<__nv_bfloat16, 128>, (size_t)(128 + p.ld_s) * 4);
+  } else {
+    set_smem(attend_simt_kernel<float, 64>, (64 * 68 * 2 + 64 * 65 + 192) * 4);
+    set_smem(score_logits_kernel<float, 64>, 2 * 64 * 68 * 4);
+    set_smem(layer_stats_kernel<float, 64>, (size_t)(64 + p.ld_s) * 4);
+  }
+  cudaGetLastError();
+  std::string tc_err;
+  if (!ctx->tc.init(cfg->dtype, p.d, ctx->pool + p.off_k, ctx->pool + p.off_v, p.n_pages, p.P, tc_err)) {
+    scalekv_status s = fail(ctx, SCALEKV_ERR_CUDA, "tensor-core attend set-up failed: %s", tc_err.c_str());
+    fprintf(stderr, "scalekv_init: %s\n", ctx->err.c_str());
+    return bail(s);
+  }
+  *out = ctx;
+  return SCALEKV_OK;
+}
+
+scalekv_status scalekv_reset(scalekv_ctx *ctx) {
+  if (!ctx) return SCALEKV_ERR_INVALID_ARG;
+  const Plan &p = ctx->plan;
+  if (ctx->s_side != ctx->s_main) {
+    cudaEvent_t e = ctx->ev_compress[0];
+    CU(cudaEventRecord(e, ctx->s_side));
+    CU(cudaStreamWaitEvent(ctx->s_main, e, 0));
+  }
+  CU(cudaMemsetAsync(ctx->pool + p.off_len, 0, (size_t)p.n_layers * p.n_slices * 4, ctx->s_main));
+  if (ctx->s_side != ctx->s_main) {
+    // later side-stream work must not overtake the reset
+    CU(cudaEventRecord(ctx->ev_attend[0], ctx->s_main));
+    CU(cudaStreamWaitEvent(ctx->s_side, ctx->ev_attend[0], 0));
+  }
+  std::fill(ctx->next_scale.begin(), ctx->next_scale.end(), 0);
+  std::fill(ctx->hist.begin(), ctx->hist.end(), 0);
+  std::fill(ctx->pending.begin(), ctx->pending.end(), 0);
+  std::fill(ctx->attended.begin(), ctx->attended.end(), 0);
+  std::fill(ctx->ev_compress_live.begin(), ctx->ev_compress_live.end(), 0);
+  return SCALEKV_OK;
+}
+
+scalekv_status scalekv_destroy(scalekv_ctx *ctx) {
+  if (!ctx) return SCALEKV_ERR_INVALID_ARG;
+  cudaStreamSynchronize(ctx->s_main);
+  if (ctx->s_side != ctx->s_main) cudaStreamSynchronize(ctx->s_side);
+  drain_profile(ctx);
+  for (auto e : ctx->ev_attend) cudaEventDestroy(e);
+  for (auto e : ctx->ev_compress) cudaEventDestroy(e);
+  for (auto e : ctx->event_pool) cudaEventDestroy(e);
+  delete ctx;
+  return SCALEKV_OK;
+}
+
+scalekv_status scalekv_append(scalekv_ctx *ctx, int32_t layer, int32_t scale, scalekv_tensor K, scalekv_tensor V) {
+  if (!ctx) return SCALEKV_ERR_INVALID_ARG;
+  const Plan &p = ctx->plan;
+  if (layer < 0 || layer >= p.n_layers) return fail(ctx, SCALEKV_ERR_INVALID_ARG, "layer %d out of range", layer);
+  if (scale < 0 || scale >= p.K) return fail(ctx, SCALEKV_ERR_INVALID_ARG, "scale %d out of range", scale);
+  if (scale != ctx->next_scale[layer])
+    return fail(ctx, SCALEKV_ERR_BAD_STATE, "layer %d expects scale %d, got %d", layer, ctx->next_scale[layer], scale);
+  if (!tensor_ok(K, p.esize) || !tensor_ok(V, p.esize)) return fail(ctx, SCALEKV_ERR_INVALID_ARG, "K/V null or rows not 16-byte aligned");
+  // the previous compress of this layer, and the compress of the layer that last used the same
+  // transient page set, must have finished
+  if (ctx->s_side != ctx->s_main) {
+    if (ctx->ev_compress_live[layer]) CU(cudaStreamWaitEvent(ctx->s_main, ctx->ev_compress[layer], 0));
+    const int other = layer >= 2 ? layer - 2 : -1;
+    if (other >= 0 && ctx->ev_compress_live[other]) CU(cudaStreamWaitEvent(ctx->s_main, ctx->ev_compress[other], 0));
+    if (layer < 2 && scale > 0) {
+      // transient set reuse across scales: the last layer of this parity at the previous scale
+      for (int o = p.n_layers - 1; o >= 0; --o)
+        if ((o & 1) == (layer & 1)) { if (ctx->ev_compress_live[o]) CU(cudaStreamWaitEvent(ctx->s_main, ctx->ev_compress[o], 0)); break; }
+    }
+  }
+  scalekv_status st = commit_pending(ctx, layer, ctx->s_main);
+  if (st != SCALEKV_OK) return st;
+  const int nk = p.n[scale];
+  if (ctx->hist[layer] + nk > p.layers[layer].total_pages * p.P)
+    return fail(ctx, SCALEKV_ERR_CAPACITY, "layer %d: %d + %d entries exceed the planned capacity", layer, ctx->hist[layer], nk);
+  {
+    Scope sc(ctx, ctx->s_main, kAppend);
+    dim3 grid((nk + 63) / 64, p.n_slices);
+    append_kernel<<<grid, 256, 0, ctx->s_main>>>(layer_view(ctx, layer), tview(K), tview(V), nk, p.N[scale], p.esize);
+  }
+  ctx->pending[layer] = nk;
+  ctx->attended[layer] = 0;
+  ctx->next_scale[layer] = scale + 1;
+  return check_launch(ctx, "append");
+}
+
+scalekv_status scalekv_attend(scalekv_ctx *ctx, int32_t layer, scalekv_tensor Q, scalekv_tensor O, float *lse) {
+  if (!ctx) return SCALEKV_ERR_INVALID_ARG;
+  const Plan &p = ctx->plan;
+  if (layer < 0 || layer >= p.n_layers) return fail(ctx, SCALEKV_ERR_INVALID_ARG, "layer %d out of range", layer);
+  if (ctx->pending[layer] == 0) return fail(ctx, SCALEKV_ERR_BAD_STATE, "layer %d: attend needs a preceding append", layer);
+  if (!tensor_ok(Q, p.esize) || !tensor_ok(O, p.esize)) return fail(ctx, SCALEKV_ERR_INVALID_ARG, "Q/O null or rows not 16-byte aligned");
+  const int nk = ctx->pending[layer];
+  LayerView lv = layer_view(ctx, layer);
+  {
+    Scope sc(ctx, ctx->s_main, kAttend);
+    if (ctx->tc.enabled()) {
+      std::string e;
+      if (!ctx->tc.launch(lv, tview(Q), tview(O), lse, nk, ctx->hist[layer] + nk, ctx->scale, ctx->s_main, e))
+        return fail(ctx, SCALEKV_ERR_CUDA, "attend launch: %s", e.c_str());
+    } else {
+      dim3 grid((nk + 63) / 64, p.n_slices);
+      if (ctx->dtype == SCALEKV_BF16)
+        attend_simt_kernel<__nv_bfloat16, 128><<<grid, 256, (64 * 132 * 2 + 64 * 65 + 192) * 4, ctx->s_main>>>(
+            lv, tview(Q), tview(O), lse, nk, ctx->scale);
+      else
+        attend_simt_kernel<float, 64><<<grid, 256, (64 * 68 * 2 + 64 * 65 + 192) * 4, ctx->s_main>>>(
+            lv, tview(Q), tview(O), lse, nk, ctx->scale);
+    }
+  }
+  ctx->attended[layer] = 1;
+  if (ctx->s_side != ctx->s_main) CU(cudaEventRecord(ctx->ev_attend[layer], ctx->s_main));
+  return check_launch(ctx, "attend");
+}
+
+scalekv_status scalekv_compress(scalekv_ctx *ctx, int32_t layer, scalekv_tensor Qw, int32_t w, const int32_t *window_pos,
+                                int32_t qw_is_full_map) {
+  if (!ctx) return SCALEKV_ERR_INVALID_ARG;
+  const Plan &p = ctx->plan;
+  if (layer < 0 || layer >= p.n_layers) return fail(ctx, SCALEKV_ERR_INVALID_ARG, "layer %d out of range", layer);
+  if (ctx->pending[layer] == 0) return fail(ctx, SCALEKV_ERR_BAD_STATE, "layer %d: compress needs a preceding append", layer);
+  if (!tensor_ok(Qw, p.esize)) return fail(ctx, SCALEKV_ERR_INVALID_ARG, "Qw null or rows not 16-byte aligned");
+  WindowArg wa;
+  scalekv_status st = fill_window(ctx, layer, w, window_pos, wa);
+  if (st != SCALEKV_OK) return st;
+  const int k = ctx->next_scale[layer] - 1;
+  const int L = ctx->hist[layer] + ctx->pending[layer];
+  const int cand = L - wa.w;
+  const int budget = p.budgets[(size_t)layer * p.K + k];
+  const bool evict = budget != SCALEKV_KEEP_ALL && budget < cand;
+  cudaStream_t s = ctx->s_side;
+  if (s != ctx->s_main) {
+    if (!ctx->attended[layer]) CU(cudaEventRecord(ctx->ev_attend[layer], ctx->s_main));
+    CU(cudaStreamWaitEvent(s, ctx->ev_attend[layer], 0));
+  }
+  if (!evict) {
+    st = commit_pending(ctx, layer, s);
+    if (st != SCALEKV_OK) return st;
+  } else {
+    LayerView lv = layer_view(ctx, layer);
+    float *logits = reinterpret_cast<float *>(ctx->ws + p.off_logits);
+    float *scores = reinterpret_cast<float *>(ctx->ws + p.off_scores);
+    uint32_t *keys = reinterpret_cast<uint32_t *>(ctx->ws + p.off_keys);
+    int *keep = reinterpret_cast<int *>(ctx->ws + p.off_keep);
+    int *kept = reinterpret_cast<int *>(ctx->ws + p.off_kept);
+    {
+      Scope sc(ctx, s, kScore);
+      dim3 grid((L + 63) / 64, p.n_slices);
+      if (ctx->dtype == SCALEKV_BF16)
+        score_logits_kernel<__nv_bfloat16, 128><<<grid, 256, 2 * 64 * 132 * 4, s>>>(lv, tview(Qw), wa, qw_is_full_map, logits,
+                                                                                  p.ld_s, ctx->scale);
+      else
+        score_logits_kernel<float, 64><<<grid, 256, 2 * 64 * 68 * 4, s>>>(lv, tview(Qw), wa, qw_is_full_map, logits, p.ld_s,
+                                                                         ctx->scale);
+    }
+    {
+      Scope sc(ctx, s, kScore);
+      score_reduce_kernel<<<p.n_slices, 512, 0, s>>>(lv, wa, logits, p.ld_s, scores, p.ld_s);
+    }
+    {
+      Scope sc(ctx, s, kSelect);
+      select_kernel<<<p.n_slices, 1024, 0, s>>>(lv, wa, budget, scores, p.ld_s, keys, keep, kept);
+    }
+    {
+      Scope sc(ctx, s, kCompact);
+      compact_kernel<<<dim3(p.n_slices, 2), 256, 0, s>>>(lv, keep, p.ld_s, kept);
+    }
+    ctx->scores_len = L;
+    ctx->hist[layer] = budget + wa.w;
+    ctx->pending[layer] = 0;
+    ctx->attended[layer] = 0;
+    st = check_launch(ctx, "compress");
+    if (st != SCALEKV_OK) return st;
+  }
+  if (s != ctx->s_main) {
+    CU(cudaEventRecord(ctx->ev_compress[layer], s));
+    ctx->ev_compress_live[layer] = 1;
+  }
+  return SCALEKV_OK;
+}
+
+scalekv_status scalekv_step_host(scalekv_ctx *ctx, int32_t layer, int32_t scale, const void *Q_host, const void *K_host,
+                                 const void *V_host, void *O_host, void *staging, size_t staging_bytes, int32_t w,
+                                 const int32_t *window_pos) {
+  if (!ctx) return SCALEKV_ERR_INVALID_ARG;
+  const Plan &p = ctx->plan;
+  if (scale < 0 || scale >= p.K) return fail(ctx, SCALEKV_ERR_INVALID_ARG, "scale %d out of range", scale);
+  if (!Q_host || !K_host || !V_host || !O_host || !staging) return fail(ctx, SCALEKV_ERR_INVALID_ARG, "null buffer");
+  const int nk = p.n[scale];
+  const size_t bytes = (size_t)p.n_slices * nk * p.d * p.esize;
+  if (staging_bytes < 4 * bytes) return fail(ctx, SCALEKV_ERR_CAPACITY, "staging needs %zu bytes", 4 * bytes);
+  char *dq = static_cast<char *>(staging), *dk = dq + bytes, *dv = dk + bytes, *dout = dv + bytes;
+  CU(cudaMemcpyAsync(dk, K_host, bytes, cudaMemcpyHostToDevice, ctx->s_main));
+  CU(cudaMemcpyAsync(dv, V_host, bytes, cudaMemcpyHostToDevice, ctx->s_main));
+  CU(cudaMemcpyAsync(dq, Q_host, bytes, cudaMemcpyHostToDevice, ctx->s_main));
+  auto dense = [&](const void *ptr) {
+    scalekv_tensor t; t.ptr = ptr; t.stride_t = p.d; t.stride_h = (int64_t)nk * p.d; t.stride_b = (int64_t)p.H * nk * p.d;
+    return t;
+  };
+  scalekv_status st = scalekv_append(ctx, layer, scale, dense(dk), dense(dv));
+  if (st != SCALEKV_OK) return st;
+  st = scalekv_attend(ctx, layer, dense(dq), dense(dout), nullptr);
+  if (st != SCALEKV_OK) return st;
+  CU(cudaMemcpyAsync(O_host, dout, bytes, cudaMemcpyDeviceToHost, ctx->s_main));
+  if (w > 0) {
+    st = scalekv_compress(ctx, layer, dense(dq), w, window_pos, 1);
+    if (st != SCALEKV_OK) return st;
+  } else if (w < 0) {
+    st = scalekv_compress(ctx, layer, dense(dq), 0, nullptr, 1);
+    if (st != SCALEKV_OK) return st;
+  }
+  return SCALEKV_OK;
+}
+
+scalekv_status scalekv_layer_stats(scalekv_ctx *ctx, int32_t layer, scalekv_tensor Q, int32_t topk_prime,
+                                   int32_t query_stride, double *car, double *htk) {
+  if (!ctx || !car || !htk) return SCALEKV_ERR_INVALID_ARG;
+  const Plan &p = ctx->plan;
+  if (layer < 0 || layer >= p.n_layers) return fail(ctx, SCALEKV_ERR_INVALID_ARG, "layer %d out of range", layer);
+  if (ctx->pending[layer] == 0) return fail(ctx, SCALEKV_ERR_BAD_STATE, "layer %d: layer_stats needs a preceding append", layer);
+  if (topk_prime < 0 || topk_prime > 64 || query_stride < 1) return fail(ctx, SCALEKV_ERR_INVALID_ARG, "topk_prime in [0,64], stride >= 1");
+  if (!tensor_ok(Q, p.esize)) return fail(ctx, SCALEKV_ERR_INVALID_ARG, "Q null or rows not 16-byte aligned");
+  const int nk = ctx->pending[layer];
+  const int k = ctx->next_scale[layer] - 1;
+  const int L = ctx->hist[layer] + nk;
+  const int rows = (nk + query_stride - 1) / query_stride;
+  double *acc = reinterpret_cast<double *>(ctx->ws + p.off_acc);
+  CU(cudaMemsetAsync(acc, 0, 16, ctx->s_main));
+  {
+    Scope sc(ctx, ctx->s_main, kOther);
+    dim3 grid(rows, p.n_slices);
+    if (ctx->dtype == SCALEKV_BF16)
+      layer_stats_kernel<__nv_bfloat16, 128><<<grid, 256, (size_t)(128 + L) * 4, ctx->s_main>>>(
+          layer_view(ctx, layer), tview(Q), nk, p.N[k], query_stride, topk_prime, ctx->scale, acc);
+    else
+      layer_stats_kernel<float, 64><<<grid, 256, (size_t)(64 + L) * 4, ctx->s_main>>>(
+          layer_view(ctx, layer), tview(Q), nk, p.N[k], query_stride, topk_prime, ctx->scale, acc);
+  }
+  scalekv_status st = check_launch(ctx, "layer_stats");
+  if (st != SCALEKV_OK) return st;
+  double host[2];
+  CU(cudaMemcpyAsync(host, acc, 16, cudaMemcpyDeviceToHost, ctx->s_main));
+  CU(cudaStreamSynchronize(ctx->s_main));
+  const double cnt = (double)rows * p.n_slices;
+  *car = host[0] / cnt;
+  *htk = host[1] / cnt;
+  return SCALEKV_OK;
+}
+
+scalekv_status scalekv_window_centroids(int32_t h, int32_t w, int32_t n_patches, int32_t *pos, int32_t *count) {
+  if (h < 1 || w < 1 || n_patches < 1 || !pos || !count) return SCALEKV_ERR_INVALID_ARG;
+  if ((long long)h * w <= n_patches) {
+    for (int i = 0; i < h * w; ++i) pos[i] = i;
+    *count = h * w;
+    return SCALEKV_OK;
+  }
+  int g = (int)std::floor(std::sqrt((double)n_patches));
+  while ((g + 1) * (g + 1) <= n_patches) ++g;
+  while (g * g > n_patches) --g;
+  std::vector<int> out;
+  for (int a = 0; a < g; ++a) {
+    const int r0 = (int)((long long)a * h / g), r1 = (int)((long long)(a + 1) * h / g);
+    if (r1 <= r0) continue;
+    for (int b = 0; b < g; ++b) {
+      const int c0 = (int)((long long)b * w / g), c1 = (int)((long long)(b + 1) * w / g);
+      if (c1 <= c0) continue;
+      out.push_back(((r0 + r1 - 1) / 2) * w + (c0 + c1 - 1) / 2);
+    }
+  }
+  std::sort(out.begin(), out.end());
+  out.erase(std::unique(out.begin(), out.end()), out.end());
+  for (size_t i = 0; i < out.size(); ++i) pos[i] = out[i];
+  *count = (int)out.size();
+  return SCALEKV_OK;
+}
+
+scalekv_status scalekv_assign_roles(const double *asi, int32_t L, int32_t K, int32_t n_drafters, int32_t mode, double eps,
+                                    uint8_t *is_drafter) {
+  if (!asi || !is_drafter || L < 1 || K < 1 || n_drafters < 0) return SCALEKV_ERR_INVALID_ARG;
+  std::vector<double> z((size_t)L * K, 0.0);
+  for (int k = 0; k < K; ++k) {
+    double mu = 0; for (int l = 0; l < L; ++l) mu += asi[(size_t)l * K + k];
+    mu /= L;
+    double var = 0; for (int l = 0; l < L; ++l) { double dlt = asi[(size_t)l * K + k] - mu; var += dlt * dlt; }
+    const double sd = std::sqrt(var / L);
+    for (int l = 0; l < L; ++l) z[(size_t)l * K + k] = (asi[(size_t)l * K + k] - mu) / (sd + eps);
+  }
+  std::memset(is_drafter, 0, (size_t)L * K);
+  struct Cell { double z; int k, l; };
+  auto less = [](const Cell &a, const Cell &b) { return a.z != b.z ? a.z < b.z : (a.k != b.k ? a.k < b.k : a.l < b.l); };
+  if (mode == 0) {
+    std::vector<Cell> cells;
+    for (int k = 1; k < K - 1; ++k) for (int l = 0; l < L; ++l) cells.push_back({z[(size_t)l * K + k], k, l});
+    std::sort(cells.begin(), cells.end(), less);
+    for (int i = 0; i < n_drafters && i < (int)cells.size(); ++i) is_drafter[(size_t)cells[i].l * K + cells[i].k] = 1;
+  } else {
+    for (int k = 1; k < K - 1; ++k) {
+      std::vector<Cell> cells;
+      for (int l = 0; l < L; ++l) cells.push_back({z[(size_t)l * K + k], k, l});
+      std::sort(cells.begin(), cells.end(), less);
+      for (int i = 0; i < n_drafters && i < L; ++i) is_drafter[(size_t)cells[i].l * K + k] = 1;
+    }
+  }
+  return SCALEKV_OK;
+}
+
+scalekv_status scalekv_make_budgets(const uint8_t *is_drafter, int32_t L, int32_t K, double b_uniform, double b_r0, double delta,
+                                    int32_t *budgets_out) {
+  if (!is_drafter || !budgets_out || L < 1 || K < 1) return SCALEKV_ERR_INVALID_ARG;
+  for (int k = 0; k < K; ++k) {
+    int nd = 0; for (int l = 0; l < L; ++l) nd += is_drafter[(size_t)l * K + k] ? 1 : 0;
+    const int nr = L - nd;
+    const double br = std::max(b_r0 - delta * (k + 1), 0.0);
+    if (nd == 0) {
+      for (int l = 0; l < L; ++l) budgets_out[(size_t)l * K + k] = (int32_t)std::floor(b_uniform + 0.5);
+      continue;
+    }
+    const double bd = (b_uniform * L - nr * br) / nd;
+    for (int l = 0; l < L; ++l)
+      budgets_out[(size_t)l * K + k] = (int32_t)std::floor((is_drafter[(size_t)l * K + k] ? bd : br) + 0.5);
+  }
+  return SCALEKV_OK;
+}
+
+scalekv_status scalekv_sync(scalekv_ctx *ctx) {
+  if (!ctx) return SCALEKV_ERR_INVALID_ARG;
+  CU(cudaStreamSynchronize(ctx->s_main));
+  if (ctx->s_side != ctx->s_main) CU(cudaStreamSynchronize(ctx->s_side));
+  int status = 0;
+  CU(cudaMemcpy(&status, ctx->pool + ctx->plan.off_status, 4, cudaMemcpyDeviceToHost));
+  if (status == kDevTimeout) return fail(ctx, SCALEKV_ERR_TIMEOUT, "a bounded device-side wait gave up");
+  if (status != 0) return fail(ctx, SCALEKV_ERR_DEVICE_CHECK, "device-side check failed (code %d)", status);
+  return SCALEKV_OK;
+}
+
+scalekv_status scalekv_lengths(scalekv_ctx *ctx, int32_t layer, int32_t *len_host) {
+  if (!ctx || !len_host) return SCALEKV_ERR_INVALID_ARG;
+  const Plan &p = ctx->plan;
+  if (layer < 0 || layer >= p.n_layers) return fail(ctx, SCALEKV_ERR_INVALID_ARG, "layer %d out of range", layer);
+  scalekv_status st = scalekv_sync(ctx);
+  if (st != SCALEKV_OK) return st;
+  CU(cudaMemcpy(len_host, ctx->pool + p.off_len + (size_t)layer * p.n_slices * 4, (size_t)p.n_slices * 4, cudaMemcpyDeviceToHost));
+  for (int s = 0; s < p.n_slices; ++s) len_host[s] += ctx->pending[layer];
+  return SCALEKV_OK;
+}
+
+scalekv_status scalekv_export_slice(scalekv_ctx *ctx, int32_t layer, int32_t b, int32_t h, int32_t *pos_host, void *K_host,
+                                    void *V_host, int32_t cap, int32_t *len) {
+  if (!ctx || !len) return SCALEKV_ERR_INVALID_ARG;
+  const Plan &p = ctx->plan;
+  if (layer < 0 || layer >= p.n_layers || b < 0 || b >= p.B || h < 0 || h >= p.H)
+    return fail(ctx, SCALEKV_ERR_INVALID_ARG, "slice index out of range");
+  scalekv_status st = scalekv_sync(ctx);
+  if (st != SCALEKV_OK) return st;
+  const int slice = b * p.H + h;
+  int hist = 0;
+  CU(cudaMemcpy(&hist, ctx->pool + p.off_len + ((size_t)layer * p.n_slices + slice) * 4, 4, cudaMemcpyDeviceToHost));
+  const int L = hist + ctx->pending[layer];
+  *len = L;
+  if (L > cap) return fail(ctx, SCALEKV_ERR_CAPACITY, "slice holds %d entries, cap is %d", L, cap);
+  const LayerPlan &lp = p.layers[layer];
+  const size_t row_bytes = (size_t)p.d * p.esize;
+  for (int s0 = 0; s0 < L; s0 += p.P) {
+    const int cnt = std::min(p.P, L - s0);
+    const size_t page = (size_t)ctx->page_table_host[lp.page_table_off + (size_t)slice * lp.total_pages + s0 / p.P];
+    if (pos_host) CU(cudaMemcpy(pos_host + s0, ctx->pool + p.off_pos + page * p.P * 4, (size_t)cnt * 4, cudaMemcpyDeviceToHost));
+    if (K_host) CU(cudaMemcpy(static_cast<char *>(K_host) + s0 * row_bytes, ctx->pool + p.off_k + page * p.P * row_bytes, cnt * row_bytes, cudaMemcpyDeviceToHost));
+    if (V_host) CU(cudaMemcpy(static_cast<char *>(V_host) + s0 * row_bytes, ctx->pool + p.off_v + page * p.P * row_bytes, cnt * row_bytes, cudaMemcpyDeviceToHost));
+  }
+  return SCALEKV_OK;
+}
+
+scalekv_status scalekv_export_scores(scalekv_ctx *ctx, int32_t b, int32_t h, float *s_host, int32_t cap, int32_t *len) {
+  if (!ctx || !s_host || !len) return SCALEKV_ERR_INVALID_ARG;
+  const Plan &p = ctx->plan;
+  if (b < 0 || b >= p.B || h < 0 || h >= p.H) return fail(ctx, SCALEKV_ERR_INVALID_ARG, "slice index out of range");
+  scalekv_status st = scalekv_sync(ctx);
+  if (st != SCALEKV_OK) return st;
+  *len = ctx->scores_len;
+  if (ctx->scores_len > cap) return fail(ctx, SCALEKV_ERR_CAPACITY, "scores hold %d entries, cap is %d", ctx->scores_len, cap);
+  CU(cudaMemcpy(s_host, ctx->ws + p.off_scores + (size_t)(b * p.H + h) * p.ld_s * 4, (size_t)ctx->scores_len * 4, cudaMemcpyDeviceToHost));
+  return SCALEKV_OK;
+}
+
+scalekv_status scalekv_launch_count(scalekv_ctx *ctx, int64_t *count) {
+  if (!ctx || !count) return SCALEKV_ERR_INVALID_ARG;
+  *count = ctx->launches;
+  return SCALEKV_OK;
+}
+
+scalekv_status scalekv_profile_enable(scalekv_ctx *ctx, int32_t on) {
+  if (!ctx) return SCALEKV_ERR_INVALID_ARG;
+  scalekv_status st = scalekv_sync(ctx);
+  if (st != SCALEKV_OK) return st;
+  drain_profile(ctx);
+  if (on) for (int i = 0; i < kNumClasses; ++i) { ctx->prof_ms[i] = 0; ctx->prof_n[i] = 0; }
+  ctx->profile = on != 0;
+  return SCALEKV_OK;
+}
+
+scalekv_status scalekv_profile_read(scalekv_ctx *ctx, int32_t which, double *ms_total, int64_t *launches) {
+  if (!ctx || which < 0 || which >= kNumClasses || !ms_total || !launches) return SCALEKV_ERR_INVALID_ARG;
+  scalekv_status st = scalekv_sync(ctx);
+  if (st != SCALEKV_OK) return st;
+  drain_profile(ctx);
+  *ms_total = ctx->prof_ms[which];
+  *launches = ctx->prof_n[which];
+  return SCALEKV_OK;
+}
+
+const char *scalekv_error_string(scalekv_ctx *ctx) { return ctx ? ctx->err.c_str() : "null context"; }
+
+}  // extern "C"

@@ -1,0 +1,134 @@
+"""Drivers around the C-ABI context: the per-scale loop of one pass, offline role calibration and
+the budget tables of the named workloads.  Only call sequencing lives here; all arithmetic runs
+in the library."""
+from __future__ import annotations
+
+import dataclasses
+
+import numpy as np
+import torch
+
+from . import binding, synth
+
+
+def windows_for(sides, n_patches=16):
+    """Observation-window raster indices for every scale (Sec. 3.3), from the library's helper."""
+    return [binding.scalekv_window_centroids(a, a, n_patches) for a in sides]
+
+
+def pct_budget(fraction_num, fraction_den, t_c):
+    """round-half-up of (num/den) * T_c in integers."""
+    return (2 * fraction_num * t_c + fraction_den) // (2 * fraction_den)
+
+
+def budget_table(wl: synth.Workload, roles, drafter_pct=(30, 100), refiner_pct=(3, 100)):
+    """budgets[l][k]: drafter or refiner budget by role (percentages of T_c = N_{K-1})."""
+    t_c = sum(wl.n_tokens[:-1])
+    bd, br = pct_budget(*drafter_pct, t_c), pct_budget(*refiner_pct, t_c)
+    return [[bd if roles[l][k] else br for k in range(wl.n_scales)] for l in range(wl.n_layers)]
+
+
+def calibrate_roles(wl: synth.Workload, n_drafters, topk_prime=16, query_stride=16, batch=1, device=0):
+    """Runs the workload's seeded inputs with a full cache (reduced batch) and collects the
+    Attention Selectivity Index per (layer, scale) with scalekv_layer_stats (Eq. 2); returns
+    (asi [L][K], is_drafter [L][K]) with the n_drafters lowest-Z layers per ranked scale (Eq. 3)."""
+    cal = dataclasses.replace(wl, batch=batch)
+    keep_all = [[binding.KEEP_ALL] * wl.n_scales for _ in range(wl.n_layers)]
+    kv = binding.ScaleKV(wl.n_layers, batch, wl.n_heads, wl.head_dim, wl.dtype, wl.sides, wl.sides, keep_all,
+                         max_window=min(wl.window, binding.MAX_WINDOW), device=device, side_stream=False)
+    asi = np.zeros((wl.n_layers, wl.n_scales))
+    dev = f"cuda:{device}"
+    for k in range(wl.n_scales):
+        stride = max(1, min(query_stride, wl.n_tokens[k] // 16))
+        for l in range(wl.n_layers):
+            Q, K, V = synth.scale_inputs(cal, l, k, device=dev)
+            torch.cuda.synchronize()
+            kv.scalekv_append(l, k, K, V)
+            car, htk = kv.scalekv_layer_stats(l, Q, topk_prime, stride)
+            asi[l, k] = car * htk
+    kv.close()
+    roles = binding.scalekv_assign_roles(asi, n_drafters, mode=1)
+    return asi, roles
+
+
+class PassInputs:
+    """Device-resident Q/K/V of every (layer, scale) of a workload, generated once."""
+
+    def __init__(self, wl: synth.Workload, device=0, share_layers=False):
+        dev = f"cuda:{device}"
+        self.wl = wl
+        self.data = {}
+        for l in range(wl.n_layers):
+            for k in range(wl.n_scales):
+                if share_layers and l > 0:
+                    self.data[(l, k)] = self.data[(0, k)]
+                else:
+                    self.data[(l, k)] = synth.scale_inputs(wl, l, k, device=dev)
+        n_max = max(wl.n_tokens)
+        self.O = torch.empty(wl.batch, wl.n_heads, n_max, wl.head_dim, dtype=synth.torch_dtype(wl.dtype), device=dev)
+        torch.cuda.synchronize()
+
+    def bytes(self):
+        seen, total = set(), 0
+        for q, k, v in self.data.values():
+            if q.data_ptr() in seen:
+                continue
+            seen.add(q.data_ptr())
+            total += 3 * q.numel() * q.element_size()
+        return total
+
+
+def run_pass(kv: binding.ScaleKV, inputs: PassInputs, windows, compress_last=False):
+    """One pass: reset, then for every scale and layer append -> attend -> compress."""
+    wl = inputs.wl
+    kv.scalekv_reset()
+    for k in range(wl.n_scales):
+        nk = wl.n_tokens[k]
+        O = inputs.O[:, :, :nk, :]
+        last = k + 1 == wl.n_scales
+        for l in range(wl.n_layers):
+            Q, K, V = inputs.data[(l, k)]
+            kv.scalekv_append(l, k, K, V)
+            kv.scalekv_attend(l, Q, O)
+            if not last or compress_last:
+                if windows[k] is None:
+                    kv.scalekv_compress(l, Q, None)
+                else:
+                    kv.scalekv_compress(l, Q, windows[k], qw_is_full_map=True)
+
+
+def pass_work(wl: synth.Workload, budgets, windows):
+    """Algorithmic work of one pass, from the schedule alone: attention flops (4 n_k L d per
+    slice-step), bytes of K read by scoring, bytes moved by compaction (upper bound: every kept row
+    beyond the untouched prefix is unknown on the host, so all kept rows are counted), append bytes."""
+    n = wl.n_tokens
+    d = wl.head_dim
+    esz = 2 if wl.dtype == "bf16" else 4
+    slices = wl.batch * wl.n_heads
+    out = {"attend_flop": 0, "attend_min_bytes": 0, "score_bytes": 0, "compact_bytes": 0, "append_bytes": 0,
+           "select_bytes": 0, "attend_launches": 0}
+    per_scale_flop = [0] * wl.n_scales
+    for l in range(wl.n_layers):
+        hist = 0
+        for k in range(wl.n_scales):
+            L = hist + n[k]
+            f = 4 * n[k] * L * d * slices
+            out["attend_flop"] += f
+            per_scale_flop[k] += f
+            out["attend_min_bytes"] += (2 * L + 2 * n[k]) * d * esz * slices
+            out["append_bytes"] += 2 * 2 * n[k] * d * esz * slices
+            out["attend_launches"] += 1
+            if k + 1 == wl.n_scales:
+                break
+            w = len(windows[k]) if windows[k] is not None else n[k]
+            cand = L - w
+            b = budgets[l][k]
+            if b != binding.KEEP_ALL and b < cand:
+                out["score_bytes"] += L * d * esz * slices
+                out["select_bytes"] += (4 * L + 4 * (b + w)) * slices
+                out["compact_bytes"] += (b + w) * 2 * 2 * d * esz * slices
+                hist = b + w
+            else:
+                hist = L
+    out["per_scale_flop"] = per_scale_flop
+    return out

@@ -1,0 +1,94 @@
+"""CPU-only checks of the C-ABI library: it builds for sm_100a, loads, exports every symbol the
+header declares, and its host-only helpers agree with the oracle.  No kernel is launched."""
+import ctypes as C
+import math
+
+import numpy as np
+import pytest
+
+from oracle import scalekv_oracle as orc
+from paper_2505_19602_b200 import binding
+
+SIDES_13 = (1, 2, 4, 6, 8, 12, 16, 20, 24, 32, 40, 48, 64)
+SIDES_16 = SIDES_13 + (80, 96, 128)
+
+
+@pytest.fixture(scope="module")
+def lib():
+    binding.build_library()
+    return binding.load_library()
+
+
+def test_exports_every_declared_symbol(lib):
+    names = binding.exported_symbols()
+    assert len(names) >= 20 and "scalekv_attend" in names and "scalekv_compress" in names
+    for name in names:
+        assert hasattr(lib, name), name
+
+
+def test_window_centroids_match_oracle(lib):
+    for a in SIDES_16:
+        for n in (16, 4, 9, 1):
+            assert binding.scalekv_window_centroids(a, a, n) == orc.window_centroids(a, a, n)
+    assert binding.scalekv_window_centroids(6, 10, 16) == orc.window_centroids(6, 10, 16)
+
+
+def test_assign_roles_and_budgets_match_oracle(lib):
+    rng = np.random.default_rng(0)
+    asi = rng.random((12, 7)) * 0.2
+    for mode, nd in ((0, 9), (1, 3)):
+        assert np.array_equal(binding.scalekv_assign_roles(asi, nd, mode), orc.assign_roles(asi, nd, mode))
+    roles = orc.assign_roles(asi, 3, 1)
+    for delta in (0, 20, 70):
+        assert np.array_equal(binding.scalekv_make_budgets(roles, 650, 600, delta), orc.make_budgets(roles, 650, 600, delta))
+
+
+def make_cfg(n_layers, B, H, d, dtype, sides, budgets, max_window=16, page_tokens=0):
+    cfg = binding.scalekv_config()
+    cfg.n_layers, cfg.batch, cfg.n_heads, cfg.head_dim, cfg.dtype = n_layers, B, H, d, dtype
+    cfg.n_scales = len(sides)
+    keep = (binding._i32_array(sides), binding._i32_array([x for r in budgets for x in r]))
+    cfg.scale_h, cfg.scale_w, cfg.budgets = keep[0], keep[0], keep[1]
+    cfg.max_window, cfg.page_tokens = max_window, page_tokens
+    return cfg, keep
+
+
+def test_query_sizes_accounting(lib):
+    n13 = orc.scale_token_counts(SIDES_13)
+    # full cache, one layer, B 8, H 16: K and V pages cover 10521 tokens per slice
+    cfg, keep = make_cfg(1, 8, 16, 128, binding.BF16, SIDES_13, [[-1] * 13])
+    pb, wb = C.c_size_t(), C.c_size_t()
+    assert lib.scalekv_query_sizes(C.byref(cfg), C.byref(pb), C.byref(wb)) == 0
+    pages = math.ceil(10521 / 128)
+    kv_bytes = 128 * pages * 128 * 2 * 2 * 128
+    assert kv_bytes <= pb.value <= kv_bytes * 1.05
+    # 10 % drafter/refiner budgets need far less than the full cache
+    bd, br = orc.budget_tokens(0.30, n13), orc.budget_tokens(0.03, n13)
+    budgets = [[bd] * 13 if l < 8 else [br] * 13 for l in range(32)]
+    cfg2, keep2 = make_cfg(32, 8, 16, 128, binding.BF16, SIDES_13, budgets)
+    pb2 = C.c_size_t()
+    assert lib.scalekv_query_sizes(C.byref(cfg2), C.byref(pb2), C.byref(wb)) == 0
+    full32 = 32 * kv_bytes
+    assert pb2.value < 0.2 * full32
+
+
+def test_query_sizes_rejects_bad_configs(lib):
+    pb, wb = C.c_size_t(), C.c_size_t()
+    cfg, keep = make_cfg(1, 1, 4, 64, binding.BF16, (1, 2), [[-1, -1]])
+    assert lib.scalekv_query_sizes(C.byref(cfg), C.byref(pb), C.byref(wb)) == 4      # UNSUPPORTED
+    cfg, keep = make_cfg(1, 1, 4, 64, binding.F32, (1, 2), [[-1, -1]], max_window=65)
+    assert lib.scalekv_query_sizes(C.byref(cfg), C.byref(pb), C.byref(wb)) == 1      # INVALID_ARG
+    cfg, keep = make_cfg(1, 1, 4, 64, binding.F32, (1, 2), [[-1, -1]], page_tokens=48)
+    assert lib.scalekv_query_sizes(C.byref(cfg), C.byref(pb), C.byref(wb)) == 1
+    cfg, keep = make_cfg(1, 1, 4, 64, binding.F32, (1, 2), [[-1, -5]])
+    assert lib.scalekv_query_sizes(C.byref(cfg), C.byref(pb), C.byref(wb)) == 1
+    assert lib.scalekv_query_sizes(None, C.byref(pb), C.byref(wb)) == 1
+
+
+def test_product_path_refuses_to_run_without_gpu():
+    import torch
+
+    if torch.cuda.is_available():
+        pytest.skip("GPU present")
+    with pytest.raises(RuntimeError):
+        binding.ScaleKV(1, 1, 4, 64, "f32", (1, 2), (1, 2), [[-1, -1]])

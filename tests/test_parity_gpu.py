@@ -1,0 +1,194 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same seeded
+inputs - attention outputs within the dtype's bound, kept index sets exact (or inside the stated
+tie band), compacted rows bit-exact."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import scalekv_oracle as orc
+from paper_2505_19602_b200 import binding, synth
+from parity_util import ParityRun
+
+pytestmark = pytest.mark.gpu
+
+
+def randn_inputs(B, H, d, n, dtype, seed):
+    def fn(layer, scale):
+        g = torch.Generator().manual_seed(seed * 1000 + layer * 50 + scale)
+        return tuple(torch.randn(B, H, n[scale], d, generator=g).to(dtype) for _ in range(3))
+    return fn
+
+
+def all_slices(n_layers, B, H):
+    return [(l, b, h) for l in range(n_layers) for b in range(B) for h in range(H)]
+
+
+def test_tiny_config_fp32_whole_map_window():
+    """configs[0]: B 1, 1 layer, 4 heads, d 64, fp32, sides 1,2,4,8; window = whole current map;
+    budget 16; compress also after the last scale so that eviction happens."""
+    wl = synth.WORKLOADS["tiny"]
+    budgets = [[16] * 4]
+    kv = binding.ScaleKV(1, 1, 4, 64, "f32", wl.sides, wl.sides, budgets, max_window=64)
+    run = ParityRun(kv, "f32", wl.sides, budgets, lambda l, k: synth.scale_inputs(wl, l, k), lambda k: None,
+                    all_slices(1, 1, 4), compress_last=True).run()
+    assert run.evictions == 4 and run.resyncs == 0
+    assert kv.scalekv_lengths(0) == [[16 + 64] * 4]
+    kv.close()
+
+
+@pytest.mark.parametrize("budget", [2, 4, 8])
+def test_tiny_variants_evict_early(budget):
+    sides = (1, 2, 4, 8)
+    n = orc.scale_token_counts(sides)
+    budgets = [[budget] * 4]
+    kv = binding.ScaleKV(1, 2, 3, 64, "f32", sides, sides, budgets, max_window=4)
+    run = ParityRun(kv, "f32", sides, budgets, randn_inputs(2, 3, 64, n, torch.float32, 7 + budget),
+                    lambda k: orc.window_centroids(sides[k], sides[k], 4), all_slices(1, 2, 3), compress_last=True).run()
+    assert run.evictions > 0
+    kv.close()
+
+
+@pytest.mark.parametrize("page_tokens", [0, 16])
+def test_bf16_ragged_multi_tile(page_tokens):
+    """bf16, d 128: lengths that are not multiples of any tile or page, several pages per slice,
+    a drafter-like and a refiner-like layer, explicit 16-token windows."""
+    sides = (1, 2, 3, 5, 9, 14, 19)
+    n = orc.scale_token_counts(sides)
+    budgets = [[150] * len(sides), [21] * len(sides)]
+    kv = binding.ScaleKV(2, 2, 2, 128, "bf16", sides, sides, budgets, max_window=16, page_tokens=page_tokens)
+    wl = synth.Workload("t", 2, 2, 2, 128, "bf16", sides, seed=11, n_drafters=1)
+    run = ParityRun(kv, "bf16", sides, budgets, lambda l, k: synth.scale_inputs(wl, l, k),
+                    lambda k: orc.window_centroids(sides[k], sides[k], 16), all_slices(2, 2, 2)).run()
+    assert run.evictions >= 8
+    lens = kv.scalekv_lengths(1)
+    assert lens == [[21 + 16 + n[-1]] * 2] * 2      # last scale is not compressed
+    kv.close()
+
+
+def test_keep_all_matches_full_attention():
+    sides = (1, 2, 4, 6, 8, 12)
+    n = orc.scale_token_counts(sides)
+    budgets = [[binding.KEEP_ALL] * len(sides)]
+    kv = binding.ScaleKV(1, 1, 2, 128, "bf16", sides, sides, budgets)
+    run = ParityRun(kv, "bf16", sides, budgets, randn_inputs(1, 2, 128, n, torch.bfloat16, 3),
+                    lambda k: orc.window_centroids(sides[k], sides[k], 16), all_slices(1, 1, 2)).run()
+    assert run.evictions == 0
+    assert kv.scalekv_lengths(0) == [[sum(n)] * 2]
+    pos = kv.scalekv_export_slice(0, 0, 1)
+    assert pos.tolist() == list(range(sum(n)))
+    kv.close()
+
+
+def test_exact_ties_keep_lowest_positions():
+    """Q = 0 makes every score bit-equal: the kept candidates are the lowest positions."""
+    sides = (2, 4, 8)
+    n = orc.scale_token_counts(sides)
+    budgets = [[5] * 3]
+    kv = binding.ScaleKV(1, 1, 2, 64, "f32", sides, sides, budgets, max_window=4)
+    g = torch.Generator().manual_seed(5)
+    for k in range(2):
+        K = torch.randn(1, 2, n[k], 64, generator=g).cuda()
+        V = torch.randn(1, 2, n[k], 64, generator=g).cuda()
+        Q = torch.zeros(1, 2, n[k], 64).cuda()
+        torch.cuda.synchronize()
+        kv.scalekv_append(0, k, K, V)
+        O = kv.scalekv_attend(0, Q)
+        wpos = orc.window_centroids(sides[k], sides[k], 4)
+        kv.scalekv_compress(0, Q, wpos, qw_is_full_map=True)
+        kv.scalekv_sync()
+        if k == 0:
+            assert kv.scalekv_export_slice(0, 0, 0).tolist() == [0, 1, 2, 3]
+        else:
+            base = 4
+            want = sorted(set(list(range(5)) + [base + p for p in wpos]))
+            # candidates exclude the window; the 5 lowest candidate positions are kept
+            cands = [p for p in list(range(4)) + [base + i for i in range(16)] if p not in [base + q for q in wpos]]
+            want = sorted(cands[:5] + [base + q for q in wpos])
+            assert kv.scalekv_export_slice(0, 0, 1).tolist() == want
+    # uniform attention: O is the mean of V over the cache
+    kv.close()
+
+
+def test_deterministic_and_reset():
+    sides = (1, 2, 4, 8, 12)
+    n = orc.scale_token_counts(sides)
+    budgets = [[30] * 5]
+    kv = binding.ScaleKV(1, 2, 2, 128, "bf16", sides, sides, budgets)
+    inputs = randn_inputs(2, 2, 128, n, torch.bfloat16, 9)
+    outs = []
+    for rep in range(2):
+        kv.scalekv_reset()
+        rec = []
+        for k in range(5):
+            Q, K, V = (t.cuda() for t in inputs(0, k))
+            torch.cuda.synchronize()
+            kv.scalekv_append(0, k, K, V)
+            rec.append(kv.scalekv_attend(0, Q))
+            if k < 4:
+                kv.scalekv_compress(0, Q, orc.window_centroids(sides[k], sides[k], 16), qw_is_full_map=True)
+        kv.scalekv_sync()
+        rec.append(kv.scalekv_export_slice(0, 1, 1))
+        outs.append([t.cpu() for t in rec])
+    for a, b in zip(*outs):
+        assert torch.equal(a, b)
+    assert kv.scalekv_launch_count() > 0
+    kv.close()
+
+
+def test_call_order_and_argument_errors():
+    sides = (1, 2, 4)
+    kv = binding.ScaleKV(1, 1, 2, 64, "f32", sides, sides, [[4] * 3], max_window=4)
+    x = torch.randn(1, 2, 1, 64, device="cuda")
+    torch.cuda.synchronize()
+    with pytest.raises(binding.ScaleKVError) as e:
+        kv.scalekv_attend(0, x)
+    assert e.value.status == 2                      # BAD_STATE: no append yet
+    with pytest.raises(binding.ScaleKVError) as e:
+        kv.scalekv_append(0, 1, x, x)
+    assert e.value.status == 2                      # scales must ascend from 0
+    with pytest.raises(binding.ScaleKVError) as e:
+        kv.scalekv_append(3, 0, x, x)
+    assert e.value.status == 1
+    kv.scalekv_append(0, 0, x, x)
+    kv.scalekv_attend(0, x)
+    with pytest.raises(binding.ScaleKVError) as e:
+        kv.scalekv_compress(0, x, [0, 0])           # not distinct / larger than the map
+    assert e.value.status == 1
+    kv.scalekv_compress(0, x, [0])
+    kv.scalekv_sync()
+    assert kv.scalekv_lengths(0) == [[1, 1]]
+    kv.close()
+
+
+def test_layer_stats_matches_oracle_and_recovers_planted_roles():
+    sides = (1, 2, 4, 8, 12)
+    n = orc.scale_token_counts(sides)
+    N = orc.cumulative_token_counts(n)
+    L_layers, B, H = 4, 1, 2
+    wl = synth.Workload("t", L_layers, B, H, 128, "bf16", sides, seed=21, n_drafters=1)
+    budgets = [[binding.KEEP_ALL] * len(sides)] * L_layers
+    kv = binding.ScaleKV(L_layers, B, H, 128, "bf16", sides, sides, budgets)
+    asi = np.zeros((L_layers, len(sides)))
+    caches = {(l, b, h): orc.SliceCache(n, 128) for l in range(L_layers) for b in range(B) for h in range(H)}
+    for k in range(len(sides)):
+        for l in range(L_layers):
+            Q, K, V = synth.scale_inputs(wl, l, k)
+            Qd, Kd, Vd = Q.cuda(), K.cuda(), V.cuda()
+            torch.cuda.synchronize()
+            kv.scalekv_append(l, k, Kd, Vd)
+            car, htk = kv.scalekv_layer_stats(l, Qd, topk_prime=4, query_stride=2)
+            sc = st = cnt = 0
+            for b in range(B):
+                for h in range(H):
+                    c = caches[(l, b, h)]
+                    c.append(K[b, h].double().numpy(), V[b, h].double().numpy())
+                    a = orc.layer_stats_slice(Q[b, h].double().numpy(), c.K, c.pos, N[k], 4, 2)
+                    sc, st, cnt = sc + a[0], st + a[1], cnt + a[2]
+            want_asi, want_car, want_htk = orc.asi_from_sums(sc, st, cnt)
+            assert abs(car - want_car) < 1e-4 and abs(htk - want_htk) < 1e-4
+            asi[l, k] = car * htk
+    roles = binding.scalekv_assign_roles(asi, 1, mode=1)
+    planted = synth.drafter_layers(wl)
+    for k in range(2, len(sides) - 1):
+        assert np.nonzero(roles[:, k])[0].tolist() == planted
+    kv.close()
