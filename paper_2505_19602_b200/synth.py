@@ -10,9 +10,10 @@ below stands in for them:
   so that attention is peaked within scales.
 * 4 "sink" keys per slice (position 0 plus 3 seeded positions below T_c) have their rows
   multiplied by 4.
-* layer gain gamma_l in {0, 1}: Q_k += gamma_l * mu_k.  Layers with gamma = 1 look at their
-  own scale (refiner-like), layers with gamma = 0 spread attention (drafter-like).  This
-  gives the offline layer statistics a known answer.
+* planted layer roles (workloads with n_drafters > 0): refiner layers get Q_k += mu_k, which
+  lifts the logits of their own scale (concentrated, local attention); drafter layers get
+  Q_k *= 0.25, a high softmax temperature that disperses attention over the whole history.
+  This gives the offline layer statistics a known answer.
 
 Everything is a pure function of (seed, layer, scale): tensors for one (layer, scale) can be
 regenerated at any time, in any order, on the same device type.
@@ -39,7 +40,7 @@ class Workload:
     sides: tuple
     seed: int
     planted: bool = True
-    n_drafters: int = 0          # layers with gamma = 0
+    n_drafters: int = 0          # layers planted as drafters
     drafter_pct: float = 0.30
     refiner_pct: float = 0.03
     window: int = 16
@@ -121,8 +122,11 @@ def scale_inputs(wl: Workload, layer: int, scale: int, device="cpu"):
     if wl.planted:
         mu = 0.5 * torch.randn((wl.batch, wl.n_heads, 1, d), generator=g, device=dev, dtype=torch.float32)
         K += mu
-        if wl.n_drafters > 0 and layer not in drafter_layers(wl):
-            Q += mu
+        if wl.n_drafters > 0:
+            if layer in drafter_layers(wl):
+                Q *= 0.25
+            else:
+                Q += mu
         base = sum(n[:scale])
         sinks = sink_positions(wl, layer).to(dev) - base          # [B, H, 4] relative to this map
         inside = (sinks >= 0) & (sinks < nk)
