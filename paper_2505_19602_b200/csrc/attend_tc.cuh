@@ -1,17 +1,502 @@
-// Tensor-core (tcgen05 / TMEM / TMA) attention over the paged store.  Placeholder host object
-// until the kernel lands: reports "not enabled" so that the SIMT kernel serves every dtype.
+// Tensor-core attention over the paged store for bf16, head_dim 128 (Sec. 3.3, Eq. 5):
+// O = softmax(scale * Q K^T) V with online softmax, one CTA per (slice, 128-query tile).
+//
+// Roles inside a CTA of 192 threads:
+//   warp 0 (one thread) : TMA producer.  Q tile once; then per 128-key tile the K and V rows, page
+//                         by page through the slice's page table, into 128B-swizzled shared memory.
+//   warp 1 (one thread) : tcgen05.mma issuer.  S_j = Q K_j^T into one of two TMEM buffers, then
+//                         O += P_{j-1} V_{j-1}; S_j is issued before the PV of the previous tile so the
+//                         tensor pipe works under the softmax of tile j-1.  Owns the TMEM allocation.
+//   warps 2-5           : softmax.  Each thread owns one query row (TMEM lane): tcgen05.ld of the S
+//                         row, running max with lazy rescale (O is only rescaled when the max grows by
+//                         more than 2^8), exp2, bf16 P written to shared memory in the K-major swizzled
+//                         operand layout, and at the end the O / l epilogue.
+// Every mbarrier wait is bounded; a wait that gives up raises the sticky device status, sets a
+// CTA-wide abort flag and all roles fall through to the common exit where TMEM is released.
 #pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cstdlib>
 #include <string>
 
 #include "common.cuh"
 
 namespace scalekv {
+namespace tc {
 
+constexpr int kThreads = 192;
+constexpr int kKStages = 2, kVStages = 2;
+constexpr uint32_t kTileBytes = 128 * 128 * 2;   // one 128 x 128 bf16 operand tile
+constexpr uint32_t kHalfBytes = kTileBytes / 2;  // 64 head-dim columns = one 128-byte swizzle span
+constexpr uint32_t kOffQ = 0;
+constexpr uint32_t kOffP = kOffQ + kTileBytes;
+constexpr uint32_t kOffK = kOffP + kTileBytes;
+constexpr uint32_t kOffV = kOffK + kKStages * kTileBytes;
+constexpr uint32_t kOffBar = kOffV + kVStages * kTileBytes;
+constexpr uint32_t kSmemBytes = kOffBar + 256 + 1024;  // + barriers + alignment slack
+// barrier slots (8 bytes each)
+enum { bQFull = 0, bKFull = 1, bKEmpty = 3, bVFull = 5, bVEmpty = 7, bSFull = 9, bSEmpty = 11, bPFull = 13, bPvDone = 14, bCount = 15 };
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kColS = 0, kColO = 256;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ unsigned long long globaltimer() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: false when the CTA is aborting or the time limit ran out (status raised).
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status) {
+  const unsigned long long t0 = globaltimer();
+  while (true) {
+    for (int i = 0; i < 64; ++i)
+      if (mbar_try(bar, parity)) return true;
+    if (*abort_flag || *reinterpret_cast<volatile int *>(status) != 0) return false;
+    if (globaltimer() - t0 > kWaitLimitNs) {
+      *abort_flag = 1;
+      atomicExch(status, kDevTimeout);
+      return false;
+    }
+  }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status) {
+  if (mbar_try(bar, parity)) return true;
+  return mbar_wait_slow(bar, parity, abort_flag, status);
+}
+// Same, with a warp-uniform result (the callers go on to warp-collective tcgen05 instructions).
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status) {
+  return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, status));
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tm, int x, int y, uint32_t bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+               "l"(tm), "r"(x), "r"(y), "r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *tm, int x, int y, int z, int w, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];" ::"r"(dst),
+      "l"(tm), "r"(x), "r"(y), "r"(z), "r"(w), "r"(bar)
+      : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// 32 consecutive fp32 columns of this thread's TMEM lane
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, float *v) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+        "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]),
+        "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+        "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tc_st32(uint32_t taddr, const float *v) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};" ::"r"(taddr),
+      "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])), "r"(__float_as_uint(v[3])),
+      "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])), "r"(__float_as_uint(v[7])),
+      "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])), "r"(__float_as_uint(v[11])),
+      "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])), "r"(__float_as_uint(v[15])),
+      "r"(__float_as_uint(v[16])), "r"(__float_as_uint(v[17])), "r"(__float_as_uint(v[18])), "r"(__float_as_uint(v[19])),
+      "r"(__float_as_uint(v[20])), "r"(__float_as_uint(v[21])), "r"(__float_as_uint(v[22])), "r"(__float_as_uint(v[23])),
+      "r"(__float_as_uint(v[24])), "r"(__float_as_uint(v[25])), "r"(__float_as_uint(v[26])), "r"(__float_as_uint(v[27])),
+      "r"(__float_as_uint(v[28])), "r"(__float_as_uint(v[29])), "r"(__float_as_uint(v[30])), "r"(__float_as_uint(v[31]))
+      : "memory");
+}
+
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle, operand tiles whose 8-row groups are 1024 B
+// apart.  K-major operands (Q, K, P): rows of 128 B, the leading offset is not used.  MN-major
+// operand (V as [key][d]): 64 d-columns are contiguous, the next 64 start `lbo` bytes further.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+  d |= 1ull << 46;   // descriptor version of this architecture
+  d |= 2ull << 61;   // 128-byte swizzle
+  return d;
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = 128, A K-major; B K-major or MN-major.
+__host__ __device__ constexpr uint32_t instr_desc(bool b_mn_major) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+}
+
+struct Params {
+  LayerView lv;
+  TensorView O;
+  float *lse;
+  int n_k;
+  float scale_log2e;   // softmax scale * log2(e)
+  int box_rows;        // rows per K/V TMA box = min(page_tokens, 128)
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                 const __grid_constant__ CUtensorMap tmV, const Params prm) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t *base_ptr = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t bars = base + kOffBar;
+  volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(base_ptr + kOffBar + 128);
+  volatile int *abort_flag = reinterpret_cast<volatile int *>(base_ptr + kOffBar + 132);
+  auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const LayerView &lv = prm.lv;
+  const int slice = blockIdx.y;
+  const int b = slice / lv.n_heads, h = slice % lv.n_heads;
+  const int q0 = blockIdx.x * 128;
+  const int n_k = prm.n_k;
+  const int L = lv.hist_len[slice] + n_k;
+  const int T = (L + 127) >> 7;
+  int *status = lv.status;
+  if (*reinterpret_cast<volatile int *>(status) != 0) return;   // an earlier CTA gave up: do not pile on
+
+  if (tid == 0) {
+    *abort_flag = 0;
+    mbar_init(bar(bQFull), 1);
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(bar(bKFull + s), 1);
+      mbar_init(bar(bKEmpty + s), 1);
+      mbar_init(bar(bVFull + s), 1);
+      mbar_init(bar(bVEmpty + s), 1);
+      mbar_init(bar(bSFull + s), 1);
+      mbar_init(bar(bSEmpty + s), 128);
+    }
+    mbar_init(bar(bPFull), 128);
+    mbar_init(bar(bPvDone), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(base + kOffBar + 128), "r"(kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      // ---------------------------------------------------------------- TMA producer
+      mbar_expect_tx(bar(bQFull), kTileBytes);
+      tma_load_4d(base + kOffQ, &tmQ, 0, q0, h, b, bar(bQFull));
+      tma_load_4d(base + kOffQ + kHalfBytes, &tmQ, 64, q0, h, b, bar(bQFull));
+      const int R = prm.box_rows;
+      const int last_page = (L - 1) >> lv.page_shift;
+      const int *pt = lv.page_table + (size_t)slice * lv.pages_per_slice;
+      bool ok = true;
+      for (int j = 0; j < T && ok; ++j) {
+        const int ks = j % kKStages, vs = j % kVStages;
+        ok = mbar_wait(bar(bKEmpty + ks), ((j / kKStages) & 1) ^ 1, abort_flag, status);
+        if (!ok) break;
+        mbar_expect_tx(bar(bKFull + ks), kTileBytes);
+        for (int r0 = 0; r0 < 128; r0 += R) {
+          const int slot = j * 128 + r0;
+          int lp = slot >> lv.page_shift;
+          lp = lp > last_page ? last_page : lp;
+          const int row = (__ldg(pt + lp) << lv.page_shift) + (slot & lv.page_mask);
+          const uint32_t dst = base + kOffK + ks * kTileBytes + r0 * 128;
+          tma_load_2d(dst, &tmK, 0, row, bar(bKFull + ks));
+          tma_load_2d(dst + kHalfBytes, &tmK, 64, row, bar(bKFull + ks));
+        }
+        ok = mbar_wait(bar(bVEmpty + vs), ((j / kVStages) & 1) ^ 1, abort_flag, status);
+        if (!ok) break;
+        mbar_expect_tx(bar(bVFull + vs), kTileBytes);
+        for (int r0 = 0; r0 < 128; r0 += R) {
+          const int slot = j * 128 + r0;
+          int lp = slot >> lv.page_shift;
+          lp = lp > last_page ? last_page : lp;
+          const int row = (__ldg(pt + lp) << lv.page_shift) + (slot & lv.page_mask);
+          const uint32_t dst = base + kOffV + vs * kTileBytes + r0 * 128;
+          tma_load_2d(dst, &tmV, 0, row, bar(bVFull + vs));
+          tma_load_2d(dst + kHalfBytes, &tmV, 64, row, bar(bVFull + vs));
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      // ---------------------------------------------------------------- MMA issuer
+      constexpr uint32_t idesc_qk = instr_desc(false);
+      constexpr uint32_t idesc_pv = instr_desc(true);
+      bool ok = mbar_wait(bar(bQFull), 0, abort_flag, status);
+      auto issue_pv = [&](int t) -> bool {
+        const int vs = t % kVStages;
+        if (!mbar_wait(bar(bVFull + vs), (t / kVStages) & 1, abort_flag, status)) return false;
+        if (!mbar_wait(bar(bPFull), t & 1, abort_flag, status)) return false;
+        tc_fence_after();
+        const uint32_t p_addr = base + kOffP, v_addr = base + kOffV + vs * kTileBytes;
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk) {
+          const uint64_t ad = smem_desc(p_addr + (kk >> 2) * kHalfBytes + (kk & 3) * 32, 16, 1024);
+          const uint64_t bd = smem_desc(v_addr + kk * 2048, kHalfBytes, 1024);
+          tc_mma(tmem + kColO, ad, bd, idesc_pv, (t > 0 || kk > 0) ? 1u : 0u);
+        }
+        tc_commit(bar(bVEmpty + vs));
+        tc_commit(bar(bPvDone));
+        return true;
+      };
+      for (int j = 0; j < T && ok; ++j) {
+        const int sb = j & 1, ks = j % kKStages;
+        ok = mbar_wait(bar(bKFull + ks), (j / kKStages) & 1, abort_flag, status) &&
+             mbar_wait(bar(bSEmpty + sb), ((j >> 1) & 1) ^ 1, abort_flag, status);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t q_addr = base + kOffQ, k_addr = base + kOffK + ks * kTileBytes;
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk) {
+          const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
+          tc_mma(tmem + kColS + sb * 128, smem_desc(q_addr + off, 16, 1024), smem_desc(k_addr + off, 16, 1024), idesc_qk,
+                 kk > 0 ? 1u : 0u);
+        }
+        tc_commit(bar(bKEmpty + ks));
+        tc_commit(bar(bSFull + sb));
+        if (j > 0) ok = issue_pv(j - 1);
+      }
+      if (ok) issue_pv(T - 1);
+    }
+  } else {
+    // ------------------------------------------------------------------ softmax + epilogue
+    const int q = warp & 3;
+    const int row = q * 32 + lane;
+    const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16);
+    const float c = prm.scale_log2e;
+    float m_used = -INFINITY, l = 0.f;
+    bool ok = true;
+    for (int j = 0; j < T && ok; ++j) {
+      const int sb = j & 1;
+      ok = mbar_wait_warp(bar(bSFull + sb), (j >> 1) & 1, abort_flag, status);
+      if (!ok) break;
+      tc_fence_after();
+      float s[128];
+#pragma unroll
+      for (int cc = 0; cc < 4; ++cc) tc_ld32(lane_addr + kColS + sb * 128 + cc * 32, s + cc * 32);
+      tc_wait_ld();
+      tc_fence_before();
+      mbar_arrive(bar(bSEmpty + sb));
+      if (j == T - 1) {
+        const int valid = L - j * 128;
+        if (valid < 128) {
+#pragma unroll
+          for (int i = 0; i < 128; ++i)
+            if (i >= valid) s[i] = -INFINITY;
+        }
+      }
+      float mt = s[0];
+#pragma unroll
+      for (int i = 1; i < 128; ++i) mt = fmaxf(mt, s[i]);
+      const float mz = mt * c;
+      const bool need = mz > m_used + 8.f;
+      bool waited = false;
+      if (__any_sync(0xffffffffu, need)) {
+        if (j > 0) {
+          ok = mbar_wait_warp(bar(bPvDone), (j - 1) & 1, abort_flag, status);
+          if (!ok) break;
+          tc_fence_after();
+          waited = true;
+        }
+        const float m_new = need ? mz : m_used;
+        const float sc = need ? ex2(m_used - m_new) : 1.f;
+        l *= sc;
+        m_used = m_new;
+        if (j > 0) {
+#pragma unroll
+          for (int cc = 0; cc < 4; ++cc) {
+            float o[32];
+            tc_ld32(lane_addr + kColO + cc * 32, o);
+            tc_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) o[i] *= sc;
+            tc_st32(lane_addr + kColO + cc * 32, o);
+          }
+          tc_wait_st();
+          tc_fence_before();
+        }
+      }
+      const float neg_m = -m_used;
+      uint32_t pk[64];
+      float sum = 0.f;
+#pragma unroll
+      for (int i = 0; i < 64; ++i) {
+        const float p0 = ex2(fmaf(s[2 * i], c, neg_m));
+        const float p1 = ex2(fmaf(s[2 * i + 1], c, neg_m));
+        sum += p0 + p1;
+        pk[i] = pack_bf16(p0, p1);
+      }
+      l += sum;
+      if (!waited && j > 0) {
+        ok = mbar_wait_warp(bar(bPvDone), (j - 1) & 1, abort_flag, status);
+        if (!ok) break;
+      }
+      // P row -> shared memory, K-major 128B-swizzled operand layout (16-byte chunk index XOR row % 8)
+      const uint32_t prow = base + kOffP + row * 128;
+#pragma unroll
+      for (int ch = 0; ch < 16; ++ch) {
+        const uint32_t addr = prow + (ch >> 3) * kHalfBytes + (((ch & 7) ^ (row & 7)) << 4);
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(pk[4 * ch]), "r"(pk[4 * ch + 1]),
+                     "r"(pk[4 * ch + 2]), "r"(pk[4 * ch + 3])
+                     : "memory");
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      mbar_arrive(bar(bPFull));
+    }
+    if (ok) ok = mbar_wait_warp(bar(bPvDone), (T - 1) & 1, abort_flag, status);
+    if (ok) {
+      tc_fence_after();
+      const float inv = 1.f / l;
+      const int qi = q0 + row;
+      __nv_bfloat16 *orow = const_cast<__nv_bfloat16 *>(row_ptr<__nv_bfloat16>(prm.O, b, h, qi < n_k ? qi : 0));
+#pragma unroll
+      for (int cc = 0; cc < 4; ++cc) {
+        float o[32];
+        tc_ld32(lane_addr + kColO + cc * 32, o);
+        tc_wait_ld();
+        if (qi < n_k) {
+#pragma unroll
+          for (int v4 = 0; v4 < 4; ++v4) {
+            uint4 w;
+            w.x = pack_bf16(o[8 * v4 + 0] * inv, o[8 * v4 + 1] * inv);
+            w.y = pack_bf16(o[8 * v4 + 2] * inv, o[8 * v4 + 3] * inv);
+            w.z = pack_bf16(o[8 * v4 + 4] * inv, o[8 * v4 + 5] * inv);
+            w.w = pack_bf16(o[8 * v4 + 6] * inv, o[8 * v4 + 7] * inv);
+            reinterpret_cast<uint4 *>(orow + cc * 32)[v4] = w;
+          }
+        }
+      }
+      if (prm.lse != nullptr && qi < n_k)
+        prm.lse[(size_t)slice * n_k + qi] = (m_used + log2f(l)) * 0.6931471805599453f;
+      tc_fence_before();
+    }
+  }
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+  }
+}
+
+}  // namespace tc
+
+// Host side: tensor maps over the K and V pools (built once) and over Q (per call), launch.
 struct AttendTc {
-  bool init(int, int, void *, void *, long long, int, std::string &) { return true; }
-  bool enabled() const { return false; }
-  bool launch(const LayerView &, const TensorView &, const TensorView &, float *, int, int, float, cudaStream_t, std::string &) {
-    return false;
+  using EncodeFn = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+  EncodeFn encode = nullptr;
+  CUtensorMap tmK, tmV;
+  bool on = false;
+  int box_rows = 128;
+
+  bool init(int dtype, int head_dim, void *k_pool, void *v_pool, long long n_pages, int page_tokens, std::string &err) {
+    on = false;
+    if (dtype != 0 || head_dim != 128) return true;   // f32 x 64 is served by the FMA kernel
+    const char *env = std::getenv("SCALEKV_ATTEND");
+    if (env && std::string(env) == "simt") return true;
+    void *fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn) {
+      err = "cuTensorMapEncodeTiled not available";
+      return false;
+    }
+    encode = reinterpret_cast<EncodeFn>(fn);
+    box_rows = page_tokens < 128 ? page_tokens : 128;
+    const cuuint64_t dims[2] = {128, (cuuint64_t)n_pages * (cuuint64_t)page_tokens};
+    const cuuint64_t strides[1] = {256};
+    const cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    for (int i = 0; i < 2; ++i) {
+      CUresult r = encode(i == 0 ? &tmK : &tmV, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, i == 0 ? k_pool : v_pool, dims, strides, box,
+                          estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+      if (r != CUDA_SUCCESS) { err = "cuTensorMapEncodeTiled(pool) failed with code " + std::to_string((int)r); return false; }
+    }
+    if (cudaFuncSetAttribute(tc::attend_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc::kSmemBytes) != cudaSuccess) {
+      err = "cannot raise the dynamic shared memory limit";
+      return false;
+    }
+    on = true;
+    return true;
+  }
+  bool enabled() const { return on; }
+
+  bool launch(const LayerView &lv, const TensorView &Q, const TensorView &O, float *lse, int n_k, int /*L_host*/, float scale,
+              cudaStream_t stream, std::string &err) {
+    CUtensorMap tmQ;
+    const int B = lv.n_slices / lv.n_heads;
+    const cuuint64_t dims[4] = {128, (cuuint64_t)n_k, (cuuint64_t)lv.n_heads, (cuuint64_t)B};
+    const cuuint64_t strides[3] = {(cuuint64_t)Q.st * 2, (cuuint64_t)Q.sh * 2, (cuuint64_t)Q.sb * 2};
+    const cuuint32_t box[4] = {64, 128, 1, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = encode(&tmQ, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<char *>(Q.ptr), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { err = "cuTensorMapEncodeTiled(Q) failed with code " + std::to_string((int)r); return false; }
+    tc::Params prm;
+    prm.lv = lv; prm.O = O; prm.lse = lse; prm.n_k = n_k;
+    prm.scale_log2e = scale * 1.4426950408889634f;
+    prm.box_rows = box_rows;
+    dim3 grid((n_k + 127) / 128, lv.n_slices);
+    tc::attend_tc_kernel<<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(tmQ, tmK, tmV, prm);
+    return true;
   }
 };
 

@@ -329,6 +329,8 @@ scalekv_status scalekv_init(const scalekv_config *cfg, scalekv_ctx **out) {
   }
   if (cudaMemcpy(ctx->pool + p.off_pt, ctx->page_table_host.data(), p.pt_elems * 4, cudaMemcpyHostToDevice) != cudaSuccess)
     return bail(SCALEKV_ERR_CUDA);
+  // pages start out as zeros: tiles are loaded whole, and rows beyond a slice's length must be finite
+  if (cudaMemset(ctx->pool + p.off_k, 0, p.off_pos - p.off_k) != cudaSuccess) return bail(SCALEKV_ERR_CUDA);
   if (cudaMemset(ctx->pool + p.off_len, 0, (size_t)p.n_layers * p.n_slices * 4) != cudaSuccess) return bail(SCALEKV_ERR_CUDA);
   if (cudaMemset(ctx->pool + p.off_status, 0, 256) != cudaSuccess) return bail(SCALEKV_ERR_CUDA);
   ctx->next_scale.assign(p.n_layers, 0);
