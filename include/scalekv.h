@@ -203,6 +203,36 @@ scalekv_status scalekv_launch_count(scalekv_ctx *ctx, int64_t *count);
 scalekv_status scalekv_profile_enable(scalekv_ctx *ctx, int32_t on);
 scalekv_status scalekv_profile_read(scalekv_ctx *ctx, int32_t which, double *ms_total, int64_t *launches);
 
+/* ---- allocation-free top-k ------------------------------------------------------------------ */
+
+/* (The paper has no counterpart of this call; it exists for integration reasons only.)
+ * Some hosts of this library may not allocate device memory at the point where they need a
+ * selection: an inference engine that sized every buffer at start-up and has handed the rest of
+ * the GPU to its own pool, or code running in a phase where an allocation (cudaMalloc
+ * synchronises the whole device) would stall concurrent work.  scalekv_select_static serves
+ * them: it needs no context, no pool and no workspace.  The keys of its radix select live in a
+ * fixed array inside the library image, so the call allocates nothing - no cudaMalloc, no
+ * cudaFree, no allocating library routine.
+ *
+ *   scores   device, n_rows rows of `len` non-negative finite floats, row stride `ld` (>= len)
+ *   k        1 <= k <= len: how many entries of each row to select
+ *   idx_out  device, [n_rows][k] int32: the ascending indices of each row's k largest scores;
+ *            equal scores are taken lowest index first (the rule of scalekv_compress)
+ *   stream   cudaStream_t of the CURRENT device; the kernel is enqueued there, the call returns
+ *
+ * Limit: n_rows * len <= SCALEKV_SELECT_STATIC_MAX_ENTRIES (4 MiB of keys); larger requests
+ * return SCALEKV_ERR_CAPACITY and print the reason to stderr.  Every device that loads the
+ * library holds this array until the process ends.
+ * The first call on each device looks up the array's device address (once, under a lock);
+ * make that first call before starting any stream capture on that device.
+ * All calls on a device share the one array and find in it whatever the previous call left;
+ * nothing in it has to start at zero, because every call first overwrites the keys it reads.
+ * Two calls whose kernels may overlap on the GPU (different streams, no ordering) race on it:
+ * order them on one stream or with events. */
+#define SCALEKV_SELECT_STATIC_MAX_ENTRIES (1 << 20)
+scalekv_status scalekv_select_static(const float *scores, int32_t n_rows, int32_t len, int32_t ld, int32_t k,
+                                     int32_t *idx_out, void *stream);
+
 /* Text of the last error of this context (never NULL; valid until the next call). */
 const char *scalekv_error_string(scalekv_ctx *ctx);
 

@@ -14,7 +14,7 @@ import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libscalekv.so")
-SOURCES = [os.path.join(_HERE, "csrc", f) for f in ("scalekv.cu", "kernels_simt.cuh", "attend_tc.cuh", "common.cuh")]
+SOURCES = [os.path.join(_HERE, "csrc", f) for f in ("scalekv.cu", "select_static.cu", "kernels_simt.cuh", "attend_tc.cuh", "common.cuh")]
 HEADER = os.path.join(os.path.dirname(_HERE), "include", "scalekv.h")
 
 KEEP_ALL = -1
@@ -54,7 +54,7 @@ def build_library(force=False, verbose=False):
         if os.path.getmtime(LIB_PATH) >= newest:
             return LIB_PATH
     cmd = ["nvcc", "-shared", "-Xcompiler", "-fPIC", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
-           "-O3", "-std=c++17", SOURCES[0], "-o", LIB_PATH]
+           "-O3", "-std=c++17", SOURCES[0], SOURCES[1], "-o", LIB_PATH]
     if verbose:
         cmd.insert(1, "-Xptxas=-v")
     res = subprocess.run(cmd, capture_output=True, text=True)
@@ -100,6 +100,7 @@ def load_library():
         "scalekv_launch_count": [ctx_p, P(i64)],
         "scalekv_profile_enable": [ctx_p, i32],
         "scalekv_profile_read": [ctx_p, i32, P(f64), P(i64)],
+        "scalekv_select_static": [C.c_void_p, i32, i32, i32, i32, C.c_void_p, C.c_void_p],
     }
     for name, args in sig.items():
         fn = getattr(lib, name)
@@ -167,6 +168,23 @@ def scalekv_make_budgets(is_drafter, b_uniform, b_r0, delta):
     if st:
         raise ScaleKVError(st)
     return out
+
+
+def scalekv_select_static(scores: torch.Tensor, k: int, idx_out: torch.Tensor = None, stream=None):
+    """Allocation-free top-k: scores [n_rows, len] float32 on the current CUDA device (row stride
+    = scores.stride(0)); returns idx_out [n_rows, k] int32, the ascending indices of each row's k
+    largest scores.  The library call itself allocates nothing; pass idx_out to avoid the torch
+    allocation made here for convenience."""
+    lib = load_library()
+    assert scores.is_cuda and scores.dtype == torch.float32 and scores.dim() == 2 and scores.stride(1) == 1
+    n_rows, length = scores.shape
+    if idx_out is None:
+        idx_out = torch.empty(n_rows, k, dtype=torch.int32, device=scores.device)
+    st = stream if stream is not None else torch.cuda.current_stream(scores.device)
+    rc = lib.scalekv_select_static(scores.data_ptr(), n_rows, length, scores.stride(0), k, idx_out.data_ptr(), st.cuda_stream)
+    if rc:
+        raise ScaleKVError(rc, "scalekv_select_static")
+    return idx_out
 
 
 # ---- the context ---------------------------------------------------------------------------
