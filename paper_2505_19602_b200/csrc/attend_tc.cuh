@@ -1,16 +1,21 @@
 // Tensor-core attention over the paged store for bf16, head_dim 128 (Sec. 3.3, Eq. 5):
-// O = softmax(scale * Q K^T) V with online softmax, one CTA per (slice, 128-query tile).
+// O = softmax(scale * Q K^T) V with online softmax.  One CTA owns up to two 128-query tiles (A, B)
+// of one slice and streams the slice's K/V pages once for both.
 //
-// Roles inside a CTA of 192 threads:
-//   warp 0 (one thread) : TMA producer.  Q tile once; then per 128-key tile the K and V rows, page
-//                         by page through the slice's page table, into 128B-swizzled shared memory.
-//   warp 1 (one thread) : tcgen05.mma issuer.  S_j = Q K_j^T into one of two TMEM buffers, then
-//                         O += P_{j-1} V_{j-1}; S_j is issued before the PV of the previous tile so the
-//                         tensor pipe works under the softmax of tile j-1.  Owns the TMEM allocation.
-//   warps 2-5           : softmax.  Each thread owns one query row (TMEM lane): tcgen05.ld of the S
-//                         row, running max with lazy rescale (O is only rescaled when the max grows by
-//                         more than 2^8), exp2, bf16 P written to shared memory in the K-major swizzled
-//                         operand layout, and at the end the O / l epilogue.
+// Roles inside a CTA of 320 threads:
+//   warp 0 (one thread) : TMA producer.  The query tiles once; then per 128-key tile the K and V rows,
+//                         page by page through the slice's page table, into 128B-swizzled shared memory.
+//   warp 1 (one thread) : tcgen05.mma issuer; owns the TMEM allocation (512 columns: two S/P buffers
+//                         and two O accumulators).  With two query tiles the issue order per key tile
+//                         j is  S_A(j), PV_B(j-1), S_B(j), PV_A(j): while one tile's softmax runs, the
+//                         tensor pipe works for the other tile.  With one query tile the two S buffers
+//                         alternate and S(j+1) is issued ahead of PV(j).
+//   warps 2-5 / 6-9     : softmax of tile A / tile B.  Each thread owns one query row (one TMEM lane):
+//                         a first sweep over the S row (tcgen05.ld) finds the row maximum, a second one
+//                         computes exp2 with packed f32x2 arithmetic and writes P as bf16 pairs back
+//                         into the S buffer's columns (tcgen05.st), from where the PV product takes
+//                         its A operand.  O is rescaled lazily, only when the running maximum grew by
+//                         more than 2^8.  At the end the same warps normalise and store O.
 // Every mbarrier wait is bounded; a wait that gives up raises the sticky device status, sets a
 // CTA-wide abort flag and all roles fall through to the common exit where TMEM is released.
 #pragma once
@@ -25,20 +30,19 @@
 namespace scalekv {
 namespace tc {
 
-constexpr int kThreads = 192;
+constexpr int kThreads = 320;
 constexpr int kKStages = 2, kVStages = 2;
 constexpr uint32_t kTileBytes = 128 * 128 * 2;   // one 128 x 128 bf16 operand tile
 constexpr uint32_t kHalfBytes = kTileBytes / 2;  // 64 head-dim columns = one 128-byte swizzle span
-constexpr uint32_t kOffQ = 0;
-constexpr uint32_t kOffP = kOffQ + kTileBytes;
-constexpr uint32_t kOffK = kOffP + kTileBytes;
+constexpr uint32_t kOffQ = 0;                    // two query tiles
+constexpr uint32_t kOffK = kOffQ + 2 * kTileBytes;
 constexpr uint32_t kOffV = kOffK + kKStages * kTileBytes;
 constexpr uint32_t kOffBar = kOffV + kVStages * kTileBytes;
 constexpr uint32_t kSmemBytes = kOffBar + 256 + 1024;  // + barriers + alignment slack
-// barrier slots (8 bytes each)
-enum { bQFull = 0, bKFull = 1, bKEmpty = 3, bVFull = 5, bVEmpty = 7, bSFull = 9, bSEmpty = 11, bPFull = 13, bPvDone = 14, bCount = 15 };
+// barrier slots (8 bytes each); [2] = one per stage or per S buffer / query tile
+enum { bQFull = 0, bKFull = 1, bKEmpty = 3, bVFull = 5, bVEmpty = 7, bSFull = 9, bPFull = 11, bPvDone = 13, bCount = 15 };
 constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kColS = 0, kColO = 256;
+constexpr uint32_t kColS = 0, kColO = 256;       // S/P buffers at 0 and 128, O accumulators at 256 and 384
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -109,11 +113,20 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+// D[tmem] (+)= A[smem] * B[smem]
+__device__ __forceinline__ void tc_mma_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
   asm volatile(
       "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
       "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem]
+__device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
@@ -150,6 +163,15 @@ __device__ __forceinline__ void tc_st32(uint32_t taddr, const float *v) {
       "r"(__float_as_uint(v[28])), "r"(__float_as_uint(v[29])), "r"(__float_as_uint(v[30])), "r"(__float_as_uint(v[31]))
       : "memory");
 }
+// 16 consecutive 32-bit columns (32 bf16 values of P) of this thread's TMEM lane
+__device__ __forceinline__ void tc_st16(uint32_t taddr, const uint32_t *v) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};" ::"r"(taddr),
+      "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]), "r"(v[9]), "r"(v[10]),
+      "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
+      : "memory");
+}
 
 __device__ __forceinline__ float ex2(float x) {
   float y;
@@ -161,9 +183,33 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
   return r;
 }
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
+// packed pairs of fp32 in one 64-bit register
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float &lo, float &hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
 
 // Shared-memory matrix descriptor, 128-byte swizzle, operand tiles whose 8-row groups are 1024 B
-// apart.  K-major operands (Q, K, P): rows of 128 B, the leading offset is not used.  MN-major
+// apart.  K-major operands (Q, K): rows of 128 B, the leading offset is not used.  MN-major
 // operand (V as [key][d]): 64 d-columns are contiguous, the next 64 start `lbo` bytes further.
 __device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
   uint64_t d = 0;
@@ -203,8 +249,9 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   const LayerView &lv = prm.lv;
   const int slice = blockIdx.y;
   const int b = slice / lv.n_heads, h = slice % lv.n_heads;
-  const int q0 = blockIdx.x * 128;
   const int n_k = prm.n_k;
+  const int q_first = blockIdx.x * 256;                  // first query row of tile A
+  const bool single = q_first + 128 >= n_k;              // tile B would be empty
   const int L = lv.hist_len[slice] + n_k;
   const int T = (L + 127) >> 7;
   int *status = lv.status;
@@ -219,10 +266,9 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       mbar_init(bar(bVFull + s), 1);
       mbar_init(bar(bVEmpty + s), 1);
       mbar_init(bar(bSFull + s), 1);
-      mbar_init(bar(bSEmpty + s), 128);
+      mbar_init(bar(bPFull + s), 128);
+      mbar_init(bar(bPvDone + s), 1);
     }
-    mbar_init(bar(bPFull), 128);
-    mbar_init(bar(bPvDone), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -238,9 +284,12 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   if (warp == 0) {
     if (lane == 0) {
       // ---------------------------------------------------------------- TMA producer
-      mbar_expect_tx(bar(bQFull), kTileBytes);
-      tma_load_4d(base + kOffQ, &tmQ, 0, q0, h, b, bar(bQFull));
-      tma_load_4d(base + kOffQ + kHalfBytes, &tmQ, 64, q0, h, b, bar(bQFull));
+      const int nq = single ? 1 : 2;
+      mbar_expect_tx(bar(bQFull), nq * kTileBytes);
+      for (int t = 0; t < nq; ++t) {
+        tma_load_4d(base + kOffQ + t * kTileBytes, &tmQ, 0, q_first + t * 128, h, b, bar(bQFull));
+        tma_load_4d(base + kOffQ + t * kTileBytes + kHalfBytes, &tmQ, 64, q_first + t * 128, h, b, bar(bQFull));
+      }
       const int R = prm.box_rows;
       const int last_page = (L - 1) >> lv.page_shift;
       const int *pt = lv.page_table + (size_t)slice * lv.pages_per_slice;
@@ -279,152 +328,177 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       constexpr uint32_t idesc_qk = instr_desc(false);
       constexpr uint32_t idesc_pv = instr_desc(true);
       bool ok = mbar_wait(bar(bQFull), 0, abort_flag, status);
-      auto issue_pv = [&](int t) -> bool {
-        const int vs = t % kVStages;
-        if (!mbar_wait(bar(bVFull + vs), (t / kVStages) & 1, abort_flag, status)) return false;
-        if (!mbar_wait(bar(bPFull), t & 1, abort_flag, status)) return false;
-        tc_fence_after();
-        const uint32_t p_addr = base + kOffP, v_addr = base + kOffV + vs * kTileBytes;
-#pragma unroll
-        for (int kk = 0; kk < 8; ++kk) {
-          const uint64_t ad = smem_desc(p_addr + (kk >> 2) * kHalfBytes + (kk & 3) * 32, 16, 1024);
-          const uint64_t bd = smem_desc(v_addr + kk * 2048, kHalfBytes, 1024);
-          tc_mma(tmem + kColO, ad, bd, idesc_pv, (t > 0 || kk > 0) ? 1u : 0u);
-        }
-        tc_commit(bar(bVEmpty + vs));
-        tc_commit(bar(bPvDone));
-        return true;
-      };
-      for (int j = 0; j < T && ok; ++j) {
-        const int sb = j & 1, ks = j % kKStages;
-        ok = mbar_wait(bar(bKFull + ks), (j / kKStages) & 1, abort_flag, status) &&
-             mbar_wait(bar(bSEmpty + sb), ((j >> 1) & 1) ^ 1, abort_flag, status);
-        if (!ok) break;
-        tc_fence_after();
-        const uint32_t q_addr = base + kOffQ, k_addr = base + kOffK + ks * kTileBytes;
+      // S buffer `buf` = Q tile `qt` times K tile j (transposed)
+      auto issue_s = [&](int j, int qt, int buf) {
+        const uint32_t q_addr = base + kOffQ + qt * kTileBytes, k_addr = base + kOffK + (j % kKStages) * kTileBytes;
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk) {
           const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
-          tc_mma(tmem + kColS + sb * 128, smem_desc(q_addr + off, 16, 1024), smem_desc(k_addr + off, 16, 1024), idesc_qk,
-                 kk > 0 ? 1u : 0u);
+          tc_mma_ss(tmem + kColS + buf * 128, smem_desc(q_addr + off, 16, 1024), smem_desc(k_addr + off, 16, 1024), idesc_qk,
+                    kk > 0 ? 1u : 0u);
         }
-        tc_commit(bar(bKEmpty + ks));
-        tc_commit(bar(bSFull + sb));
-        if (j > 0) ok = issue_pv(j - 1);
+        tc_commit(bar(bSFull + buf));
+      };
+      // O of tile `qt` += P (bf16 pairs in S buffer `buf`) times V tile t
+      auto issue_pv = [&](int t, int qt, int buf, uint32_t p_parity, bool release_v) -> bool {
+        const int vs = t % kVStages;
+        if (!mbar_wait(bar(bVFull + vs), (t / kVStages) & 1, abort_flag, status)) return false;
+        if (!mbar_wait(bar(bPFull + buf), p_parity, abort_flag, status)) return false;
+        tc_fence_after();
+        const uint32_t v_addr = base + kOffV + vs * kTileBytes;
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk)
+          tc_mma_ts(tmem + kColO + qt * 128, tmem + kColS + buf * 128 + kk * 8, smem_desc(v_addr + kk * 2048, kHalfBytes, 1024),
+                    idesc_pv, (t > 0 || kk > 0) ? 1u : 0u);
+        tc_commit(bar(bPvDone + qt));
+        if (release_v) tc_commit(bar(bVEmpty + vs));
+        return true;
+      };
+      if (!single) {
+        for (int j = 0; j < T && ok; ++j) {
+          ok = mbar_wait(bar(bKFull + j % kKStages), (j / kKStages) & 1, abort_flag, status);
+          if (!ok) break;
+          tc_fence_after();
+          issue_s(j, 0, 0);
+          if (j > 0) ok = issue_pv(j - 1, 1, 1, (j - 1) & 1, true);
+          if (!ok) break;
+          issue_s(j, 1, 1);
+          tc_commit(bar(bKEmpty + j % kKStages));
+          ok = issue_pv(j, 0, 0, j & 1, false);
+        }
+        if (ok) issue_pv(T - 1, 1, 1, (T - 1) & 1, true);
+      } else {
+        for (int j = 0; j < T && ok; ++j) {
+          ok = mbar_wait(bar(bKFull + j % kKStages), (j / kKStages) & 1, abort_flag, status);
+          if (!ok) break;
+          tc_fence_after();
+          issue_s(j, 0, j & 1);
+          tc_commit(bar(bKEmpty + j % kKStages));
+          if (j > 0) ok = issue_pv(j - 1, 0, (j - 1) & 1, ((j - 1) >> 1) & 1, true);
+        }
+        if (ok) issue_pv(T - 1, 0, (T - 1) & 1, ((T - 1) >> 1) & 1, true);
       }
-      if (ok) issue_pv(T - 1);
     }
   } else {
     // ------------------------------------------------------------------ softmax + epilogue
-    const int q = warp & 3;
-    const int row = q * 32 + lane;
-    const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16);
-    const float c = prm.scale_log2e;
-    float m_used = -INFINITY, l = 0.f;
-    bool ok = true;
-    for (int j = 0; j < T && ok; ++j) {
-      const int sb = j & 1;
-      ok = mbar_wait_warp(bar(bSFull + sb), (j >> 1) & 1, abort_flag, status);
-      if (!ok) break;
-      tc_fence_after();
-      float s[128];
+    const int qt = (warp - 2) >> 2;              // 0: tile A, 1: tile B
+    if (!(single && qt == 1)) {
+      const int quarter = warp & 3;              // the TMEM lane quarter this warp may access
+      const int row = quarter * 32 + lane;
+      const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
+      const float c = prm.scale_log2e;
+      const uint64_t c2 = pack2(c, c);
+      float m_used = -INFINITY, l = 0.f;
+      bool ok = true;
+      for (int j = 0; j < T && ok; ++j) {
+        const int buf = single ? (j & 1) : qt;
+        const uint32_t par = single ? ((j >> 1) & 1) : (j & 1);
+        ok = mbar_wait_warp(bar(bSFull + buf), par, abort_flag, status);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t s_addr = lane_addr + kColS + buf * 128;
+        const int valid = L - j * 128;             // < 128 only in the last tile
+        float v[2][32];
+        // sweep 1: row maximum
+        float mt = -INFINITY;
+        tc_ld32(s_addr, v[0]);
 #pragma unroll
-      for (int cc = 0; cc < 4; ++cc) tc_ld32(lane_addr + kColS + sb * 128 + cc * 32, s + cc * 32);
-      tc_wait_ld();
-      tc_fence_before();
-      mbar_arrive(bar(bSEmpty + sb));
-      if (j == T - 1) {
-        const int valid = L - j * 128;
-        if (valid < 128) {
+        for (int cc = 0; cc < 4; ++cc) {
+          tc_wait_ld();
+          if (cc < 3) tc_ld32(s_addr + (cc + 1) * 32, v[(cc + 1) & 1]);
+          float *x = v[cc & 1];
+          if (valid < 128) {
 #pragma unroll
-          for (int i = 0; i < 128; ++i)
-            if (i >= valid) s[i] = -INFINITY;
+            for (int i = 0; i < 32; ++i)
+              if (cc * 32 + i >= valid) x[i] = -INFINITY;
+          }
+#pragma unroll
+          for (int i = 0; i < 32; i += 2) mt = max3(mt, x[i], x[i + 1]);
         }
-      }
-      float mt = s[0];
-#pragma unroll
-      for (int i = 1; i < 128; ++i) mt = fmaxf(mt, s[i]);
-      const float mz = mt * c;
-      const bool need = mz > m_used + 8.f;
-      bool waited = false;
-      if (__any_sync(0xffffffffu, need)) {
-        if (j > 0) {
-          ok = mbar_wait_warp(bar(bPvDone), (j - 1) & 1, abort_flag, status);
-          if (!ok) break;
-          tc_fence_after();
-          waited = true;
-        }
-        const float m_new = need ? mz : m_used;
-        const float sc = need ? ex2(m_used - m_new) : 1.f;
-        l *= sc;
-        m_used = m_new;
-        if (j > 0) {
-#pragma unroll
-          for (int cc = 0; cc < 4; ++cc) {
-            float o[32];
-            tc_ld32(lane_addr + kColO + cc * 32, o);
+        // start the second sweep's first load before the (rare) rescale
+        tc_ld32(s_addr, v[0]);
+        const float mz = mt * c;
+        const bool need = mz > m_used + 8.f;
+        if (__any_sync(0xffffffffu, need)) {
+          const float m_new = need ? mz : m_used;
+          const float sc = need ? ex2(m_used - m_new) : 1.f;
+          l *= sc;
+          m_used = m_new;
+          if (j > 0) {
+            // the previous PV of this tile must have landed before O is touched
+            ok = mbar_wait_warp(bar(bPvDone + qt), (j - 1) & 1, abort_flag, status);
+            if (!ok) break;
+            tc_fence_after();
             tc_wait_ld();
 #pragma unroll
-            for (int i = 0; i < 32; ++i) o[i] *= sc;
-            tc_st32(lane_addr + kColO + cc * 32, o);
-          }
-          tc_wait_st();
-          tc_fence_before();
-        }
-      }
-      const float neg_m = -m_used;
-      uint32_t pk[64];
-      float sum = 0.f;
+            for (int cc = 0; cc < 4; ++cc) {
+              float o[32];
+              tc_ld32(lane_addr + kColO + qt * 128 + cc * 32, o);
+              tc_wait_ld();
 #pragma unroll
-      for (int i = 0; i < 64; ++i) {
-        const float p0 = ex2(fmaf(s[2 * i], c, neg_m));
-        const float p1 = ex2(fmaf(s[2 * i + 1], c, neg_m));
-        sum += p0 + p1;
-        pk[i] = pack_bf16(p0, p1);
-      }
-      l += sum;
-      if (!waited && j > 0) {
-        ok = mbar_wait_warp(bar(bPvDone), (j - 1) & 1, abort_flag, status);
-        if (!ok) break;
-      }
-      // P row -> shared memory, K-major 128B-swizzled operand layout (16-byte chunk index XOR row % 8)
-      const uint32_t prow = base + kOffP + row * 128;
-#pragma unroll
-      for (int ch = 0; ch < 16; ++ch) {
-        const uint32_t addr = prow + (ch >> 3) * kHalfBytes + (((ch & 7) ^ (row & 7)) << 4);
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(pk[4 * ch]), "r"(pk[4 * ch + 1]),
-                     "r"(pk[4 * ch + 2]), "r"(pk[4 * ch + 3])
-                     : "memory");
-      }
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      mbar_arrive(bar(bPFull));
-    }
-    if (ok) ok = mbar_wait_warp(bar(bPvDone), (T - 1) & 1, abort_flag, status);
-    if (ok) {
-      tc_fence_after();
-      const float inv = 1.f / l;
-      const int qi = q0 + row;
-      __nv_bfloat16 *orow = const_cast<__nv_bfloat16 *>(row_ptr<__nv_bfloat16>(prm.O, b, h, qi < n_k ? qi : 0));
-#pragma unroll
-      for (int cc = 0; cc < 4; ++cc) {
-        float o[32];
-        tc_ld32(lane_addr + kColO + cc * 32, o);
-        tc_wait_ld();
-        if (qi < n_k) {
-#pragma unroll
-          for (int v4 = 0; v4 < 4; ++v4) {
-            uint4 w;
-            w.x = pack_bf16(o[8 * v4 + 0] * inv, o[8 * v4 + 1] * inv);
-            w.y = pack_bf16(o[8 * v4 + 2] * inv, o[8 * v4 + 3] * inv);
-            w.z = pack_bf16(o[8 * v4 + 4] * inv, o[8 * v4 + 5] * inv);
-            w.w = pack_bf16(o[8 * v4 + 6] * inv, o[8 * v4 + 7] * inv);
-            reinterpret_cast<uint4 *>(orow + cc * 32)[v4] = w;
+              for (int i = 0; i < 32; ++i) o[i] *= sc;
+              tc_st32(lane_addr + kColO + qt * 128 + cc * 32, o);
+            }
           }
         }
+        // sweep 2: p = exp2(s * c - m), row sum, bf16 pairs back into the S buffer's columns
+        const uint64_t negm2 = pack2(-m_used, -m_used);
+        uint64_t sum2 = pack2(0.f, 0.f);
+#pragma unroll
+        for (int cc = 0; cc < 4; ++cc) {
+          tc_wait_ld();
+          if (cc < 3) tc_ld32(s_addr + (cc + 1) * 32, v[(cc + 1) & 1]);
+          float *x = v[cc & 1];
+          if (valid < 128) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (cc * 32 + i >= valid) x[i] = -INFINITY;
+          }
+          uint32_t pk[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            float a, bb;
+            unpack2(fma2(pack2(x[2 * i], x[2 * i + 1]), c2, negm2), a, bb);
+            const float p0 = ex2(a), p1 = ex2(bb);
+            sum2 = add2(sum2, pack2(p0, p1));
+            pk[i] = pack_bf16(p0, p1);
+          }
+          tc_st16(s_addr + cc * 16, pk);
+        }
+        float s0, s1;
+        unpack2(sum2, s0, s1);
+        l += s0 + s1;
+        tc_wait_st();
+        tc_fence_before();
+        mbar_arrive(bar(bPFull + buf));
       }
-      if (prm.lse != nullptr && qi < n_k)
-        prm.lse[(size_t)slice * n_k + qi] = (m_used + log2f(l)) * 0.6931471805599453f;
-      tc_fence_before();
+      if (ok) ok = mbar_wait_warp(bar(bPvDone + qt), (T - 1) & 1, abort_flag, status);
+      if (ok) {
+        tc_fence_after();
+        const float inv = 1.f / l;
+        const int qi = q_first + qt * 128 + row;
+        __nv_bfloat16 *orow = const_cast<__nv_bfloat16 *>(row_ptr<__nv_bfloat16>(prm.O, b, h, qi < n_k ? qi : 0));
+#pragma unroll
+        for (int cc = 0; cc < 4; ++cc) {
+          float o[32];
+          tc_ld32(lane_addr + kColO + qt * 128 + cc * 32, o);
+          tc_wait_ld();
+          if (qi < n_k) {
+#pragma unroll
+            for (int v4 = 0; v4 < 4; ++v4) {
+              uint4 w;
+              w.x = pack_bf16(o[8 * v4 + 0] * inv, o[8 * v4 + 1] * inv);
+              w.y = pack_bf16(o[8 * v4 + 2] * inv, o[8 * v4 + 3] * inv);
+              w.z = pack_bf16(o[8 * v4 + 4] * inv, o[8 * v4 + 5] * inv);
+              w.w = pack_bf16(o[8 * v4 + 6] * inv, o[8 * v4 + 7] * inv);
+              reinterpret_cast<uint4 *>(orow + cc * 32)[v4] = w;
+            }
+          }
+        }
+        if (prm.lse != nullptr && qi < n_k)
+          prm.lse[(size_t)slice * n_k + qi] = (m_used + log2f(l)) * 0.6931471805599453f;
+        tc_fence_before();
+      }
     }
   }
   __syncthreads();
@@ -494,7 +568,7 @@ struct AttendTc {
     prm.lv = lv; prm.O = O; prm.lse = lse; prm.n_k = n_k;
     prm.scale_log2e = scale * 1.4426950408889634f;
     prm.box_rows = box_rows;
-    dim3 grid((n_k + 127) / 128, lv.n_slices);
+    dim3 grid((n_k + 255) / 256, lv.n_slices);
     tc::attend_tc_kernel<<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(tmQ, tmK, tmV, prm);
     return true;
   }
