@@ -2,7 +2,7 @@
 // O = softmax(scale * Q K^T) V with online softmax.  One CTA owns up to two 128-query tiles (A, B)
 // of one slice and streams the slice's K/V pages once for both.
 //
-// Roles inside a CTA of 320 threads:
+// Roles inside a CTA of 384 threads (three warpgroups):
 //   warp 0 (one thread) : TMA producer.  The query tiles once; then per 128-key tile the K and V rows,
 //                         page by page through the slice's page table, into 128B-swizzled shared memory.
 //   warp 1 (one thread) : tcgen05.mma issuer; owns the TMEM allocation (512 columns: two S/P buffers
@@ -10,12 +10,14 @@
 //                         j is  S_A(j), PV_B(j-1), S_B(j), PV_A(j): while one tile's softmax runs, the
 //                         tensor pipe works for the other tile.  With one query tile the two S buffers
 //                         alternate and S(j+1) is issued ahead of PV(j).
-//   warps 2-5 / 6-9     : softmax of tile A / tile B.  Each thread owns one query row (one TMEM lane):
-//                         a first sweep over the S row (tcgen05.ld) finds the row maximum, a second one
-//                         computes exp2 with packed f32x2 arithmetic and writes P as bf16 pairs back
-//                         into the S buffer's columns (tcgen05.st), from where the PV product takes
-//                         its A operand.  O is rescaled lazily, only when the running maximum grew by
-//                         more than 2^8.  At the end the same warps normalise and store O.
+//   warps 4-7 / 8-11    : softmax of tile A / tile B.  Each thread owns one query row (one TMEM lane):
+//                         one sweep over the S row (tcgen05.ld) computes p = exp2(s * c - m) against the
+//                         running reference m with packed f32x2 arithmetic, the row sum and the
+//                         maximum of the exponents, and writes P as bf16 pairs back into the S
+//                         buffer's columns (tcgen05.st), from where the PV product takes its A
+//                         operand.  Only when a row's maximum outgrew m by more than 2^8 are P, the
+//                         row sum and O rescaled (by an exact power of two).  At the end the same
+//                         warps normalise and store O.
 // Every mbarrier wait is bounded; a wait that gives up raises the sticky device status, sets a
 // CTA-wide abort flag and all roles fall through to the common exit where TMEM is released.
 #pragma once
@@ -30,17 +32,18 @@
 namespace scalekv {
 namespace tc {
 
-constexpr int kThreads = 320;
-constexpr int kKStages = 2, kVStages = 2;
+constexpr int kThreads = 384;          // three warpgroups: {TMA, MMA, 2 idle warps}, softmax A, softmax B
+constexpr int kStages = 5;                       // one ring for the K and V tiles: K_0, V_0, K_1, V_1, ...
 constexpr uint32_t kTileBytes = 128 * 128 * 2;   // one 128 x 128 bf16 operand tile
 constexpr uint32_t kHalfBytes = kTileBytes / 2;  // 64 head-dim columns = one 128-byte swizzle span
 constexpr uint32_t kOffQ = 0;                    // two query tiles
-constexpr uint32_t kOffK = kOffQ + 2 * kTileBytes;
-constexpr uint32_t kOffV = kOffK + kKStages * kTileBytes;
-constexpr uint32_t kOffBar = kOffV + kVStages * kTileBytes;
+constexpr uint32_t kOffRing = kOffQ + 2 * kTileBytes;
+constexpr uint32_t kOffBar = kOffRing + kStages * kTileBytes;
 constexpr uint32_t kSmemBytes = kOffBar + 256 + 1024;  // + barriers + alignment slack
-// barrier slots (8 bytes each); [2] = one per stage or per S buffer / query tile
-enum { bQFull = 0, bKFull = 1, bKEmpty = 3, bVFull = 5, bVEmpty = 7, bSFull = 9, bPFull = 11, bPvDone = 13, bCount = 15 };
+// barrier slots (8 bytes each): one full/empty pair per ring stage, one S/P/PV barrier per S buffer or query tile
+enum { bQFull = 0, bFull = 1, bEmpty = bFull + kStages, bSFull = bEmpty + kStages, bPFull = bSFull + 2, bPvDone = bPFull + 2,
+       bCount = bPvDone + 2 };
+static_assert(bCount * 8 <= 192, "barriers overlap the TMEM slot");
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColS = 0, kColO = 256;       // S/P buffers at 0 and 128, O accumulators at 256 and 384
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
@@ -108,25 +111,38 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *tm,
       : "memory");
 }
 
+// True in exactly one lane of a converged warp.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
+  return pred != 0;
+}
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
+// The 64-bit shared-memory descriptors are passed as (low word, high word): the low word holds the
+// start address field, so stepping through a tile is one 32-bit add per operand.
 // D[tmem] (+)= A[smem] * B[smem]
-__device__ __forceinline__ void tc_mma_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+__device__ __forceinline__ void tc_mma_ss(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
+                                          uint32_t accumulate) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
-      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+      "mov.b64 da, {%1, %2};\n\tmov.b64 db, {%3, %4};\n\tsetp.ne.b32 p, %6, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}" ::"r"(d_tmem),
+      "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 // D[tmem] (+)= A[tmem] * B[smem]
-__device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+__device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
+                                          uint32_t accumulate) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d_tmem),
-      "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
+      "mov.b64 db, {%2, %3};\n\tsetp.ne.b32 p, %5, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}" ::"r"(d_tmem),
+      "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
@@ -211,18 +227,58 @@ __device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
 // Shared-memory matrix descriptor, 128-byte swizzle, operand tiles whose 8-row groups are 1024 B
 // apart.  K-major operands (Q, K): rows of 128 B, the leading offset is not used.  MN-major
 // operand (V as [key][d]): 64 d-columns are contiguous, the next 64 start `lbo` bytes further.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-  uint64_t d = 0;
-  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
-  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
-  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
-  d |= 1ull << 46;   // descriptor version of this architecture
-  d |= 2ull << 61;   // 128-byte swizzle
-  return d;
+// Low word: start address >> 4 (bits 0-13), leading byte offset >> 4 (bits 16-29).
+// High word: stride byte offset >> 4 (bits 0-13), descriptor version (bit 14), swizzle mode (bits 29-31).
+__device__ __forceinline__ uint32_t desc_lo(uint32_t saddr, uint32_t lbo_bytes) {
+  return ((saddr & 0x3FFFFu) >> 4) | (((lbo_bytes >> 4) & 0x3FFFu) << 16);
+}
+__host__ __device__ constexpr uint32_t desc_hi(uint32_t sbo_bytes) {
+  return ((sbo_bytes >> 4) & 0x3FFFu) | (1u << 14) | (2u << 29);
 }
 // Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = 128, A K-major; B K-major or MN-major.
 __host__ __device__ constexpr uint32_t instr_desc(bool b_mn_major) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+}
+
+// Rare path of the softmax (a row's maximum outgrew the reference by more than 2^8): the row's P is
+// recomputed from the S row, which is still intact at s_addr, against the new reference m_new and
+// written over the first 64 columns (a chunk's columns are only overwritten after it was read); the
+// O accumulator (128 fp32 columns at o_addr) is multiplied by sc once the previous PV product of
+// the tile has landed.  Returns the new row sum, or a negative number when a wait gave up.
+// Warp-collective.
+__device__ __noinline__ float redo_tile(uint32_t s_addr, uint32_t o_addr, int valid, float c, float m_new, float sc, bool with_o,
+                                        uint32_t pv_bar, uint32_t pv_parity, volatile int *abort_flag, int *status) {
+  float sum = 0.f;
+#pragma unroll 1
+  for (int cc = 0; cc < 4; ++cc) {
+    float x[32];
+    uint32_t pk[16];
+    tc_ld32(s_addr + cc * 32, x);
+    tc_wait_ld();
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const float p0 = (cc * 32 + 2 * i < valid) ? ex2(fmaf(x[2 * i], c, -m_new)) : 0.f;
+      const float p1 = (cc * 32 + 2 * i + 1 < valid) ? ex2(fmaf(x[2 * i + 1], c, -m_new)) : 0.f;
+      sum += p0 + p1;
+      pk[i] = pack_bf16(p0, p1);
+    }
+    tc_st16(s_addr + cc * 16, pk);
+  }
+  if (with_o) {
+    if (!mbar_wait_warp(pv_bar, pv_parity, abort_flag, status)) return -1.f;
+    tc_fence_after();
+#pragma unroll 1
+    for (int cc = 0; cc < 4; ++cc) {
+      float o[32];
+      tc_ld32(o_addr + cc * 32, o);
+      tc_wait_ld();
+#pragma unroll
+      for (int i = 0; i < 32; ++i) o[i] *= sc;
+      tc_st32(o_addr + cc * 32, o);
+    }
+  }
+  tc_wait_st();
+  return sum;
 }
 
 struct Params {
@@ -241,8 +297,8 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t *base_ptr = smem_raw + (base - smem_u32(smem_raw));
   const uint32_t bars = base + kOffBar;
-  volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(base_ptr + kOffBar + 128);
-  volatile int *abort_flag = reinterpret_cast<volatile int *>(base_ptr + kOffBar + 132);
+  volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(base_ptr + kOffBar + 192);
+  volatile int *abort_flag = reinterpret_cast<volatile int *>(base_ptr + kOffBar + 196);
   auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -260,11 +316,11 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   if (tid == 0) {
     *abort_flag = 0;
     mbar_init(bar(bQFull), 1);
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(bar(bFull + s), 1);
+      mbar_init(bar(bEmpty + s), 1);
+    }
     for (int s = 0; s < 2; ++s) {
-      mbar_init(bar(bKFull + s), 1);
-      mbar_init(bar(bKEmpty + s), 1);
-      mbar_init(bar(bVFull + s), 1);
-      mbar_init(bar(bVEmpty + s), 1);
       mbar_init(bar(bSFull + s), 1);
       mbar_init(bar(bPFull + s), 128);
       mbar_init(bar(bPvDone + s), 1);
@@ -272,7 +328,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(base + kOffBar + 128), "r"(kTmemCols)
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(base + kOffBar + 192), "r"(kTmemCols)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -281,107 +337,115 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
 
+  if (warp < 4) {
   if (warp == 0) {
-    if (lane == 0) {
+    {
       // ---------------------------------------------------------------- TMA producer
+      // (the whole warp walks the loop so that addresses stay warp-uniform; one lane issues)
       const int nq = single ? 1 : 2;
-      mbar_expect_tx(bar(bQFull), nq * kTileBytes);
-      for (int t = 0; t < nq; ++t) {
-        tma_load_4d(base + kOffQ + t * kTileBytes, &tmQ, 0, q_first + t * 128, h, b, bar(bQFull));
-        tma_load_4d(base + kOffQ + t * kTileBytes + kHalfBytes, &tmQ, 64, q_first + t * 128, h, b, bar(bQFull));
+      if (elect_one()) {
+        mbar_expect_tx(bar(bQFull), nq * kTileBytes);
+        for (int t = 0; t < nq; ++t) {
+          tma_load_4d(base + kOffQ + t * kTileBytes, &tmQ, 0, q_first + t * 128, h, b, bar(bQFull));
+          tma_load_4d(base + kOffQ + t * kTileBytes + kHalfBytes, &tmQ, 64, q_first + t * 128, h, b, bar(bQFull));
+        }
       }
       const int R = prm.box_rows;
       const int last_page = (L - 1) >> lv.page_shift;
       const int *pt = lv.page_table + (size_t)slice * lv.pages_per_slice;
       bool ok = true;
-      for (int j = 0; j < T && ok; ++j) {
-        const int ks = j % kKStages, vs = j % kVStages;
-        ok = mbar_wait(bar(bKEmpty + ks), ((j / kKStages) & 1) ^ 1, abort_flag, status);
+      // ring tile t = 2 j is K_j, t = 2 j + 1 is V_j
+      for (int t = 0; t < 2 * T && ok; ++t) {
+        const int st = t % kStages, j = t >> 1;
+        ok = mbar_wait_warp(bar(bEmpty + st), ((t / kStages) & 1) ^ 1, abort_flag, status);
         if (!ok) break;
-        mbar_expect_tx(bar(bKFull + ks), kTileBytes);
-        for (int r0 = 0; r0 < 128; r0 += R) {
-          const int slot = j * 128 + r0;
-          int lp = slot >> lv.page_shift;
-          lp = lp > last_page ? last_page : lp;
-          const int row = (__ldg(pt + lp) << lv.page_shift) + (slot & lv.page_mask);
-          const uint32_t dst = base + kOffK + ks * kTileBytes + r0 * 128;
-          tma_load_2d(dst, &tmK, 0, row, bar(bKFull + ks));
-          tma_load_2d(dst + kHalfBytes, &tmK, 64, row, bar(bKFull + ks));
+        const CUtensorMap *tm = (t & 1) ? &tmV : &tmK;
+        if (elect_one()) {
+          mbar_expect_tx(bar(bFull + st), kTileBytes);
+          for (int r0 = 0; r0 < 128; r0 += R) {
+            const int slot = j * 128 + r0;
+            int lp = slot >> lv.page_shift;
+            lp = lp > last_page ? last_page : lp;
+            const int row = (__ldg(pt + lp) << lv.page_shift) + (slot & lv.page_mask);
+            const uint32_t dst = base + kOffRing + st * kTileBytes + r0 * 128;
+            tma_load_2d(dst, tm, 0, row, bar(bFull + st));
+            tma_load_2d(dst + kHalfBytes, tm, 64, row, bar(bFull + st));
+          }
         }
-        ok = mbar_wait(bar(bVEmpty + vs), ((j / kVStages) & 1) ^ 1, abort_flag, status);
-        if (!ok) break;
-        mbar_expect_tx(bar(bVFull + vs), kTileBytes);
-        for (int r0 = 0; r0 < 128; r0 += R) {
-          const int slot = j * 128 + r0;
-          int lp = slot >> lv.page_shift;
-          lp = lp > last_page ? last_page : lp;
-          const int row = (__ldg(pt + lp) << lv.page_shift) + (slot & lv.page_mask);
-          const uint32_t dst = base + kOffV + vs * kTileBytes + r0 * 128;
-          tma_load_2d(dst, &tmV, 0, row, bar(bVFull + vs));
-          tma_load_2d(dst + kHalfBytes, &tmV, 64, row, bar(bVFull + vs));
-        }
+        __syncwarp();
       }
     }
   } else if (warp == 1) {
-    if (lane == 0) {
+    {
       // ---------------------------------------------------------------- MMA issuer
+      // (the whole warp walks the loop and waits; one elected lane issues the MMAs and commits)
       constexpr uint32_t idesc_qk = instr_desc(false);
       constexpr uint32_t idesc_pv = instr_desc(true);
-      bool ok = mbar_wait(bar(bQFull), 0, abort_flag, status);
+      bool ok = mbar_wait_warp(bar(bQFull), 0, abort_flag, status);
       // S buffer `buf` = Q tile `qt` times K tile j (transposed)
+      constexpr uint32_t dhi = desc_hi(1024);
+      const bool leader = elect_one();
+      const uint32_t q_lo[2] = {desc_lo(base + kOffQ, 16), desc_lo(base + kOffQ + kTileBytes, 16)};
       auto issue_s = [&](int j, int qt, int buf) {
-        const uint32_t q_addr = base + kOffQ + qt * kTileBytes, k_addr = base + kOffK + (j % kKStages) * kTileBytes;
+        const uint32_t a_lo = q_lo[qt], b_lo = desc_lo(base + kOffRing + ((2 * j) % kStages) * kTileBytes, 16);
+        const uint32_t d = tmem + kColS + buf * 128;
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk) {
-          const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
-          tc_mma_ss(tmem + kColS + buf * 128, smem_desc(q_addr + off, 16, 1024), smem_desc(k_addr + off, 16, 1024), idesc_qk,
-                    kk > 0 ? 1u : 0u);
+          constexpr uint32_t dummy = 0;
+          const uint32_t off = (((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4) + dummy;
+          if (leader) tc_mma_ss(d, a_lo + off, dhi, b_lo + off, dhi, idesc_qk, kk > 0 ? 1u : 0u);
         }
-        tc_commit(bar(bSFull + buf));
+        if (leader) tc_commit(bar(bSFull + buf));
+        __syncwarp();
       };
       // O of tile `qt` += P (bf16 pairs in S buffer `buf`) times V tile t
       auto issue_pv = [&](int t, int qt, int buf, uint32_t p_parity, bool release_v) -> bool {
-        const int vs = t % kVStages;
-        if (!mbar_wait(bar(bVFull + vs), (t / kVStages) & 1, abort_flag, status)) return false;
-        if (!mbar_wait(bar(bPFull + buf), p_parity, abort_flag, status)) return false;
+        const int vt = 2 * t + 1, vs = vt % kStages;
+        if (!mbar_wait_warp(bar(bFull + vs), (vt / kStages) & 1, abort_flag, status)) return false;
+        if (!mbar_wait_warp(bar(bPFull + buf), p_parity, abort_flag, status)) return false;
         tc_fence_after();
-        const uint32_t v_addr = base + kOffV + vs * kTileBytes;
+        const uint32_t b_lo = desc_lo(base + kOffRing + vs * kTileBytes, kHalfBytes);
+        const uint32_t d = tmem + kColO + qt * 128, a = tmem + kColS + buf * 128;
+        const uint32_t acc0 = t > 0 ? 1u : 0u;
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk)
-          tc_mma_ts(tmem + kColO + qt * 128, tmem + kColS + buf * 128 + kk * 8, smem_desc(v_addr + kk * 2048, kHalfBytes, 1024),
-                    idesc_pv, (t > 0 || kk > 0) ? 1u : 0u);
-        tc_commit(bar(bPvDone + qt));
-        if (release_v) tc_commit(bar(bVEmpty + vs));
+          if (leader) tc_mma_ts(d, a + kk * 8, b_lo + kk * (2048 >> 4), dhi, idesc_pv, kk > 0 ? 1u : acc0);
+        if (leader) {
+          tc_commit(bar(bPvDone + qt));
+          if (release_v) tc_commit(bar(bEmpty + vs));
+        }
+        __syncwarp();
         return true;
       };
       if (!single) {
         for (int j = 0; j < T && ok; ++j) {
-          ok = mbar_wait(bar(bKFull + j % kKStages), (j / kKStages) & 1, abort_flag, status);
+          ok = mbar_wait_warp(bar(bFull + (2 * j) % kStages), ((2 * j) / kStages) & 1, abort_flag, status);
           if (!ok) break;
           tc_fence_after();
           issue_s(j, 0, 0);
           if (j > 0) ok = issue_pv(j - 1, 1, 1, (j - 1) & 1, true);
           if (!ok) break;
           issue_s(j, 1, 1);
-          tc_commit(bar(bKEmpty + j % kKStages));
+          if (leader) tc_commit(bar(bEmpty + (2 * j) % kStages));
           ok = issue_pv(j, 0, 0, j & 1, false);
         }
         if (ok) issue_pv(T - 1, 1, 1, (T - 1) & 1, true);
       } else {
         for (int j = 0; j < T && ok; ++j) {
-          ok = mbar_wait(bar(bKFull + j % kKStages), (j / kKStages) & 1, abort_flag, status);
+          ok = mbar_wait_warp(bar(bFull + (2 * j) % kStages), ((2 * j) / kStages) & 1, abort_flag, status);
           if (!ok) break;
           tc_fence_after();
           issue_s(j, 0, j & 1);
-          tc_commit(bar(bKEmpty + j % kKStages));
+          if (leader) tc_commit(bar(bEmpty + (2 * j) % kStages));
           if (j > 0) ok = issue_pv(j - 1, 0, (j - 1) & 1, ((j - 1) >> 1) & 1, true);
         }
         if (ok) issue_pv(T - 1, 0, (T - 1) & 1, ((T - 1) >> 1) & 1, true);
       }
     }
+  }
   } else {
     // ------------------------------------------------------------------ softmax + epilogue
-    const int qt = (warp - 2) >> 2;              // 0: tile A, 1: tile B
+    const int qt = (warp - 4) >> 2;              // 0: tile A, 1: tile B
     if (!(single && qt == 1)) {
       const int quarter = warp & 3;              // the TMEM lane quarter this warp may access
       const int row = quarter * 32 + lane;
@@ -399,51 +463,33 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         const uint32_t s_addr = lane_addr + kColS + buf * 128;
         const int valid = L - j * 128;             // < 128 only in the last tile
         float v[2][32];
-        // sweep 1: row maximum
-        float mt = -INFINITY;
         tc_ld32(s_addr, v[0]);
+        if (j == 0) {
+          // first tile: a sweep of its own finds the row maximum that the exponentials refer to
+          float mt = -INFINITY;
 #pragma unroll
-        for (int cc = 0; cc < 4; ++cc) {
-          tc_wait_ld();
-          if (cc < 3) tc_ld32(s_addr + (cc + 1) * 32, v[(cc + 1) & 1]);
-          float *x = v[cc & 1];
-          if (valid < 128) {
-#pragma unroll
-            for (int i = 0; i < 32; ++i)
-              if (cc * 32 + i >= valid) x[i] = -INFINITY;
-          }
-#pragma unroll
-          for (int i = 0; i < 32; i += 2) mt = max3(mt, x[i], x[i + 1]);
-        }
-        // start the second sweep's first load before the (rare) rescale
-        tc_ld32(s_addr, v[0]);
-        const float mz = mt * c;
-        const bool need = mz > m_used + 8.f;
-        if (__any_sync(0xffffffffu, need)) {
-          const float m_new = need ? mz : m_used;
-          const float sc = need ? ex2(m_used - m_new) : 1.f;
-          l *= sc;
-          m_used = m_new;
-          if (j > 0) {
-            // the previous PV of this tile must have landed before O is touched
-            ok = mbar_wait_warp(bar(bPvDone + qt), (j - 1) & 1, abort_flag, status);
-            if (!ok) break;
-            tc_fence_after();
+          for (int cc = 0; cc < 4; ++cc) {
             tc_wait_ld();
+            if (cc < 3) tc_ld32(s_addr + (cc + 1) * 32, v[(cc + 1) & 1]);
+            float *x = v[cc & 1];
+            if (valid < 128) {
 #pragma unroll
-            for (int cc = 0; cc < 4; ++cc) {
-              float o[32];
-              tc_ld32(lane_addr + kColO + qt * 128 + cc * 32, o);
-              tc_wait_ld();
-#pragma unroll
-              for (int i = 0; i < 32; ++i) o[i] *= sc;
-              tc_st32(lane_addr + kColO + qt * 128 + cc * 32, o);
+              for (int i = 0; i < 32; ++i)
+                if (cc * 32 + i >= valid) x[i] = -INFINITY;
             }
+#pragma unroll
+            for (int i = 0; i < 32; i += 2) mt = max3(mt, x[i], x[i + 1]);
           }
+          m_used = mt * c;
+          tc_ld32(s_addr, v[0]);
         }
-        // sweep 2: p = exp2(s * c - m), row sum, bf16 pairs back into the S buffer's columns
+        // one sweep: x = s * c - m, p = exp2(x), row sum, maximum of x; the bf16 pairs of p stay in
+        // registers until the maximum is known to be inside the lazy band, then go to the S buffer's
+        // first 64 columns
         const uint64_t negm2 = pack2(-m_used, -m_used);
-        uint64_t sum2 = pack2(0.f, 0.f);
+        uint64_t sum2a = pack2(0.f, 0.f), sum2b = sum2a;
+        float xm0 = -INFINITY, xm1 = -INFINITY, xm2 = -INFINITY, xm3 = -INFINITY;
+        uint32_t pk[64];
 #pragma unroll
         for (int cc = 0; cc < 4; ++cc) {
           tc_wait_ld();
@@ -454,20 +500,50 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             for (int i = 0; i < 32; ++i)
               if (cc * 32 + i >= valid) x[i] = -INFINITY;
           }
-          uint32_t pk[16];
 #pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            float a, bb;
-            unpack2(fma2(pack2(x[2 * i], x[2 * i + 1]), c2, negm2), a, bb);
-            const float p0 = ex2(a), p1 = ex2(bb);
-            sum2 = add2(sum2, pack2(p0, p1));
-            pk[i] = pack_bf16(p0, p1);
+          for (int i = 0; i < 16; i += 4) {
+            float a0, a1, a2, a3, a4, a5, a6, a7;
+            unpack2(fma2(pack2(x[2 * i + 0], x[2 * i + 1]), c2, negm2), a0, a1);
+            unpack2(fma2(pack2(x[2 * i + 2], x[2 * i + 3]), c2, negm2), a2, a3);
+            unpack2(fma2(pack2(x[2 * i + 4], x[2 * i + 5]), c2, negm2), a4, a5);
+            unpack2(fma2(pack2(x[2 * i + 6], x[2 * i + 7]), c2, negm2), a6, a7);
+            xm0 = max3(xm0, a0, a1);
+            xm1 = max3(xm1, a2, a3);
+            xm2 = max3(xm2, a4, a5);
+            xm3 = max3(xm3, a6, a7);
+            const float p0 = ex2(a0), p1 = ex2(a1), p2 = ex2(a2), p3 = ex2(a3);
+            const float p4 = ex2(a4), p5 = ex2(a5), p6 = ex2(a6), p7 = ex2(a7);
+            sum2a = add2(sum2a, pack2(p0, p1));
+            sum2b = add2(sum2b, pack2(p2, p3));
+            sum2a = add2(sum2a, pack2(p4, p5));
+            sum2b = add2(sum2b, pack2(p6, p7));
+            pk[cc * 16 + i + 0] = pack_bf16(p0, p1);
+            pk[cc * 16 + i + 1] = pack_bf16(p2, p3);
+            pk[cc * 16 + i + 2] = pack_bf16(p4, p5);
+            pk[cc * 16 + i + 3] = pack_bf16(p6, p7);
           }
-          tc_st16(s_addr + cc * 16, pk);
         }
-        float s0, s1;
-        unpack2(sum2, s0, s1);
-        l += s0 + s1;
+        float s0, s1, s2, s3;
+        unpack2(sum2a, s0, s1);
+        unpack2(sum2b, s2, s3);
+        float lt = (s0 + s1) + (s2 + s3);
+        const float xmax = fmaxf(fmaxf(xm0, xm1), fmaxf(xm2, xm3));
+        // rare: the row maximum outgrew the reference by more than 2^8 (p may even have overflowed):
+        // move the reference to the new maximum and recompute the tile from S, which is still intact
+        if (__any_sync(0xffffffffu, xmax > 8.f)) {
+          const float m_new = xmax > 8.f ? m_used + xmax : m_used;
+          const float sc = ex2(m_used - m_new);
+          lt = redo_tile(s_addr, lane_addr + kColO + qt * 128, valid, c, m_new, sc, j > 0, bar(bPvDone + qt), (j - 1) & 1,
+                         abort_flag, status);
+          ok = __all_sync(0xffffffffu, lt >= 0.f);
+          if (!ok) break;
+          m_used = m_new;
+          l *= sc;
+        } else {
+#pragma unroll
+          for (int cc = 0; cc < 4; ++cc) tc_st16(s_addr + cc * 16, pk + cc * 16);
+        }
+        l += lt;
         tc_wait_st();
         tc_fence_before();
         mbar_arrive(bar(bPFull + buf));
