@@ -10,14 +10,17 @@
 //                         j is  S_A(j), PV_B(j-1), S_B(j), PV_A(j): while one tile's softmax runs, the
 //                         tensor pipe works for the other tile.  With one query tile the two S buffers
 //                         alternate and S(j+1) is issued ahead of PV(j).
-//   warps 4-7 / 8-11    : softmax of tile A / tile B.  Each thread owns one query row (one TMEM lane):
-//                         one sweep over the S row (tcgen05.ld) computes p = exp2(s * c - m) against the
-//                         running reference m with packed f32x2 arithmetic, the row sum and the
-//                         maximum of the exponents, and writes P as bf16 pairs back into the S
-//                         buffer's columns (tcgen05.st), from where the PV product takes its A
-//                         operand.  Only when a row's maximum outgrew m by more than 2^8 are P, the
-//                         row sum and O rescaled (by an exact power of two).  At the end the same
-//                         warps normalise and store O.
+//   warps 4-11          : softmax.  Warps 4-7 own columns 0-63 and warps 8-11 columns 64-127 of every S
+//                         tile; warp w and warp w + 4 share the 32 query rows (TMEM lanes) of quarter
+//                         w % 4, and all eight warps work on tile A's S, then on tile B's.  A thread
+//                         sweeps its half row once (tcgen05.ld): p = exp2(s * c - m) against the running
+//                         reference m with packed f32x2 arithmetic (a share of the exponentials on the
+//                         FMA pipe), the partial row sum, and P as bf16 pairs written back into the first
+//                         columns of its own half of the S buffer (tcgen05.st), from where the PV product
+//                         takes its A operand.  The two warps of a quarter meet on an mbarrier per tile:
+//                         only when a half row's sum shows that an exponent left the lazy band (2^8) do
+//                         both recompute the row against a new reference and rescale O.  At the end the
+//                         same warps normalise and store O, 64 columns each.
 // Every mbarrier wait is bounded; a wait that gives up raises the sticky device status, sets a
 // CTA-wide abort flag and all roles fall through to the common exit where TMEM is released.
 #pragma once
@@ -39,13 +42,15 @@ constexpr uint32_t kHalfBytes = kTileBytes / 2;  // 64 head-dim columns = one 12
 constexpr uint32_t kOffQ = 0;                    // two query tiles
 constexpr uint32_t kOffRing = kOffQ + 2 * kTileBytes;
 constexpr uint32_t kOffBar = kOffRing + kStages * kTileBytes;
-constexpr uint32_t kSmemBytes = kOffBar + 256 + 1024;  // + barriers + alignment slack
+constexpr uint32_t kOffX = kOffBar + 256;           // exchange area of the softmax warp pairs: flags [2][4][2], values [4][2][32]
+constexpr uint32_t kSmemBytes = kOffX + 1280 + 1024;   // + alignment slack
 // barrier slots (8 bytes each): one full/empty pair per ring stage, one S/P/PV barrier per S buffer or query tile
 enum { bQFull = 0, bFull = 1, bEmpty = bFull + kStages, bSFull = bEmpty + kStages, bPFull = bSFull + 2, bPvDone = bPFull + 2,
-       bCount = bPvDone + 2 };
+       bPair = bPvDone + 2, bCount = bPair + 4 };
 static_assert(bCount * 8 <= 192, "barriers overlap the TMEM slot");
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColS = 0, kColO = 256;       // S/P buffers at 0 and 128, O accumulators at 256 and 384
+constexpr int kPolyPairs = 1;                   // of every 4 pairs of exponentials, this many run on the FMA pipe
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -224,6 +229,26 @@ __device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
   return d;
 }
 
+// 2^x for a pair of exponents on the FMA pipe instead of the transcendental unit: x = n + f with
+// n = round(x) (magic-number rounding) and f in [-0.5, 0.5], 2^f by a cubic fitted for minimal relative
+// error (7.5e-5, far below the bf16 rounding of P), 2^n by adding n to the exponent field.
+// x is clamped to [-126, 127]: below, the result is smaller than every normal number; above, the
+// exponent field would wrap (the caller's overflow check sees 2^127).
+__device__ __forceinline__ void exp2_poly_pair(float x0, float x1, float &p0, float &p1) {
+  const uint64_t x = pack2(fminf(fmaxf(x0, -126.f), 127.f), fminf(fmaxf(x1, -126.f), 127.f));
+  const uint64_t t = add2(x, pack2(12582912.f, 12582912.f));            // 1.5 * 2^23: integer part lands in the mantissa
+  const uint64_t n = add2(t, pack2(-12582912.f, -12582912.f));
+  const uint64_t f = fma2(n, pack2(-1.f, -1.f), x);
+  uint64_t q = fma2(f, pack2(0.05517147481441498f, 0.05517147481441498f), pack2(0.242610901594162f, 0.242610901594162f));
+  q = fma2(q, f, pack2(0.6932609677314758f, 0.6932609677314758f));
+  q = fma2(q, f, pack2(0.9999281167984009f, 0.9999281167984009f));
+  float t0, t1, q0, q1;
+  unpack2(t, t0, t1);
+  unpack2(q, q0, q1);
+  p0 = __uint_as_float(__float_as_uint(q0) + (__float_as_uint(t0) << 23));
+  p1 = __uint_as_float(__float_as_uint(q1) + (__float_as_uint(t1) << 23));
+}
+
 // Shared-memory matrix descriptor, 128-byte swizzle, operand tiles whose 8-row groups are 1024 B
 // apart.  K-major operands (Q, K): rows of 128 B, the leading offset is not used.  MN-major
 // operand (V as [key][d]): 64 d-columns are contiguous, the next 64 start `lbo` bytes further.
@@ -240,17 +265,39 @@ __host__ __device__ constexpr uint32_t instr_desc(bool b_mn_major) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
 }
 
-// Rare path of the softmax (a row's maximum outgrew the reference by more than 2^8): the row's P is
-// recomputed from the S row, which is still intact at s_addr, against the new reference m_new and
-// written over the first 64 columns (a chunk's columns are only overwritten after it was read); the
-// O accumulator (128 fp32 columns at o_addr) is multiplied by sc once the previous PV product of
-// the tile has landed.  Returns the new row sum, or a negative number when a wait gave up.
-// Warp-collective.
-__device__ __noinline__ float redo_tile(uint32_t s_addr, uint32_t o_addr, int valid, float c, float m_new, float sc, bool with_o,
-                                        uint32_t pv_bar, uint32_t pv_parity, volatile int *abort_flag, int *status) {
+// Rare path of the softmax, taken together by the two warps that share a quarter's rows when the fast
+// sweep of one of their half rows overflowed the lazy band (always in the first tile, where no
+// reference exists yet).  The S half row is still intact at s_addr: a first sweep finds its maximum,
+// the two halves exchange theirs through shared memory (mine -> x_mine, the partner's <- x_other, with
+// one rendezvous on pair_bar), the reference moves up to the row maximum if that is larger, the half
+// row's P is recomputed against it and written over the first 32 columns (a chunk's columns are only
+// overwritten after it was read), and this warp's 64 columns of the O accumulator at o_addr are
+// multiplied by 2^(old reference - new reference) once the previous PV product of the tile has landed.
+// `valid` = number of columns of this half that hold keys (may be <= 0).  Returns the half row's sum
+// and the new reference; sum < 0 when a wait gave up.
+struct Redo { float sum, m; };
+__device__ __noinline__ Redo redo_half(uint32_t s_addr, uint32_t o_addr, int valid, float c, float m_used, bool with_o,
+                                       uint32_t pv_bar, uint32_t pv_parity, uint32_t pair_bar, uint32_t pair_parity,
+                                       volatile float *x_mine, volatile float *x_other, volatile int *abort_flag, int *status) {
+  float mt = -INFINITY;
+#pragma unroll 1
+  for (int cc = 0; cc < 2; ++cc) {
+    float x[32];
+    tc_ld32(s_addr + cc * 32, x);
+    tc_wait_ld();
+#pragma unroll
+    for (int i = 0; i < 32; ++i)
+      if (cc * 32 + i < valid) mt = fmaxf(mt, x[i]);
+  }
+  *x_mine = mt;
+  mbar_arrive(pair_bar);
+  if (!mbar_wait_warp(pair_bar, pair_parity, abort_flag, status)) return {-1.f, m_used};
+  mt = fmaxf(mt, *x_other);
+  const float m_new = fmaxf(m_used, mt * c);
+  const float sc = ex2(m_used - m_new);
   float sum = 0.f;
 #pragma unroll 1
-  for (int cc = 0; cc < 4; ++cc) {
+  for (int cc = 0; cc < 2; ++cc) {
     float x[32];
     uint32_t pk[16];
     tc_ld32(s_addr + cc * 32, x);
@@ -265,10 +312,10 @@ __device__ __noinline__ float redo_tile(uint32_t s_addr, uint32_t o_addr, int va
     tc_st16(s_addr + cc * 16, pk);
   }
   if (with_o) {
-    if (!mbar_wait_warp(pv_bar, pv_parity, abort_flag, status)) return -1.f;
+    if (!mbar_wait_warp(pv_bar, pv_parity, abort_flag, status)) return {-1.f, m_new};
     tc_fence_after();
 #pragma unroll 1
-    for (int cc = 0; cc < 4; ++cc) {
+    for (int cc = 0; cc < 2; ++cc) {
       float o[32];
       tc_ld32(o_addr + cc * 32, o);
       tc_wait_ld();
@@ -278,7 +325,7 @@ __device__ __noinline__ float redo_tile(uint32_t s_addr, uint32_t o_addr, int va
     }
   }
   tc_wait_st();
-  return sum;
+  return {sum, m_new};
 }
 
 struct Params {
@@ -322,9 +369,10 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     }
     for (int s = 0; s < 2; ++s) {
       mbar_init(bar(bSFull + s), 1);
-      mbar_init(bar(bPFull + s), 128);
+      mbar_init(bar(bPFull + s), 256);
       mbar_init(bar(bPvDone + s), 1);
     }
+    for (int s = 0; s < 4; ++s) mbar_init(bar(bPair + s), 64);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -398,7 +446,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         if (leader) tc_commit(bar(bSFull + buf));
         __syncwarp();
       };
-      // O of tile `qt` += P (bf16 pairs in S buffer `buf`) times V tile t
+      // O of tile `qt` += P (bf16 pairs in the first 32 columns of each half of S buffer `buf`) times V tile t
       auto issue_pv = [&](int t, int qt, int buf, uint32_t p_parity, bool release_v) -> bool {
         const int vt = 2 * t + 1, vs = vt % kStages;
         if (!mbar_wait_warp(bar(bFull + vs), (vt / kStages) & 1, abort_flag, status)) return false;
@@ -409,7 +457,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         const uint32_t acc0 = t > 0 ? 1u : 0u;
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk)
-          if (leader) tc_mma_ts(d, a + kk * 8, b_lo + kk * (2048 >> 4), dhi, idesc_pv, kk > 0 ? 1u : acc0);
+          if (leader) tc_mma_ts(d, a + (kk >> 2) * 64 + (kk & 3) * 8, b_lo + kk * (2048 >> 4), dhi, idesc_pv, kk > 0 ? 1u : acc0);
         if (leader) {
           tc_commit(bar(bPvDone + qt));
           if (release_v) tc_commit(bar(bEmpty + vs));
@@ -445,57 +493,47 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   }
   } else {
     // ------------------------------------------------------------------ softmax + epilogue
-    const int qt = (warp - 4) >> 2;              // 0: tile A, 1: tile B
-    if (!(single && qt == 1)) {
-      const int quarter = warp & 3;              // the TMEM lane quarter this warp may access
-      const int row = quarter * 32 + lane;
-      const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
-      const float c = prm.scale_log2e;
-      const uint64_t c2 = pack2(c, c);
-      float m_used = -INFINITY, l = 0.f;
-      bool ok = true;
-      for (int j = 0; j < T && ok; ++j) {
+    const int half = (warp - 4) >> 2;            // 0: columns 0-63, 1: columns 64-127 of every S tile
+    const int quarter = warp & 3;                // the TMEM lane quarter this warp may access
+    const int row = quarter * 32 + lane;
+    const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
+    const float c = prm.scale_log2e;
+    const uint64_t c2 = pack2(c, c);
+    volatile int *xflag = reinterpret_cast<volatile int *>(base_ptr + kOffX);           // [2][4][2]
+    volatile float *xval = reinterpret_cast<volatile float *>(base_ptr + kOffX + 64);   // [4][2][32]
+    volatile float *x_mine = xval + (quarter * 2 + half) * 32 + lane;
+    volatile float *x_other = xval + (quarter * 2 + (half ^ 1)) * 32 + lane;
+    const uint32_t pair_bar = bar(bPair + quarter);
+    uint32_t pair_uses = 0;                      // rendezvous so far of this quarter's two warps (same in both)
+    const int ntile = single ? 1 : 2;
+    float m_used[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f};
+    bool ok = true;
+    for (int j = 0; j < T && ok; ++j) {
+#pragma unroll
+      for (int qt = 0; qt < 2; ++qt) {
+        if (qt >= ntile || !ok) break;
         const int buf = single ? (j & 1) : qt;
         const uint32_t par = single ? ((j >> 1) & 1) : (j & 1);
         ok = mbar_wait_warp(bar(bSFull + buf), par, abort_flag, status);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t s_addr = lane_addr + kColS + buf * 128;
-        const int valid = L - j * 128;             // < 128 only in the last tile
+        const uint32_t s_addr = lane_addr + kColS + buf * 128 + half * 64;
+        const int valid = L - j * 128 - half * 64;     // < 64 only in the last tile; may be <= 0
         float v[2][32];
         tc_ld32(s_addr, v[0]);
-        if (j == 0) {
-          // first tile: a sweep of its own finds the row maximum that the exponentials refer to
-          float mt = -INFINITY;
-#pragma unroll
-          for (int cc = 0; cc < 4; ++cc) {
-            tc_wait_ld();
-            if (cc < 3) tc_ld32(s_addr + (cc + 1) * 32, v[(cc + 1) & 1]);
-            float *x = v[cc & 1];
-            if (valid < 128) {
-#pragma unroll
-              for (int i = 0; i < 32; ++i)
-                if (cc * 32 + i >= valid) x[i] = -INFINITY;
-            }
-#pragma unroll
-            for (int i = 0; i < 32; i += 2) mt = max3(mt, x[i], x[i + 1]);
-          }
-          m_used = mt * c;
-          tc_ld32(s_addr, v[0]);
-        }
-        // one sweep: x = s * c - m, p = exp2(x), row sum, maximum of x; the bf16 pairs of p stay in
-        // registers until the maximum is known to be inside the lazy band, then go to the S buffer's
-        // first 64 columns
-        const uint64_t negm2 = pack2(-m_used, -m_used);
+        // one sweep: x = s * c - m, p = exp2(x), partial row sum; the bf16 pairs of p stay in registers
+        // until both halves know that no exponent left the lazy band.  (64 values of at most 2^8 sum to
+        // at most 2^14; a larger, infinite or NaN sum means that some x exceeded 8 - or that there is no
+        // reference yet, m = -inf in the first tile.)
+        const uint64_t negm2 = pack2(-m_used[qt], -m_used[qt]);
         uint64_t sum2a = pack2(0.f, 0.f), sum2b = sum2a;
-        float xm0 = -INFINITY, xm1 = -INFINITY, xm2 = -INFINITY, xm3 = -INFINITY;
-        uint32_t pk[64];
+        uint32_t pk[32];
 #pragma unroll
-        for (int cc = 0; cc < 4; ++cc) {
+        for (int cc = 0; cc < 2; ++cc) {
           tc_wait_ld();
-          if (cc < 3) tc_ld32(s_addr + (cc + 1) * 32, v[(cc + 1) & 1]);
+          if (cc < 1) tc_ld32(s_addr + (cc + 1) * 32, v[(cc + 1) & 1]);
           float *x = v[cc & 1];
-          if (valid < 128) {
+          if (valid < 64) {
 #pragma unroll
             for (int i = 0; i < 32; ++i)
               if (cc * 32 + i >= valid) x[i] = -INFINITY;
@@ -507,12 +545,11 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             unpack2(fma2(pack2(x[2 * i + 2], x[2 * i + 3]), c2, negm2), a2, a3);
             unpack2(fma2(pack2(x[2 * i + 4], x[2 * i + 5]), c2, negm2), a4, a5);
             unpack2(fma2(pack2(x[2 * i + 6], x[2 * i + 7]), c2, negm2), a6, a7);
-            xm0 = max3(xm0, a0, a1);
-            xm1 = max3(xm1, a2, a3);
-            xm2 = max3(xm2, a4, a5);
-            xm3 = max3(xm3, a6, a7);
-            const float p0 = ex2(a0), p1 = ex2(a1), p2 = ex2(a2), p3 = ex2(a3);
-            const float p4 = ex2(a4), p5 = ex2(a5), p6 = ex2(a6), p7 = ex2(a7);
+            float p0, p1, p2, p3, p4, p5, p6, p7;
+            if (kPolyPairs > 0) exp2_poly_pair(a0, a1, p0, p1); else { p0 = ex2(a0); p1 = ex2(a1); }
+            if (kPolyPairs > 1) exp2_poly_pair(a2, a3, p2, p3); else { p2 = ex2(a2); p3 = ex2(a3); }
+            if (kPolyPairs > 2) exp2_poly_pair(a4, a5, p4, p5); else { p4 = ex2(a4); p5 = ex2(a5); }
+            if (kPolyPairs > 3) exp2_poly_pair(a6, a7, p6, p7); else { p6 = ex2(a6); p7 = ex2(a7); }
             sum2a = add2(sum2a, pack2(p0, p1));
             sum2b = add2(sum2b, pack2(p2, p3));
             sum2a = add2(sum2a, pack2(p4, p5));
@@ -526,56 +563,80 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         float s0, s1, s2, s3;
         unpack2(sum2a, s0, s1);
         unpack2(sum2b, s2, s3);
-        float lt = (s0 + s1) + (s2 + s3);
-        const float xmax = fmaxf(fmaxf(xm0, xm1), fmaxf(xm2, xm3));
-        // rare: the row maximum outgrew the reference by more than 2^8 (p may even have overflowed):
-        // move the reference to the new maximum and recompute the tile from S, which is still intact
-        if (__any_sync(0xffffffffu, xmax > 8.f)) {
-          const float m_new = xmax > 8.f ? m_used + xmax : m_used;
-          const float sc = ex2(m_used - m_new);
-          lt = redo_tile(s_addr, lane_addr + kColO + qt * 128, valid, c, m_new, sc, j > 0, bar(bPvDone + qt), (j - 1) & 1,
-                         abort_flag, status);
-          ok = __all_sync(0xffffffffu, lt >= 0.f);
+        const float lt = (s0 + s1) + (s2 + s3);
+        // the two warps of the quarter tell each other whether one of their rows needs the rare path
+        const int mine = __any_sync(0xffffffffu, !(lt <= 16384.f)) ? 1 : 0;
+        const int slot = (int)(pair_uses & 1u);
+        if (lane == 0) xflag[(slot * 4 + quarter) * 2 + half] = mine;
+        mbar_arrive(pair_bar);
+        ok = mbar_wait_warp(pair_bar, pair_uses & 1u, abort_flag, status);
+        ++pair_uses;
+        if (!ok) break;
+        if (mine | xflag[(slot * 4 + quarter) * 2 + (half ^ 1)]) {
+          const Redo r = redo_half(s_addr, lane_addr + kColO + qt * 128 + half * 64, valid, c, m_used[qt], j > 0, bar(bPvDone + qt),
+                                   (j - 1) & 1, pair_bar, pair_uses & 1u, x_mine, x_other, abort_flag, status);
+          ++pair_uses;
+          ok = __all_sync(0xffffffffu, r.sum >= 0.f);
           if (!ok) break;
-          m_used = m_new;
-          l *= sc;
+          l[qt] = l[qt] * ex2(m_used[qt] - r.m) + r.sum;
+          m_used[qt] = r.m;
         } else {
-#pragma unroll
-          for (int cc = 0; cc < 4; ++cc) tc_st16(s_addr + cc * 16, pk + cc * 16);
+          tc_st16(s_addr, pk);
+          tc_st16(s_addr + 16, pk + 16);
+          l[qt] += lt;
         }
-        l += lt;
         tc_wait_st();
         tc_fence_before();
         mbar_arrive(bar(bPFull + buf));
       }
-      if (ok) ok = mbar_wait_warp(bar(bPvDone + qt), (T - 1) & 1, abort_flag, status);
-      if (ok) {
-        tc_fence_after();
-        const float inv = 1.f / l;
-        const int qi = q_first + qt * 128 + row;
-        __nv_bfloat16 *orow = const_cast<__nv_bfloat16 *>(row_ptr<__nv_bfloat16>(prm.O, b, h, qi < n_k ? qi : 0));
+    }
+    if (ok) {
+      // a rendezvous of its own orders the partner's last read of the exchange area before its reuse
+      mbar_arrive(pair_bar);
+      ok = mbar_wait_warp(pair_bar, pair_uses & 1u, abort_flag, status);
+      ++pair_uses;
+    }
 #pragma unroll
-        for (int cc = 0; cc < 4; ++cc) {
-          float o[32];
-          tc_ld32(lane_addr + kColO + qt * 128 + cc * 32, o);
-          tc_wait_ld();
-          if (qi < n_k) {
+    for (int qt = 0; qt < 2; ++qt) {
+      if (qt >= ntile || !ok) break;
+      ok = mbar_wait_warp(bar(bPvDone + qt), (T - 1) & 1, abort_flag, status);
+      if (!ok) break;
+      tc_fence_after();
+      // the row sum is the sum of the two halves' partial sums
+      *x_mine = l[qt];
+      mbar_arrive(pair_bar);
+      ok = mbar_wait_warp(pair_bar, pair_uses & 1u, abort_flag, status);
+      ++pair_uses;
+      if (!ok) break;
+      const float lsum = l[qt] + *x_other;
+      mbar_arrive(pair_bar);                     // second rendezvous: the partner has read before x_mine is reused
+      ok = mbar_wait_warp(pair_bar, pair_uses & 1u, abort_flag, status);
+      ++pair_uses;
+      if (!ok) break;
+      const float inv = 1.f / lsum;
+      const int qi = q_first + qt * 128 + row;
+      __nv_bfloat16 *orow = const_cast<__nv_bfloat16 *>(row_ptr<__nv_bfloat16>(prm.O, b, h, qi < n_k ? qi : 0)) + half * 64;
 #pragma unroll
-            for (int v4 = 0; v4 < 4; ++v4) {
-              uint4 w;
-              w.x = pack_bf16(o[8 * v4 + 0] * inv, o[8 * v4 + 1] * inv);
-              w.y = pack_bf16(o[8 * v4 + 2] * inv, o[8 * v4 + 3] * inv);
-              w.z = pack_bf16(o[8 * v4 + 4] * inv, o[8 * v4 + 5] * inv);
-              w.w = pack_bf16(o[8 * v4 + 6] * inv, o[8 * v4 + 7] * inv);
-              reinterpret_cast<uint4 *>(orow + cc * 32)[v4] = w;
-            }
+      for (int cc = 0; cc < 2; ++cc) {
+        float o[32];
+        tc_ld32(lane_addr + kColO + qt * 128 + half * 64 + cc * 32, o);
+        tc_wait_ld();
+        if (qi < n_k) {
+#pragma unroll
+          for (int v4 = 0; v4 < 4; ++v4) {
+            uint4 w;
+            w.x = pack_bf16(o[8 * v4 + 0] * inv, o[8 * v4 + 1] * inv);
+            w.y = pack_bf16(o[8 * v4 + 2] * inv, o[8 * v4 + 3] * inv);
+            w.z = pack_bf16(o[8 * v4 + 4] * inv, o[8 * v4 + 5] * inv);
+            w.w = pack_bf16(o[8 * v4 + 6] * inv, o[8 * v4 + 7] * inv);
+            reinterpret_cast<uint4 *>(orow + cc * 32)[v4] = w;
           }
         }
-        if (prm.lse != nullptr && qi < n_k)
-          prm.lse[(size_t)slice * n_k + qi] = (m_used + log2f(l)) * 0.6931471805599453f;
-        tc_fence_before();
       }
+      if (prm.lse != nullptr && half == 0 && qi < n_k)
+        prm.lse[(size_t)slice * n_k + qi] = (m_used[qt] + log2f(lsum)) * 0.6931471805599453f;
     }
+    tc_fence_before();
   }
   __syncthreads();
   if (warp == 1) {
