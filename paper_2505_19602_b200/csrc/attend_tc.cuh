@@ -150,6 +150,44 @@ __device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint
       "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// Eight back-to-back MMAs of one 128 x 128 x 128 product, issued by the elected lane of a converged
+// warp; the descriptors' start addresses advance by constant steps.  SS: both operands in shared
+// memory (K-major tiles: steps of 32 B inside a 64-column half, then the next half).
+__device__ __forceinline__ void tc_mma_ss_x8(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc) {
+  asm volatile(
+      "{\n\t.reg .pred e, pf, pt;\n\t.reg .b64 da, db;\n\t.reg .b32 al, bl;\n\t"
+      "elect.sync _|e, 0xffffffff;\n\tsetp.ne.b32 pf, 0, 0;\n\tsetp.eq.b32 pt, 0, 0;\n\t"
+      "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t@e tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, pf;\n\t"
+      "add.u32 al, %1, 2;\n\tadd.u32 bl, %2, 2;\n\tmov.b64 da, {al, %3};\n\tmov.b64 db, {bl, %3};\n\t@e tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, pt;\n\t"
+      "add.u32 al, %1, 4;\n\tadd.u32 bl, %2, 4;\n\tmov.b64 da, {al, %3};\n\tmov.b64 db, {bl, %3};\n\t@e tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, pt;\n\t"
+      "add.u32 al, %1, 6;\n\tadd.u32 bl, %2, 6;\n\tmov.b64 da, {al, %3};\n\tmov.b64 db, {bl, %3};\n\t@e tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, pt;\n\t"
+      "add.u32 al, %1, 1024;\n\tadd.u32 bl, %2, 1024;\n\tmov.b64 da, {al, %3};\n\tmov.b64 db, {bl, %3};\n\t@e tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, pt;\n\t"
+      "add.u32 al, %1, 1026;\n\tadd.u32 bl, %2, 1026;\n\tmov.b64 da, {al, %3};\n\tmov.b64 db, {bl, %3};\n\t@e tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, pt;\n\t"
+      "add.u32 al, %1, 1028;\n\tadd.u32 bl, %2, 1028;\n\tmov.b64 da, {al, %3};\n\tmov.b64 db, {bl, %3};\n\t@e tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, pt;\n\t"
+      "add.u32 al, %1, 1030;\n\tadd.u32 bl, %2, 1030;\n\tmov.b64 da, {al, %3};\n\tmov.b64 db, {bl, %3};\n\t@e tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, pt;\n\t"
+      "}" ::"r"(d_tmem),
+      "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc)
+      : "memory");
+}
+// TS: A = P in TMEM (8 columns per step inside a half of the S buffer, the second half 64 columns
+// further), B = V in shared memory as the MN-major operand (16 keys = 2048 B per step).
+__device__ __forceinline__ void tc_mma_ts_x8(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t hi, uint32_t idesc,
+                                             uint32_t accumulate_first) {
+  asm volatile(
+      "{\n\t.reg .pred e, pf, pt;\n\t.reg .b64 db;\n\t.reg .b32 at, bl;\n\t"
+      "elect.sync _|e, 0xffffffff;\n\tsetp.ne.b32 pf, %5, 0;\n\tsetp.eq.b32 pt, 0, 0;\n\t"
+      "mov.b64 db, {%2, %3};\n\t@e tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, pf;\n\t"
+      "add.u32 at, %1, 8;\n\tadd.u32 bl, %2, 128;\n\tmov.b64 db, {bl, %3};\n\t@e tcgen05.mma.cta_group::1.kind::f16 [%0], [at], db, %4, pt;\n\t"
+      "add.u32 at, %1, 16;\n\tadd.u32 bl, %2, 256;\n\tmov.b64 db, {bl, %3};\n\t@e tcgen05.mma.cta_group::1.kind::f16 [%0], [at], db, %4, pt;\n\t"
+      "add.u32 at, %1, 24;\n\tadd.u32 bl, %2, 384;\n\tmov.b64 db, {bl, %3};\n\t@e tcgen05.mma.cta_group::1.kind::f16 [%0], [at], db, %4, pt;\n\t"
+      "add.u32 at, %1, 64;\n\tadd.u32 bl, %2, 512;\n\tmov.b64 db, {bl, %3};\n\t@e tcgen05.mma.cta_group::1.kind::f16 [%0], [at], db, %4, pt;\n\t"
+      "add.u32 at, %1, 72;\n\tadd.u32 bl, %2, 640;\n\tmov.b64 db, {bl, %3};\n\t@e tcgen05.mma.cta_group::1.kind::f16 [%0], [at], db, %4, pt;\n\t"
+      "add.u32 at, %1, 80;\n\tadd.u32 bl, %2, 768;\n\tmov.b64 db, {bl, %3};\n\t@e tcgen05.mma.cta_group::1.kind::f16 [%0], [at], db, %4, pt;\n\t"
+      "add.u32 at, %1, 88;\n\tadd.u32 bl, %2, 896;\n\tmov.b64 db, {bl, %3};\n\t@e tcgen05.mma.cta_group::1.kind::f16 [%0], [at], db, %4, pt;\n\t"
+      "}" ::"r"(d_tmem),
+      "r"(a_tmem), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate_first)
+      : "memory");
+}
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -437,12 +475,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       auto issue_s = [&](int j, int qt, int buf) {
         const uint32_t a_lo = q_lo[qt], b_lo = desc_lo(base + kOffRing + ((2 * j) % kStages) * kTileBytes, 16);
         const uint32_t d = tmem + kColS + buf * 128;
-#pragma unroll
-        for (int kk = 0; kk < 8; ++kk) {
-          constexpr uint32_t dummy = 0;
-          const uint32_t off = (((kk >> 2) * kHalfBytes + (kk & 3) * 32) >> 4) + dummy;
-          if (leader) tc_mma_ss(d, a_lo + off, dhi, b_lo + off, dhi, idesc_qk, kk > 0 ? 1u : 0u);
-        }
+        tc_mma_ss_x8(d, a_lo, b_lo, dhi, idesc_qk);
         if (leader) tc_commit(bar(bSFull + buf));
         __syncwarp();
       };
@@ -455,9 +488,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         const uint32_t b_lo = desc_lo(base + kOffRing + vs * kTileBytes, kHalfBytes);
         const uint32_t d = tmem + kColO + qt * 128, a = tmem + kColS + buf * 128;
         const uint32_t acc0 = t > 0 ? 1u : 0u;
-#pragma unroll
-        for (int kk = 0; kk < 8; ++kk)
-          if (leader) tc_mma_ts(d, a + (kk >> 2) * 64 + (kk & 3) * 8, b_lo + kk * (2048 >> 4), dhi, idesc_pv, kk > 0 ? 1u : acc0);
+        tc_mma_ts_x8(d, a, b_lo, dhi, idesc_pv, acc0);
         if (leader) {
           tc_commit(bar(bPvDone + qt));
           if (release_v) tc_commit(bar(bEmpty + vs));
