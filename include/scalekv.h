@@ -105,9 +105,13 @@ scalekv_status scalekv_destroy(scalekv_ctx *ctx);
 
 /* Sec. 1 / Sec. 3.3: the current map joins the cache.  K and V are [B][H][n_k][d] views of the
  * n_k = h_k * w_k rows of scale `scale` (0-based; scales must arrive in ascending order, once per
- * layer).  Row i receives original position N_{k-1} + i.  The rows are copied; the caller may
- * reuse its buffers once stream_main has passed this point.  Runs on stream_main after waiting
- * for this layer's previous compress. */
+ * layer).  Row i receives original position N_{k-1} + i.  The rows are copied into the store.
+ * For bf16 x 128 the copy is done by the scalekv_attend that follows, which reads the map from K
+ * and V directly and writes its rows to the pages while it streams them (no second read, nothing
+ * on the critical path); any other next call for this layer (compress, layer_stats, export, the
+ * next append) copies first with a kernel of its own.  K and V must therefore stay unmodified
+ * until stream_main has passed the layer's next call.  For f32 x 64 the copy is enqueued here.
+ * Ordered on stream_main after this layer's previous compress. */
 scalekv_status scalekv_append(scalekv_ctx *ctx, int32_t layer, int32_t scale, scalekv_tensor K, scalekv_tensor V);
 
 /* Eq. 5: O[b][h][i] = sum_j softmax_j(scale * <Q[b][h][i], K_j>) V_j over all L entries of the

@@ -3,8 +3,9 @@
 // of one slice and streams the slice's K/V pages once for both.
 //
 // Roles inside a CTA of 384 threads (three warpgroups):
-//   warp 0 (one thread) : TMA producer.  The query tiles once; then per 128-key tile the K and V rows,
-//                         page by page through the slice's page table, into 128B-swizzled shared memory.
+//   warp 0 (one thread) : TMA producer.  The query tiles once; then per 128-key tile the K and V rows into
+//                         128B-swizzled shared memory: history tiles page by page through the slice's
+//                         page table, tiles of a not yet appended current map from the caller's tensors.
 //   warp 1 (one thread) : tcgen05.mma issuer; owns the TMEM allocation (512 columns: two S/P buffers
 //                         and two O accumulators).  With two query tiles the issue order per key tile
 //                         j is  S_A(j), PV_B(j-1), S_B(j), PV_A(j): while one tile's softmax runs, the
@@ -21,6 +22,10 @@
 //                         only when a half row's sum shows that an exponent left the lazy band (2^8) do
 //                         both recompute the row against a new reference and rescale O.  At the end the
 //                         same warps normalise and store O, 64 columns each.
+//   warps 2-3           : append.  When the current map has not been copied into the store yet, its K/V
+//                         tiles come from the caller's tensors, and the CTA whose turn it is writes each
+//                         tile's rows from shared memory to the slice's pages (and their original
+//                         positions), so the copy costs no extra read and stays off the critical path.
 // Every mbarrier wait is bounded; a wait that gives up raises the sticky device status, sets a
 // CTA-wide abort flag and all roles fall through to the common exit where TMEM is released.
 #pragma once
@@ -35,7 +40,7 @@
 namespace scalekv {
 namespace tc {
 
-constexpr int kThreads = 384;          // three warpgroups: {TMA, MMA, 2 idle warps}, softmax A, softmax B
+constexpr int kThreads = 384;                    // warps: TMA, MMA, 2 x append, 8 x softmax
 constexpr int kStages = 5;                       // one ring for the K and V tiles: K_0, V_0, K_1, V_1, ...
 constexpr uint32_t kTileBytes = 128 * 128 * 2;   // one 128 x 128 bf16 operand tile
 constexpr uint32_t kHalfBytes = kTileBytes / 2;  // 64 head-dim columns = one 128-byte swizzle span
@@ -373,11 +378,14 @@ struct Params {
   int n_k;
   float scale_log2e;   // softmax scale * log2(e)
   int box_rows;        // rows per K/V TMA box = min(page_tokens, 128)
+  int fused_append;    // 1: the current map's K/V rows are still in the caller's tensors; read them there and copy them in
+  int n_prev;          // original position of the current map's first token
 };
 
 __global__ void __launch_bounds__(kThreads, 1)
 attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-                 const __grid_constant__ CUtensorMap tmV, const Params prm) {
+                 const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmKc,
+                 const __grid_constant__ CUtensorMap tmVc, const Params prm) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t *base_ptr = smem_raw + (base - smem_u32(smem_raw));
@@ -393,8 +401,18 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   const int n_k = prm.n_k;
   const int q_first = blockIdx.x * 256;                  // first query row of tile A
   const bool single = q_first + 128 >= n_k;              // tile B would be empty
-  const int L = lv.hist_len[slice] + n_k;
-  const int T = (L + 127) >> 7;
+  const int hist = lv.hist_len[slice];
+  const int L = hist + n_k;
+  // key tiles: Th from the pages (all of them unless the current map still waits in the caller's
+  // tensors), then Tc of the current map; each source ends in a ragged tile
+  const bool fused = prm.fused_append != 0;
+  const int Th = ((fused ? hist : L) + 127) >> 7;
+  const int Tc = fused ? (n_k + 127) >> 7 : 0;
+  const int T = Th + Tc;
+  auto tile_valid = [&](int j) {   // number of real keys in tile j
+    const int rest = j < Th ? (fused ? hist : L) - j * 128 : n_k - (j - Th) * 128;
+    return rest < 128 ? rest : 128;
+  };
   int *status = lv.status;
   if (*reinterpret_cast<volatile int *>(status) != 0) return;   // an earlier CTA gave up: do not pile on
 
@@ -403,7 +421,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     mbar_init(bar(bQFull), 1);
     for (int s = 0; s < kStages; ++s) {
       mbar_init(bar(bFull + s), 1);
-      mbar_init(bar(bEmpty + s), 1);
+      mbar_init(bar(bEmpty + s), 3);      // the MMA warp's commit and the two append warps
     }
     for (int s = 0; s < 2; ++s) {
       mbar_init(bar(bSFull + s), 1);
@@ -437,7 +455,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         }
       }
       const int R = prm.box_rows;
-      const int last_page = (L - 1) >> lv.page_shift;
+      const int last_page = fused ? (hist > 0 ? (hist - 1) >> lv.page_shift : 0) : (L - 1) >> lv.page_shift;
       const int *pt = lv.page_table + (size_t)slice * lv.pages_per_slice;
       bool ok = true;
       // ring tile t = 2 j is K_j, t = 2 j + 1 is V_j
@@ -446,7 +464,15 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         ok = mbar_wait_warp(bar(bEmpty + st), ((t / kStages) & 1) ^ 1, abort_flag, status);
         if (!ok) break;
         const CUtensorMap *tm = (t & 1) ? &tmV : &tmK;
-        if (elect_one()) {
+        if (j >= Th) {
+          if (elect_one()) {
+            const CUtensorMap *tc = (t & 1) ? &tmVc : &tmKc;
+            const uint32_t dst = base + kOffRing + st * kTileBytes;
+            mbar_expect_tx(bar(bFull + st), kTileBytes);
+            tma_load_4d(dst, tc, 0, (j - Th) * 128, h, b, bar(bFull + st));
+            tma_load_4d(dst + kHalfBytes, tc, 64, (j - Th) * 128, h, b, bar(bFull + st));
+          }
+        } else if (elect_one()) {
           mbar_expect_tx(bar(bFull + st), kTileBytes);
           for (int r0 = 0; r0 < 128; r0 += R) {
             const int slot = j * 128 + r0;
@@ -521,6 +547,36 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         if (ok) issue_pv(T - 1, 0, (T - 1) & 1, ((T - 1) >> 1) & 1, true);
       }
     }
+  } else {
+    // ------------------------------------------------------------------ append (warps 2 and 3)
+    // Every ring tile is waited for and released, so that the empty barrier's phases stay in step;
+    // only current-map tiles whose turn falls on this CTA are copied: rows [0, valid) of the tile go
+    // to slots hist + 128 (j - Th) + r of the slice, un-swizzled, 16 bytes per thread and step.
+    const int u = (warp - 2) * 32 + lane;
+    const int chunk = u & 15, rsub = u >> 4;
+    const uint32_t src_off = (uint32_t)(chunk >> 3) * kHalfBytes;
+    bool ok = true;
+    for (int t = 0; t < 2 * T && ok; ++t) {
+      const int st = t % kStages, j = t >> 1;
+      ok = mbar_wait_warp(bar(bFull + st), (t / kStages) & 1, abort_flag, status);
+      if (!ok) break;
+      if (j >= Th && (j - Th) % (int)gridDim.x == (int)blockIdx.x) {
+        const int first = (j - Th) * 128;
+        const int nvalid = tile_valid(j);
+        char *pool = (t & 1) ? lv.v_pool : lv.k_pool;
+        const uint32_t tile = base + kOffRing + st * kTileBytes + src_off;
+        for (int r = rsub; r < nvalid; r += 4) {
+          uint4 val;
+          const uint32_t addr = tile + r * 128 + (((chunk & 7) ^ (r & 7)) << 4);
+          asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(val.x), "=r"(val.y), "=r"(val.z), "=r"(val.w) : "r"(addr));
+          const size_t row = slot_row(lv, slice, hist + first + r);
+          reinterpret_cast<uint4 *>(pool + row * 256)[chunk] = val;
+          if ((t & 1) == 0 && chunk == 0) lv.pos_pool[row] = prm.n_prev + first + r;
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(bEmpty + st));
+    }
   }
   } else {
     // ------------------------------------------------------------------ softmax + epilogue
@@ -549,7 +605,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         if (!ok) break;
         tc_fence_after();
         const uint32_t s_addr = lane_addr + kColS + buf * 128 + half * 64;
-        const int valid = L - j * 128 - half * 64;     // < 64 only in the last tile; may be <= 0
+        const int valid = tile_valid(j) - half * 64;   // < 64 only in a ragged tile; may be <= 0
         float v[2][32];
         tc_ld32(s_addr, v[0]);
         // one sweep: x = s * c - m, p = exp2(x), partial row sum; the bf16 pairs of p stay in registers
@@ -720,24 +776,41 @@ struct AttendTc {
   }
   bool enabled() const { return on; }
 
-  bool launch(const LayerView &lv, const TensorView &Q, const TensorView &O, float *lse, int n_k, int /*L_host*/, float scale,
-              cudaStream_t stream, std::string &err) {
-    CUtensorMap tmQ;
-    const int B = lv.n_slices / lv.n_heads;
-    const cuuint64_t dims[4] = {128, (cuuint64_t)n_k, (cuuint64_t)lv.n_heads, (cuuint64_t)B};
-    const cuuint64_t strides[3] = {(cuuint64_t)Q.st * 2, (cuuint64_t)Q.sh * 2, (cuuint64_t)Q.sb * 2};
+  // [B][H][n_k][128] bf16 view -> 4-D tensor map with boxes of 128 rows x 64 columns
+  bool map_rows(CUtensorMap *tm, const TensorView &X, int n_k, int n_heads, int B, const char *what, std::string &err) {
+    const cuuint64_t dims[4] = {128, (cuuint64_t)n_k, (cuuint64_t)n_heads, (cuuint64_t)B};
+    const cuuint64_t strides[3] = {(cuuint64_t)X.st * 2, (cuuint64_t)X.sh * 2, (cuuint64_t)X.sb * 2};
     const cuuint32_t box[4] = {64, 128, 1, 1};
     const cuuint32_t estr[4] = {1, 1, 1, 1};
-    CUresult r = encode(&tmQ, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<char *>(Q.ptr), dims, strides, box, estr,
+    CUresult r = encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<char *>(X.ptr), dims, strides, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) { err = "cuTensorMapEncodeTiled(Q) failed with code " + std::to_string((int)r); return false; }
+    if (r != CUDA_SUCCESS) { err = std::string("cuTensorMapEncodeTiled(") + what + ") failed with code " + std::to_string((int)r); return false; }
+    return true;
+  }
+
+  // Kc / Vc: the current map's K and V when they have not been copied into the store yet (the kernel
+  // reads them there and copies them in), else nullptr.
+  bool launch(const LayerView &lv, const TensorView &Q, const TensorView &O, float *lse, int n_k, const TensorView *Kc,
+              const TensorView *Vc, int n_prev, float scale, cudaStream_t stream, std::string &err) {
+    CUtensorMap tmQ, tmKc, tmVc;
+    const int B = lv.n_slices / lv.n_heads;
+    if (!map_rows(&tmQ, Q, n_k, lv.n_heads, B, "Q", err)) return false;
+    const bool fused = Kc != nullptr && Vc != nullptr;
+    if (fused) {
+      if (!map_rows(&tmKc, *Kc, n_k, lv.n_heads, B, "K", err) || !map_rows(&tmVc, *Vc, n_k, lv.n_heads, B, "V", err)) return false;
+    } else {
+      tmKc = tmQ;
+      tmVc = tmQ;
+    }
     tc::Params prm;
     prm.lv = lv; prm.O = O; prm.lse = lse; prm.n_k = n_k;
     prm.scale_log2e = scale * 1.4426950408889634f;
     prm.box_rows = box_rows;
+    prm.fused_append = fused ? 1 : 0;
+    prm.n_prev = n_prev;
     dim3 grid((n_k + 255) / 256, lv.n_slices);
-    tc::attend_tc_kernel<<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(tmQ, tmK, tmV, prm);
+    tc::attend_tc_kernel<<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(tmQ, tmK, tmV, tmKc, tmVc, prm);
     return true;
   }
 };

@@ -144,6 +144,8 @@ struct scalekv_ctx {
   std::vector<int> hist;           // entries before the current map (uniform over slices)
   std::vector<int> pending;        // n_k of an appended, not yet committed current map (0 = none)
   std::vector<int> attended;       // attend ran for the pending map
+  std::vector<char> in_store;      // the pending map's rows have been copied into the pages
+  std::vector<scalekv_tensor> pend_k, pend_v;   // the caller's tensors of a pending map that is not in the store yet
   std::vector<cudaEvent_t> ev_attend, ev_compress;
   std::vector<char> ev_compress_live;
   int64_t launches = 0;
@@ -239,9 +241,27 @@ scalekv_status check_launch(scalekv_ctx *ctx, const char *what) {
   return SCALEKV_OK;
 }
 
+// Copies a pending current map that still lives in the caller's tensors into the pages (stream_main).
+// The tensor-core attend does this itself while it streams the map; this kernel serves every other
+// order of calls (compress, statistics or export without a preceding attend).
+scalekv_status materialize(scalekv_ctx *ctx, int l) {
+  if (ctx->pending[l] == 0 || ctx->in_store[l]) return SCALEKV_OK;
+  const Plan &p = ctx->plan;
+  const int k = ctx->next_scale[l] - 1;
+  const int nk = ctx->pending[l];
+  {
+    Scope sc(ctx, ctx->s_main, kAppend);
+    dim3 grid((nk + 63) / 64, p.n_slices);
+    append_kernel<<<grid, 256, 0, ctx->s_main>>>(layer_view(ctx, l), tview(ctx->pend_k[l]), tview(ctx->pend_v[l]), nk, p.N[k], p.esize);
+  }
+  ctx->in_store[l] = 1;
+  return check_launch(ctx, "append");
+}
+
 scalekv_status commit_pending(scalekv_ctx *ctx, int l, cudaStream_t s) {
   if (ctx->pending[l] == 0) return SCALEKV_OK;
   const Plan &p = ctx->plan;
+  if (!ctx->in_store[l]) return fail(ctx, SCALEKV_ERR_BAD_STATE, "layer %d: pending map is not in the store", l);
   const int L = ctx->hist[l] + ctx->pending[l];
   if (L > p.layers[l].persist_pages * p.P && p.layers[l].persist_pages < p.layers[l].total_pages)
     return fail(ctx, SCALEKV_ERR_CAPACITY, "layer %d: %d entries kept without compress exceed the persistent capacity %d",
@@ -337,6 +357,8 @@ scalekv_status scalekv_init(const scalekv_config *cfg, scalekv_ctx **out) {
   ctx->hist.assign(p.n_layers, 0);
   ctx->pending.assign(p.n_layers, 0);
   ctx->attended.assign(p.n_layers, 0);
+  ctx->in_store.assign(p.n_layers, 1);
+  ctx->pend_k.resize(p.n_layers); ctx->pend_v.resize(p.n_layers);
   ctx->ev_attend.resize(p.n_layers); ctx->ev_compress.resize(p.n_layers);
   ctx->ev_compress_live.assign(p.n_layers, 0);
   for (int l = 0; l < p.n_layers; ++l) {
@@ -381,6 +403,7 @@ scalekv_status scalekv_reset(scalekv_ctx *ctx) {
   std::fill(ctx->hist.begin(), ctx->hist.end(), 0);
   std::fill(ctx->pending.begin(), ctx->pending.end(), 0);
   std::fill(ctx->attended.begin(), ctx->attended.end(), 0);
+  std::fill(ctx->in_store.begin(), ctx->in_store.end(), 1);
   std::fill(ctx->ev_compress_live.begin(), ctx->ev_compress_live.end(), 0);
   return SCALEKV_OK;
 }
@@ -417,15 +440,23 @@ scalekv_status scalekv_append(scalekv_ctx *ctx, int32_t layer, int32_t scale, sc
         if ((o & 1) == (layer & 1)) { if (ctx->ev_compress_live[o]) CU(cudaStreamWaitEvent(ctx->s_main, ctx->ev_compress[o], 0)); break; }
     }
   }
-  scalekv_status st = commit_pending(ctx, layer, ctx->s_main);
+  scalekv_status st = materialize(ctx, layer);
+  if (st != SCALEKV_OK) return st;
+  st = commit_pending(ctx, layer, ctx->s_main);
   if (st != SCALEKV_OK) return st;
   const int nk = p.n[scale];
   if (ctx->hist[layer] + nk > p.layers[layer].total_pages * p.P)
     return fail(ctx, SCALEKV_ERR_CAPACITY, "layer %d: %d + %d entries exceed the planned capacity", layer, ctx->hist[layer], nk);
-  {
+  if (ctx->tc.enabled()) {
+    // the tensor-core attend reads the map from K and V and copies it into the pages as it goes
+    ctx->pend_k[layer] = K;
+    ctx->pend_v[layer] = V;
+    ctx->in_store[layer] = 0;
+  } else {
     Scope sc(ctx, ctx->s_main, kAppend);
     dim3 grid((nk + 63) / 64, p.n_slices);
     append_kernel<<<grid, 256, 0, ctx->s_main>>>(layer_view(ctx, layer), tview(K), tview(V), nk, p.N[scale], p.esize);
+    ctx->in_store[layer] = 1;
   }
   ctx->pending[layer] = nk;
   ctx->attended[layer] = 0;
@@ -441,12 +472,21 @@ scalekv_status scalekv_attend(scalekv_ctx *ctx, int32_t layer, scalekv_tensor Q,
   if (!tensor_ok(Q, p.esize) || !tensor_ok(O, p.esize)) return fail(ctx, SCALEKV_ERR_INVALID_ARG, "Q/O null or rows not 16-byte aligned");
   const int nk = ctx->pending[layer];
   LayerView lv = layer_view(ctx, layer);
+  if (!ctx->tc.enabled()) {
+    scalekv_status st = materialize(ctx, layer);
+    if (st != SCALEKV_OK) return st;
+  }
   {
     Scope sc(ctx, ctx->s_main, kAttend);
     if (ctx->tc.enabled()) {
       std::string e;
-      if (!ctx->tc.launch(lv, tview(Q), tview(O), lse, nk, ctx->hist[layer] + nk, ctx->scale, ctx->s_main, e))
+      const bool fused = !ctx->in_store[layer];
+      TensorView kc, vc;
+      if (fused) { kc = tview(ctx->pend_k[layer]); vc = tview(ctx->pend_v[layer]); }
+      if (!ctx->tc.launch(lv, tview(Q), tview(O), lse, nk, fused ? &kc : nullptr, fused ? &vc : nullptr,
+                          p.N[ctx->next_scale[layer] - 1], ctx->scale, ctx->s_main, e))
         return fail(ctx, SCALEKV_ERR_CUDA, "attend launch: %s", e.c_str());
+      ctx->in_store[layer] = 1;
     } else {
       dim3 grid((nk + 63) / 64, p.n_slices);
       if (ctx->dtype == SCALEKV_BF16)
@@ -478,8 +518,11 @@ scalekv_status scalekv_compress(scalekv_ctx *ctx, int32_t layer, scalekv_tensor 
   const int budget = p.budgets[(size_t)layer * p.K + k];
   const bool evict = budget != SCALEKV_KEEP_ALL && budget < cand;
   cudaStream_t s = ctx->s_side;
+  const bool copy_now = !ctx->in_store[layer];
+  st = materialize(ctx, layer);
+  if (st != SCALEKV_OK) return st;
   if (s != ctx->s_main) {
-    if (!ctx->attended[layer]) CU(cudaEventRecord(ctx->ev_attend[layer], ctx->s_main));
+    if (!ctx->attended[layer] || copy_now) CU(cudaEventRecord(ctx->ev_attend[layer], ctx->s_main));
     CU(cudaStreamWaitEvent(s, ctx->ev_attend[layer], 0));
   }
   if (!evict) {
@@ -569,6 +612,8 @@ scalekv_status scalekv_layer_stats(scalekv_ctx *ctx, int32_t layer, scalekv_tens
   if (ctx->pending[layer] == 0) return fail(ctx, SCALEKV_ERR_BAD_STATE, "layer %d: layer_stats needs a preceding append", layer);
   if (topk_prime < 0 || topk_prime > 64 || query_stride < 1) return fail(ctx, SCALEKV_ERR_INVALID_ARG, "topk_prime in [0,64], stride >= 1");
   if (!tensor_ok(Q, p.esize)) return fail(ctx, SCALEKV_ERR_INVALID_ARG, "Q null or rows not 16-byte aligned");
+  scalekv_status st0 = materialize(ctx, layer);
+  if (st0 != SCALEKV_OK) return st0;
   const int nk = ctx->pending[layer];
   const int k = ctx->next_scale[layer] - 1;
   const int L = ctx->hist[layer] + nk;
@@ -699,7 +744,9 @@ scalekv_status scalekv_export_slice(scalekv_ctx *ctx, int32_t layer, int32_t b, 
   const Plan &p = ctx->plan;
   if (layer < 0 || layer >= p.n_layers || b < 0 || b >= p.B || h < 0 || h >= p.H)
     return fail(ctx, SCALEKV_ERR_INVALID_ARG, "slice index out of range");
-  scalekv_status st = scalekv_sync(ctx);
+  scalekv_status st = materialize(ctx, layer);
+  if (st != SCALEKV_OK) return st;
+  st = scalekv_sync(ctx);
   if (st != SCALEKV_OK) return st;
   const int slice = b * p.H + h;
   int hist = 0;
