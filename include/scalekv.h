@@ -72,6 +72,11 @@ typedef struct {
   void *stream_main;             /* cudaStream_t: append and attend run here                        */
   void *stream_side;             /* cudaStream_t: compress runs here (may equal stream_main)        */
   int32_t device;                /* CUDA device ordinal that owns pool, workspace and streams       */
+  int32_t window_patches;        /* N of Sec. 3.3 (e.g. 16), or 0.  When > 0, scalekv_attend (bf16 x 128)  */
+                                 /* also records the logits of the N-patch centroid rows of the current */
+                                 /* map (scalekv_window_centroids) while it computes them anyway, and a */
+                                 /* scalekv_compress called with exactly that window scores the cache   */
+                                 /* from them instead of reading K again.  Any other window still works.*/
 } scalekv_config;
 
 /* A [batch][n_heads][tokens][head_dim] tensor view: device pointer + ELEMENT strides; the

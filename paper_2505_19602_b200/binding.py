@@ -39,7 +39,7 @@ class scalekv_config(C.Structure):
         ("max_window", C.c_int32), ("softmax_scale", C.c_float), ("page_tokens", C.c_int32),
         ("pool", C.c_void_p), ("pool_bytes", C.c_size_t),
         ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
-        ("stream_main", C.c_void_p), ("stream_side", C.c_void_p), ("device", C.c_int32),
+        ("stream_main", C.c_void_p), ("stream_side", C.c_void_p), ("device", C.c_int32), ("window_patches", C.c_int32),
     ]
 
 
@@ -192,7 +192,7 @@ class ScaleKV:
     """Owns the device pool / workspace (torch tensors) and one library context."""
 
     def __init__(self, n_layers, batch, n_heads, head_dim, dtype, sides_h, sides_w, budgets, max_window=16,
-                 softmax_scale=0.0, page_tokens=0, device=0, side_stream=True):
+                 softmax_scale=0.0, page_tokens=0, device=0, side_stream=True, window_patches=16):
         if not torch.cuda.is_available():
             raise RuntimeError("ScaleKV needs a CUDA device (sm_100a); there is no CPU path")
         self.lib = load_library()
@@ -211,6 +211,7 @@ class ScaleKV:
         cfg.dtype, cfg.n_scales = self.dtype, self.n_scales
         cfg.scale_h, cfg.scale_w, cfg.budgets = self._h, self._w, self._b
         cfg.max_window, cfg.softmax_scale, cfg.page_tokens, cfg.device = max_window, softmax_scale, page_tokens, device
+        cfg.window_patches = window_patches if window_patches <= max_window else 0
         pb, wb = C.c_size_t(0), C.c_size_t(0)
         st = self.lib.scalekv_query_sizes(C.byref(cfg), C.byref(pb), C.byref(wb))
         if st:

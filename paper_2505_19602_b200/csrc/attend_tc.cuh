@@ -51,7 +51,7 @@ constexpr uint32_t kOffX = kOffBar + 256;           // exchange area of the soft
 constexpr uint32_t kSmemBytes = kOffX + 1280 + 1024;   // + alignment slack
 // barrier slots (8 bytes each): one full/empty pair per ring stage, one S/P/PV barrier per S buffer or query tile
 enum { bQFull = 0, bFull = 1, bEmpty = bFull + kStages, bSFull = bEmpty + kStages, bPFull = bSFull + 2, bPvDone = bPFull + 2,
-       bPair = bPvDone + 2, bCount = bPair + 4 };
+       bPair = bPvDone + 2, bFinal = bPair + 4, bCount = bFinal + 2 };
 static_assert(bCount * 8 <= 192, "barriers overlap the TMEM slot");
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColS = 0, kColO = 256;       // S/P buffers at 0 and 128, O accumulators at 256 and 384
@@ -380,6 +380,12 @@ struct Params {
   int box_rows;        // rows per K/V TMA box = min(page_tokens, 128)
   int fused_append;    // 1: the current map's K/V rows are still in the caller's tensors; read them there and copy them in
   int n_prev;          // original position of the current map's first token
+  // observation window (Sec. 3.3): when win_logits is not null, the base-2 logits scale * log2(e) * <q, k>
+  // of the w window rows against every cache entry are recorded in win_logits[slice][rank][slot]
+  float *win_logits;
+  int ld_l;            // leading dimension of a logit row
+  int w;
+  int win_pos[kMaxWindow];   // ascending raster indices of the window rows inside the current map
 };
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -429,6 +435,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       mbar_init(bar(bPvDone + s), 1);
     }
     for (int s = 0; s < 4; ++s) mbar_init(bar(bPair + s), 64);
+    for (int s = 0; s < 2; ++s) mbar_init(bar(bFinal + s), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -534,7 +541,9 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           if (leader) tc_commit(bar(bEmpty + (2 * j) % kStages));
           ok = issue_pv(j, 0, 0, j & 1, false);
         }
-        if (ok) issue_pv(T - 1, 1, 1, (T - 1) & 1, true);
+        if (ok) ok = issue_pv(T - 1, 1, 1, (T - 1) & 1, true);
+        // one-shot barriers for the epilogue: everything issued so far has landed
+        if (ok && leader) { tc_commit(bar(bFinal + 0)); tc_commit(bar(bFinal + 1)); }
       } else {
         for (int j = 0; j < T && ok; ++j) {
           ok = mbar_wait_warp(bar(bFull + (2 * j) % kStages), ((2 * j) / kStages) & 1, abort_flag, status);
@@ -544,7 +553,8 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           if (leader) tc_commit(bar(bEmpty + (2 * j) % kStages));
           if (j > 0) ok = issue_pv(j - 1, 0, (j - 1) & 1, ((j - 1) >> 1) & 1, true);
         }
-        if (ok) issue_pv(T - 1, 0, (T - 1) & 1, ((T - 1) >> 1) & 1, true);
+        if (ok) ok = issue_pv(T - 1, 0, (T - 1) & 1, ((T - 1) >> 1) & 1, true);
+        if (ok && leader) tc_commit(bar(bFinal + 0));
       }
     }
   } else {
@@ -594,6 +604,18 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     uint32_t pair_uses = 0;                      // rendezvous so far of this quarter's two warps (same in both)
     const int ntile = single ? 1 : 2;
     float m_used[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f};
+    // window rows of this thread (rank in the window, or -1) and whether its warp has any
+    int wrank[2] = {-1, -1};
+    bool wwarp[2] = {false, false};
+    if (prm.win_logits != nullptr) {
+#pragma unroll
+      for (int qt = 0; qt < 2; ++qt) {
+        const int qi = q_first + qt * 128 + row;
+        for (int e = 0; e < prm.w; ++e)
+          if (prm.win_pos[e] == qi) wrank[qt] = e;
+        wwarp[qt] = __any_sync(0xffffffffu, wrank[qt] >= 0);
+      }
+    }
     bool ok = true;
     for (int j = 0; j < T && ok; ++j) {
 #pragma unroll
@@ -620,6 +642,17 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           tc_wait_ld();
           if (cc < 1) tc_ld32(s_addr + (cc + 1) * 32, v[(cc + 1) & 1]);
           float *x = v[cc & 1];
+          if (wwarp[qt]) {
+            if (wrank[qt] >= 0) {
+              // slot of this chunk's first column: history tiles start at 128 j, current-map tiles behind the history
+              const int slot0 = (j < Th ? j * 128 : hist + (j - Th) * 128) + half * 64 + cc * 32;
+              float *dst = prm.win_logits + ((size_t)slice * prm.w + wrank[qt]) * prm.ld_l + slot0;
+#pragma unroll
+              for (int i = 0; i < 32; ++i)
+                if (cc * 32 + i < valid) dst[i] = x[i] * c;
+            }
+            __syncwarp();   // the tcgen05 instructions that follow want the warp converged
+          }
           if (valid < 64) {
 #pragma unroll
             for (int i = 0; i < 32; ++i)
@@ -686,7 +719,9 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 #pragma unroll
     for (int qt = 0; qt < 2; ++qt) {
       if (qt >= ntile || !ok) break;
-      ok = mbar_wait_warp(bar(bPvDone + qt), (T - 1) & 1, abort_flag, status);
+      // a barrier that completes exactly once, after the last PV product: the per-tile PV barrier will
+      // not do, a parity wait cannot tell phases two apart and this warp may be that far behind it
+      ok = mbar_wait_warp(bar(bFinal + qt), 0, abort_flag, status);
       if (!ok) break;
       tc_fence_after();
       // the row sum is the sum of the two halves' partial sums
@@ -791,8 +826,10 @@ struct AttendTc {
 
   // Kc / Vc: the current map's K and V when they have not been copied into the store yet (the kernel
   // reads them there and copies them in), else nullptr.
+  // win_logits / win_pos / w: where to record the window rows' logits (nullptr: do not).
   bool launch(const LayerView &lv, const TensorView &Q, const TensorView &O, float *lse, int n_k, const TensorView *Kc,
-              const TensorView *Vc, int n_prev, float scale, cudaStream_t stream, std::string &err) {
+              const TensorView *Vc, int n_prev, float scale, float *win_logits, int ld_l, const int *win_pos, int w,
+              cudaStream_t stream, std::string &err) {
     CUtensorMap tmQ, tmKc, tmVc;
     const int B = lv.n_slices / lv.n_heads;
     if (!map_rows(&tmQ, Q, n_k, lv.n_heads, B, "Q", err)) return false;
@@ -809,6 +846,10 @@ struct AttendTc {
     prm.box_rows = box_rows;
     prm.fused_append = fused ? 1 : 0;
     prm.n_prev = n_prev;
+    prm.win_logits = win_logits;
+    prm.ld_l = ld_l;
+    prm.w = win_logits ? w : 0;
+    for (int e = 0; e < kMaxWindow; ++e) prm.win_pos[e] = (win_logits && e < w) ? win_pos[e] : -1;
     dim3 grid((n_k + 255) / 256, lv.n_slices);
     tc::attend_tc_kernel<<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(tmQ, tmK, tmV, tmKc, tmVc, prm);
     return true;

@@ -220,7 +220,8 @@ __global__ void __launch_bounds__(256) attend_simt_kernel(LayerView lv, TensorVi
 }
 
 // ------------------------------------------------------------------------------------------
-// score, step 1: scaled logits of the window rows against a tile of 64 cache entries (Eq. 5).
+// score, step 1 (only when attend did not record them): logits of the window rows against a tile of
+// 64 cache entries (Eq. 5), in base-2 units: y = scale * log2(e) * <q, k>.
 // grid (ceil(L_max / 64), n_slices), 256 threads.  logits is [n_slices][w][ld_l] fp32.
 // ------------------------------------------------------------------------------------------
 template <typename T, int D>
@@ -284,7 +285,7 @@ __global__ void __launch_bounds__(256) score_logits_kernel(LayerView lv, TensorV
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       const int col = j0 + tx + 16 * j;
-      if (col < L) logits[((size_t)slice * wa.w + r) * ld_l + col] = s[i][j] * scale;
+      if (col < L) logits[((size_t)slice * wa.w + r) * ld_l + col] = s[i][j] * (scale * 1.4426950408889634f);
     }
   }
 }
@@ -310,37 +311,17 @@ __device__ __forceinline__ float block_reduce_sum(float v, float *red) {
   return r;
 }
 
-// score, step 2: row-wise softmax normalisers, then s_i = (1/w) sum_j exp(z_ji - m_j) / Z_j
-// (Eq. 5 and the aggregation paragraph).  grid (n_slices), 512 threads.
-__global__ void __launch_bounds__(512) score_reduce_kernel(LayerView lv, WindowArg wa, const float *logits, int ld_l,
-                                                           float *scores, int ld_s) {
-  __shared__ float red[16];
-  __shared__ float m_row[kMaxWindow], inv_row[kMaxWindow];
-  const int slice = blockIdx.x;
-  const int L = lv.hist_len[slice] + wa.n_k;
-  const float *z = logits + (size_t)slice * wa.w * ld_l;
-  for (int j = 0; j < wa.w; ++j) {
-    float mx = -INFINITY;
-    for (int i = threadIdx.x; i < L; i += blockDim.x) mx = fmaxf(mx, z[(size_t)j * ld_l + i]);
-    mx = block_reduce_max(mx, red);
-    float sum = 0.f;
-    for (int i = threadIdx.x; i < L; i += blockDim.x) sum += expf(z[(size_t)j * ld_l + i] - mx);
-    sum = block_reduce_sum(sum, red);
-    if (threadIdx.x == 0) { m_row[j] = mx; inv_row[j] = 1.f / (sum * (float)wa.w); }
-  }
-  __syncthreads();
-  for (int i = threadIdx.x; i < L; i += blockDim.x) {
-    float s = 0.f;
-    for (int j = 0; j < wa.w; ++j) s += expf(z[(size_t)j * ld_l + i] - m_row[j]) * inv_row[j];
-    scores[(size_t)slice * ld_s + i] = s;
-  }
-}
-
 // ------------------------------------------------------------------------------------------
-// select: per-slice top-k' of the non-window entries by score (Sec. 3.3), radix-select on the
-// float bit patterns (scores are >= 0, so the patterns order like the values), ties by lowest
-// slot = lowest original position.  Emits the ascending slot list of survivors (selected U
-// window) and its length.  grid (n_slices), 1024 threads.
+// score, step 2, aggregation and selection in one kernel, one CTA of 1024 threads per slice
+// (Sec. 3.3, Eq. 5 and the selection paragraph).  Input: base-2 logits y[w][L] of the window rows.
+//   1. per window row j: m_j = max_i y_ji and Z_j = sum_i 2^(y_ji - m_j)   (two sweeps, 16 rows at a time)
+//   2. s_i = (1/w) sum_j 2^(y_ji - m_j) / Z_j  -> scores (global, for inspection) and, as the bit
+//      pattern of the non-negative float, the radix key of entry i in shared memory; window entries
+//      get a sentinel and never take part in the selection
+//   3. radix select of the k'-th largest key, 8 bits per pass, warp-aggregated histogram updates
+//   4. ordered emit of the ascending slot list of survivors (selected U window); ties at the
+//      threshold go to the lowest slots = lowest original positions.  Deterministic.
+// Dynamic shared memory: 4 * ld_s bytes of keys.
 // ------------------------------------------------------------------------------------------
 constexpr uint32_t kWindowKey = 0xFFFFFFFFu;
 
@@ -370,23 +351,77 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int *warp_sums, int *
   return warp_sums[wid] + incl - v;
 }
 
-__global__ void __launch_bounds__(1024) select_kernel(LayerView lv, WindowArg wa, int budget, const float *scores,
-                                                      int ld_s, uint32_t *keys, int *keep_list, int *kept_count) {
+__global__ void __launch_bounds__(1024) score_select_kernel(LayerView lv, WindowArg wa, int budget, const float *logits,
+                                                            int ld_l, float *scores, int ld_s, int *keep_list,
+                                                            int *kept_count) {
+  extern __shared__ uint32_t key[];            // [L]
+  __shared__ float part[32][16];               // per-warp partial maxima / sums of 16 rows
+  __shared__ float m_row[kMaxWindow], inv_row[kMaxWindow];
   __shared__ int hist[256];
   __shared__ int warp_sums[33];
   __shared__ uint32_t sh_prefix;
   __shared__ int sh_remaining;
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const int slice = blockIdx.x;
   const int L = lv.hist_len[slice] + wa.n_k;
-  uint32_t *key = keys + (size_t)slice * ld_s;
+  const int w = wa.w;
+  const float *y = logits + (size_t)slice * w * ld_l;
   int *out = keep_list + (size_t)slice * ld_s;
 
-  // pass 0: keys; window entries get a sentinel and never take part in the selection
+  // 1. row maxima and normalisers, 16 rows per round
+  for (int g0 = 0; g0 < w; g0 += 16) {
+    const int nr = w - g0 < 16 ? w - g0 : 16;
+    float acc[16];
+#pragma unroll
+    for (int r = 0; r < 16; ++r) acc[r] = -INFINITY;
+    for (int i = tid; i < L; i += 1024) {
+#pragma unroll
+      for (int r = 0; r < 16; ++r)
+        if (r < nr) acc[r] = fmaxf(acc[r], y[(size_t)(g0 + r) * ld_l + i]);
+    }
+#pragma unroll
+    for (int r = 0; r < 16; ++r) {
+      float v = acc[r];
+      for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+      if (lane == 0) part[wid][r] = v;
+    }
+    __syncthreads();
+    if (tid < 16) {
+      float v = part[0][tid];
+      for (int k = 1; k < 32; ++k) v = fmaxf(v, part[k][tid]);
+      if (tid < nr) m_row[g0 + tid] = v;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int r = 0; r < 16; ++r) acc[r] = 0.f;
+    for (int i = tid; i < L; i += 1024) {
+#pragma unroll
+      for (int r = 0; r < 16; ++r)
+        if (r < nr) acc[r] += exp2f(y[(size_t)(g0 + r) * ld_l + i] - m_row[g0 + r]);
+    }
+#pragma unroll
+    for (int r = 0; r < 16; ++r) {
+      float v = acc[r];
+      for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+      if (lane == 0) part[wid][r] = v;
+    }
+    __syncthreads();
+    if (tid < 16) {
+      float v = 0.f;
+      for (int k = 0; k < 32; ++k) v += part[k][tid];     // fixed order: deterministic
+      if (tid < nr) inv_row[g0 + tid] = 1.f / (v * (float)w);
+    }
+    __syncthreads();
+  }
+
+  // 2. scores and keys
   int n_win_local = 0;
-  for (int i = threadIdx.x; i < L; i += blockDim.x) {
-    const int p = lv.pos_pool[slot_row(lv, slice, i)];
-    const bool win = is_window_pos(wa, p);
-    key[i] = win ? kWindowKey : (__float_as_uint(scores[(size_t)slice * ld_s + i]) & 0x7FFFFFFFu);
+  for (int i = tid; i < L; i += 1024) {
+    float sc = 0.f;
+    for (int j = 0; j < w; ++j) sc += exp2f(y[(size_t)j * ld_l + i] - m_row[j]) * inv_row[j];
+    scores[(size_t)slice * ld_s + i] = sc;
+    const bool win = is_window_pos(wa, lv.pos_pool[slot_row(lv, slice, i)]);
+    key[i] = win ? kWindowKey : (__float_as_uint(sc) & 0x7FFFFFFFu);
     n_win_local += win ? 1 : 0;
   }
   int n_win;
@@ -394,32 +429,51 @@ __global__ void __launch_bounds__(1024) select_kernel(LayerView lv, WindowArg wa
   const int cand = L - n_win;
   const int kprime = (budget < 0 || budget > cand) ? cand : budget;
 
-  // radix select of the kprime-th largest key, 8 bits per pass from the top
+  // 3. radix select of the kprime-th largest key
   uint32_t threshold = 0;
   int n_ties_taken = 0;       // how many entries equal to the threshold are kept
   if (kprime > 0 && kprime < cand) {
-    if (threadIdx.x == 0) { sh_prefix = 0; sh_remaining = kprime; }
+    if (tid == 0) { sh_prefix = 0; sh_remaining = kprime; }
     for (int pass = 0; pass < 4; ++pass) {
       const int shift = 24 - 8 * pass;
       const uint32_t mask_hi = pass == 0 ? 0u : (0xFFFFFFFFu << (shift + 8));
-      if (threadIdx.x < 256) hist[threadIdx.x] = 0;
+      if (tid < 256) hist[tid] = 0;
       __syncthreads();
       const uint32_t prefix = sh_prefix;
-      for (int i = threadIdx.x; i < L; i += blockDim.x) {
-        const uint32_t k = key[i];
-        if (k != kWindowKey && (k & mask_hi) == prefix) atomicAdd(&hist[(k >> shift) & 0xFF], 1);
+      for (int i0 = 0; i0 < L; i0 += 1024) {
+        const int i = i0 + tid;
+        const uint32_t k = i < L ? key[i] : kWindowKey;
+        const bool in = (k != kWindowKey) && ((k & mask_hi) == prefix);
+        const uint32_t digit = in ? ((k >> shift) & 0xFFu) : 256u;
+        // one shared-memory atomic per distinct digit in the warp
+        const uint32_t peers = __match_any_sync(0xffffffffu, digit);
+        if (in && lane == (__ffs(peers) - 1)) atomicAdd(&hist[digit], __popc(peers));
       }
       __syncthreads();
-      if (threadIdx.x == 0) {
-        int rem = sh_remaining;
-        int dsel = 0;
-        for (int dgt = 255; dgt >= 0; --dgt) {
-          const int c = hist[dgt];
-          if (c >= rem) { dsel = dgt; break; }
-          rem -= c;
+      if (tid < 32) {
+        // digits 255 .. 0 in descending order, 8 per lane; find where the running count reaches `rem`
+        int c[8], tot = 0;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) { c[e] = hist[255 - (lane * 8 + e)]; tot += c[e]; }
+        int incl = tot;
+        for (int o = 1; o < 32; o <<= 1) {
+          const int t = __shfl_up_sync(0xffffffffu, incl, o);
+          if (lane >= o) incl += t;
         }
-        sh_remaining = rem;
-        sh_prefix = prefix | ((uint32_t)dsel << shift);
+        const int rem = sh_remaining;
+        int before = incl - tot;
+        const bool here = before < rem && incl >= rem;
+        if (here) {
+          int dsel = 0, r = rem - before;
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            if (r > 0) {
+              if (c[e] >= r) { dsel = 255 - (lane * 8 + e); sh_remaining = r; r = 0; }
+              else r -= c[e];
+            }
+          }
+          sh_prefix = prefix | ((uint32_t)dsel << shift);
+        }
       }
       __syncthreads();
     }
@@ -429,10 +483,10 @@ __global__ void __launch_bounds__(1024) select_kernel(LayerView lv, WindowArg wa
   const bool keep_all = (kprime >= cand);
   const bool keep_none = (kprime == 0);
 
-  // ordered emit
+  // 4. ordered emit
   int base_out = 0, base_tie = 0;
-  for (int i0 = 0; i0 < L; i0 += blockDim.x) {
-    const int i = i0 + threadIdx.x;
+  for (int i0 = 0; i0 < L; i0 += 1024) {
+    const int i = i0 + tid;
     uint32_t k = 0;
     bool win = false, gt = false, tie = false;
     if (i < L) {
@@ -451,57 +505,62 @@ __global__ void __launch_bounds__(1024) select_kernel(LayerView lv, WindowArg wa
     base_tie += tie_total;
     base_out += keep_total;
   }
-  if (threadIdx.x == 0) kept_count[slice] = base_out;
+  if (tid == 0) kept_count[slice] = base_out;
 }
 
 // ------------------------------------------------------------------------------------------
-// compact: slot j <- old slot keep[j], in place, for K (blockIdx.y = 0, also pos) and V
-// (blockIdx.y = 1).  keep is ascending, so keep[j] >= j: within a chunk every source is read
-// before any destination is written, and the sources of later chunks lie beyond every earlier
-// destination.  grid (n_slices, 2), 256 threads, 16-byte pieces (Sec. 3.3, pruning).
+// compact: slot j <- old slot keep[j], in place (Sec. 3.3, pruning).  grid (n_slices, 2, 4):
+// blockIdx.y = 0 moves K (and, in column block 0, pos), 1 moves V; blockIdx.z picks a quarter of
+// the row's 16-byte pieces, so that a slice's move is spread over 8 CTAs that touch disjoint bytes.
+// keep is ascending, so keep[j] >= j: within a chunk every source is read before any destination
+// is written, and the sources of later chunks lie beyond every earlier destination.  256 threads,
+// chunks of 256 * 8 / ppq rows (ppq = pieces per row quarter), 8 pieces in flight per thread.
 // ------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) compact_kernel(LayerView lv, const int *keep_list, int ld_s, const int *kept_count) {
   const int slice = blockIdx.x;
   const int which = blockIdx.y;
+  const int quarter = blockIdx.z;
   char *pool = which == 0 ? lv.k_pool : lv.v_pool;
   const int *list = keep_list + (size_t)slice * ld_s;
   const int kept = kept_count[slice];
-  const int ppr = lv.row_bytes >> 4;
-  const int C = 1024 / ppr;        // rows per chunk (4 pieces per thread)
-  int lo = 0, hi = kept;           // first j with keep[j] != j (the untouched prefix is skipped)
+  const int ppr = lv.row_bytes >> 4;       // 16-byte pieces per row
+  const int ppq = ppr >> 2;                // pieces of this CTA's quarter (row_bytes is a multiple of 64)
+  const int C = 2048 / ppq;                // rows per chunk
+  int lo = 0, hi = kept;                   // first j with keep[j] != j (the untouched prefix is skipped)
   while (lo < hi) {
     const int mid = (lo + hi) >> 1;
-    if (list[mid] == mid) lo = mid + 1; else hi = mid;
+    if (__ldg(list + mid) == mid) lo = mid + 1; else hi = mid;
   }
+  const bool do_pos_cta = which == 0 && quarter == 0;
   for (int c0 = lo; c0 < kept; c0 += C) {
-    uint4 buf[4];
-    int pv = 0;
+    uint4 buf[8];
+    int pv[8];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
+    for (int u = 0; u < 8; ++u) {
       const int piece = threadIdx.x + u * 256;
-      const int r = piece / ppr, c = piece % ppr;
+      const int r = piece / ppq, c = quarter * ppq + piece % ppq;
       const int j = c0 + r;
-      if (r < C && j < kept) {
-        const size_t row = slot_row(lv, slice, list[j]);
+      if (j < kept) {
+        const size_t row = slot_row(lv, slice, __ldg(list + j));
         buf[u] = reinterpret_cast<const uint4 *>(pool + row * lv.row_bytes)[c];
+        if (do_pos_cta && piece % ppq == 0) pv[u] = lv.pos_pool[row];
       }
     }
-    const bool do_pos = (which == 0) && ((int)threadIdx.x < C) && (c0 + (int)threadIdx.x < kept);
-    if (do_pos) pv = lv.pos_pool[slot_row(lv, slice, list[c0 + threadIdx.x])];
     __syncthreads();
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
+    for (int u = 0; u < 8; ++u) {
       const int piece = threadIdx.x + u * 256;
-      const int r = piece / ppr, c = piece % ppr;
+      const int r = piece / ppq, c = quarter * ppq + piece % ppq;
       const int j = c0 + r;
-      if (r < C && j < kept) {
+      if (j < kept) {
         const size_t row = slot_row(lv, slice, j);
         reinterpret_cast<uint4 *>(pool + row * lv.row_bytes)[c] = buf[u];
+        if (do_pos_cta && piece % ppq == 0) lv.pos_pool[row] = pv[u];
       }
     }
-    if (do_pos) lv.pos_pool[slot_row(lv, slice, c0 + threadIdx.x)] = pv;
   }
-  if (which == 0 && threadIdx.x == 0) lv.hist_len[slice] = kept;
+  // no CTA of this kernel reads the length (the keep list's length is kept_count)
+  if (do_pos_cta && threadIdx.x == 0) lv.hist_len[slice] = kept;
 }
 
 // ------------------------------------------------------------------------------------------

@@ -37,6 +37,7 @@ struct Plan {
   int n_layers, B, H, d, esize, K, P, page_shift, n_slices, max_window;
   std::vector<int> n, N;            // tokens per scale, cumulative (N[0] = 0)
   std::vector<int> budgets;         // [layers][K]
+  std::vector<std::vector<int>> windows;   // per scale: rows whose logits attend records (empty: none)
   std::vector<LayerPlan> layers;
   int trans_pages_per_slice = 0;    // size of one transient set per slice
   int trans_first[2] = {0, 0};
@@ -45,10 +46,34 @@ struct Plan {
   int n_max = 0;
   // pool layout (byte offsets)
   size_t off_k, off_v, off_pos, off_pt, off_len, off_status, pool_bytes;
-  size_t pt_elems;
+  size_t pt_elems, logits_elems;
   // workspace layout
   size_t off_logits, off_scores, off_keys, off_keep, off_kept, off_acc, off_qw, ws_bytes;
 };
+
+// Raster indices of the observation window of an h x w map (see scalekv_window_centroids).
+std::vector<int> centroid_window(int h, int w, int n_patches) {
+  std::vector<int> out;
+  if ((long long)h * w <= n_patches) {
+    for (int i = 0; i < h * w; ++i) out.push_back(i);
+    return out;
+  }
+  int g = (int)std::floor(std::sqrt((double)n_patches));
+  while ((g + 1) * (g + 1) <= n_patches) ++g;
+  while (g * g > n_patches) --g;
+  for (int a = 0; a < g; ++a) {
+    const int r0 = (int)((long long)a * h / g), r1 = (int)((long long)(a + 1) * h / g);
+    if (r1 <= r0) continue;
+    for (int b = 0; b < g; ++b) {
+      const int c0 = (int)((long long)b * w / g), c1 = (int)((long long)(b + 1) * w / g);
+      if (c1 <= c0) continue;
+      out.push_back(((r0 + r1 - 1) / 2) * w + (c0 + c1 - 1) / 2);
+    }
+  }
+  std::sort(out.begin(), out.end());
+  out.erase(std::unique(out.begin(), out.end()), out.end());
+  return out;
+}
 
 scalekv_status make_plan(const scalekv_config *c, Plan &p, std::string &err) {
   if (!c || !c->scale_h || !c->scale_w || !c->budgets) { err = "null config field"; return SCALEKV_ERR_INVALID_ARG; }
@@ -75,6 +100,10 @@ scalekv_status make_plan(const scalekv_config *c, Plan &p, std::string &err) {
     p.n_max = std::max(p.n_max, p.n[k]);
   }
   p.budgets.assign(c->budgets, c->budgets + (size_t)p.n_layers * p.K);
+  if (c->window_patches < 0 || c->window_patches > c->max_window) { err = "window_patches must lie in [0, max_window]"; return SCALEKV_ERR_INVALID_ARG; }
+  p.windows.assign(p.K, std::vector<int>());
+  if (c->window_patches > 0)
+    for (int k = 0; k < p.K; ++k) p.windows[k] = centroid_window(c->scale_h[k], c->scale_w[k], c->window_patches);
   p.layers.resize(p.n_layers);
   int trans_max = 0, len_max = 0;
   size_t pt = 0;
@@ -118,7 +147,8 @@ scalekv_status make_plan(const scalekv_config *c, Plan &p, std::string &err) {
   p.off_status = o; o = align_up(o + 256, 1024);
   p.pool_bytes = o;
   o = 0;
-  p.off_logits = o; o = align_up(o + (size_t)p.n_slices * p.max_window * p.ld_s * 4, 1024);
+  p.logits_elems = (size_t)p.n_slices * p.max_window * p.ld_s;   // one buffer per layer parity
+  p.off_logits = o; o = align_up(o + 2 * p.logits_elems * 4, 1024);
   p.off_scores = o; o = align_up(o + (size_t)p.n_slices * p.ld_s * 4, 1024);
   p.off_keys = o; o = align_up(o + (size_t)p.n_slices * p.ld_s * 4, 1024);
   p.off_keep = o; o = align_up(o + (size_t)p.n_slices * p.ld_s * 4, 1024);
@@ -145,6 +175,7 @@ struct scalekv_ctx {
   std::vector<int> pending;        // n_k of an appended, not yet committed current map (0 = none)
   std::vector<int> attended;       // attend ran for the pending map
   std::vector<char> in_store;      // the pending map's rows have been copied into the pages
+  std::vector<int> logits_of;      // scale whose window logits attend recorded for this layer (-1: none)
   std::vector<scalekv_tensor> pend_k, pend_v;   // the caller's tensors of a pending map that is not in the store yet
   std::vector<cudaEvent_t> ev_attend, ev_compress;
   std::vector<char> ev_compress_live;
@@ -358,6 +389,7 @@ scalekv_status scalekv_init(const scalekv_config *cfg, scalekv_ctx **out) {
   ctx->pending.assign(p.n_layers, 0);
   ctx->attended.assign(p.n_layers, 0);
   ctx->in_store.assign(p.n_layers, 1);
+  ctx->logits_of.assign(p.n_layers, -1);
   ctx->pend_k.resize(p.n_layers); ctx->pend_v.resize(p.n_layers);
   ctx->ev_attend.resize(p.n_layers); ctx->ev_compress.resize(p.n_layers);
   ctx->ev_compress_live.assign(p.n_layers, 0);
@@ -374,6 +406,7 @@ scalekv_status scalekv_init(const scalekv_config *cfg, scalekv_ctx **out) {
     set_smem(score_logits_kernel<float, 64>, 2 * 64 * 68 * 4);
     set_smem(layer_stats_kernel<float, 64>, (size_t)(64 + p.ld_s) * 4);
   }
+  set_smem(score_select_kernel, (size_t)p.ld_s * 4);
   cudaGetLastError();
   std::string tc_err;
   if (!ctx->tc.init(cfg->dtype, p.d, ctx->pool + p.off_k, ctx->pool + p.off_v, p.n_pages, p.P, tc_err)) {
@@ -404,6 +437,7 @@ scalekv_status scalekv_reset(scalekv_ctx *ctx) {
   std::fill(ctx->pending.begin(), ctx->pending.end(), 0);
   std::fill(ctx->attended.begin(), ctx->attended.end(), 0);
   std::fill(ctx->in_store.begin(), ctx->in_store.end(), 1);
+  std::fill(ctx->logits_of.begin(), ctx->logits_of.end(), -1);
   std::fill(ctx->ev_compress_live.begin(), ctx->ev_compress_live.end(), 0);
   return SCALEKV_OK;
 }
@@ -483,10 +517,14 @@ scalekv_status scalekv_attend(scalekv_ctx *ctx, int32_t layer, scalekv_tensor Q,
       const bool fused = !ctx->in_store[layer];
       TensorView kc, vc;
       if (fused) { kc = tview(ctx->pend_k[layer]); vc = tview(ctx->pend_v[layer]); }
-      if (!ctx->tc.launch(lv, tview(Q), tview(O), lse, nk, fused ? &kc : nullptr, fused ? &vc : nullptr,
-                          p.N[ctx->next_scale[layer] - 1], ctx->scale, ctx->s_main, e))
+      const int k = ctx->next_scale[layer] - 1;
+      const std::vector<int> &win = p.windows[k];
+      float *wl = win.empty() ? nullptr : reinterpret_cast<float *>(ctx->ws + p.off_logits) + (size_t)(layer & 1) * p.logits_elems;
+      if (!ctx->tc.launch(lv, tview(Q), tview(O), lse, nk, fused ? &kc : nullptr, fused ? &vc : nullptr, p.N[k], ctx->scale, wl,
+                          p.ld_s, win.data(), (int)win.size(), ctx->s_main, e))
         return fail(ctx, SCALEKV_ERR_CUDA, "attend launch: %s", e.c_str());
       ctx->in_store[layer] = 1;
+      ctx->logits_of[layer] = wl ? k : -1;
     } else {
       dim3 grid((nk + 63) / 64, p.n_slices);
       if (ctx->dtype == SCALEKV_BF16)
@@ -530,12 +568,14 @@ scalekv_status scalekv_compress(scalekv_ctx *ctx, int32_t layer, scalekv_tensor 
     if (st != SCALEKV_OK) return st;
   } else {
     LayerView lv = layer_view(ctx, layer);
-    float *logits = reinterpret_cast<float *>(ctx->ws + p.off_logits);
+    float *logits = reinterpret_cast<float *>(ctx->ws + p.off_logits) + (size_t)(layer & 1) * p.logits_elems;
     float *scores = reinterpret_cast<float *>(ctx->ws + p.off_scores);
-    uint32_t *keys = reinterpret_cast<uint32_t *>(ctx->ws + p.off_keys);
     int *keep = reinterpret_cast<int *>(ctx->ws + p.off_keep);
     int *kept = reinterpret_cast<int *>(ctx->ws + p.off_kept);
-    {
+    // the logits of exactly this window may already be there, recorded by attend
+    bool recorded = ctx->logits_of[layer] == k && (int)p.windows[k].size() == wa.w;
+    for (int j = 0; recorded && j < wa.w; ++j) recorded = p.windows[k][j] == wa.pos[j];
+    if (!recorded) {
       Scope sc(ctx, s, kScore);
       dim3 grid((L + 63) / 64, p.n_slices);
       if (ctx->dtype == SCALEKV_BF16)
@@ -545,17 +585,14 @@ scalekv_status scalekv_compress(scalekv_ctx *ctx, int32_t layer, scalekv_tensor 
         score_logits_kernel<float, 64><<<grid, 256, 2 * 64 * 68 * 4, s>>>(lv, tview(Qw), wa, qw_is_full_map, logits, p.ld_s,
                                                                          ctx->scale);
     }
-    {
-      Scope sc(ctx, s, kScore);
-      score_reduce_kernel<<<p.n_slices, 512, 0, s>>>(lv, wa, logits, p.ld_s, scores, p.ld_s);
-    }
+    ctx->logits_of[layer] = -1;
     {
       Scope sc(ctx, s, kSelect);
-      select_kernel<<<p.n_slices, 1024, 0, s>>>(lv, wa, budget, scores, p.ld_s, keys, keep, kept);
+      score_select_kernel<<<p.n_slices, 1024, (size_t)p.ld_s * 4, s>>>(lv, wa, budget, logits, p.ld_s, scores, p.ld_s, keep, kept);
     }
     {
       Scope sc(ctx, s, kCompact);
-      compact_kernel<<<dim3(p.n_slices, 2), 256, 0, s>>>(lv, keep, p.ld_s, kept);
+      compact_kernel<<<dim3(p.n_slices, 2, 4), 256, 0, s>>>(lv, keep, p.ld_s, kept);
     }
     ctx->scores_len = L;
     ctx->hist[layer] = budget + wa.w;
@@ -643,26 +680,7 @@ scalekv_status scalekv_layer_stats(scalekv_ctx *ctx, int32_t layer, scalekv_tens
 
 scalekv_status scalekv_window_centroids(int32_t h, int32_t w, int32_t n_patches, int32_t *pos, int32_t *count) {
   if (h < 1 || w < 1 || n_patches < 1 || !pos || !count) return SCALEKV_ERR_INVALID_ARG;
-  if ((long long)h * w <= n_patches) {
-    for (int i = 0; i < h * w; ++i) pos[i] = i;
-    *count = h * w;
-    return SCALEKV_OK;
-  }
-  int g = (int)std::floor(std::sqrt((double)n_patches));
-  while ((g + 1) * (g + 1) <= n_patches) ++g;
-  while (g * g > n_patches) --g;
-  std::vector<int> out;
-  for (int a = 0; a < g; ++a) {
-    const int r0 = (int)((long long)a * h / g), r1 = (int)((long long)(a + 1) * h / g);
-    if (r1 <= r0) continue;
-    for (int b = 0; b < g; ++b) {
-      const int c0 = (int)((long long)b * w / g), c1 = (int)((long long)(b + 1) * w / g);
-      if (c1 <= c0) continue;
-      out.push_back(((r0 + r1 - 1) / 2) * w + (c0 + c1 - 1) / 2);
-    }
-  }
-  std::sort(out.begin(), out.end());
-  out.erase(std::unique(out.begin(), out.end()), out.end());
+  const std::vector<int> out = centroid_window(h, w, n_patches);
   for (size_t i = 0; i < out.size(); ++i) pos[i] = out[i];
   *count = (int)out.size();
   return SCALEKV_OK;
