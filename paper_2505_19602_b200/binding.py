@@ -21,7 +21,7 @@ KEEP_ALL = -1
 MAX_WINDOW = 64
 BF16, F32 = 0, 1
 STATUS_NAMES = ["OK", "INVALID_ARG", "BAD_STATE", "CAPACITY", "UNSUPPORTED", "CUDA", "TIMEOUT", "DEVICE_CHECK"]
-KERNEL_CLASSES = ["append", "attend", "score", "select", "compact", "other"]
+KERNEL_CLASSES = ["append", "attend", "score_logits", "score_select", "compact", "other"]
 
 
 class ScaleKVError(RuntimeError):
@@ -321,7 +321,8 @@ class ScaleKV:
         self._check(self.lib.scalekv_launch_count(self.ctx, C.byref(n)))
         return n.value
 
-    def scalekv_profile_enable(self, on=True):
+    def scalekv_profile_enable(self, on=1):
+        """0 off, 1 events on the launching streams, 2 events with compress serialised onto stream_main."""
         self._check(self.lib.scalekv_profile_enable(self.ctx, int(on)))
 
     def scalekv_profile_read(self):

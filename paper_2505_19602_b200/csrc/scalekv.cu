@@ -181,7 +181,8 @@ struct scalekv_ctx {
   std::vector<char> ev_compress_live;
   int64_t launches = 0;
   int scores_len = 0;              // length of the score vectors left by the last evicting compress
-  bool profile = false;
+  bool profile = false;            // launches are bracketed by events
+  bool serialize = false;          // compress runs on stream_main (every kernel timed alone)
   struct Timed { cudaEvent_t a, b; int cls; };
   std::vector<Timed> timed;
   std::vector<cudaEvent_t> event_pool;
@@ -555,7 +556,8 @@ scalekv_status scalekv_compress(scalekv_ctx *ctx, int32_t layer, scalekv_tensor 
   const int cand = L - wa.w;
   const int budget = p.budgets[(size_t)layer * p.K + k];
   const bool evict = budget != SCALEKV_KEEP_ALL && budget < cand;
-  cudaStream_t s = ctx->s_side;
+  // while per-kernel timing is on, compress runs on stream_main too, so that every kernel is timed alone
+  cudaStream_t s = ctx->serialize ? ctx->s_main : ctx->s_side;
   const bool copy_now = !ctx->in_store[layer];
   st = materialize(ctx, layer);
   if (st != SCALEKV_OK) return st;
@@ -809,6 +811,7 @@ scalekv_status scalekv_profile_enable(scalekv_ctx *ctx, int32_t on) {
   drain_profile(ctx);
   if (on) for (int i = 0; i < kNumClasses; ++i) { ctx->prof_ms[i] = 0; ctx->prof_n[i] = 0; }
   ctx->profile = on != 0;
+  ctx->serialize = on == 2;
   return SCALEKV_OK;
 }
 

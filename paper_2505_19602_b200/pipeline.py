@@ -98,13 +98,23 @@ def run_pass(kv: binding.ScaleKV, inputs: PassInputs, windows, compress_last=Fal
 
 
 def pass_work(wl: synth.Workload, budgets, windows):
-    """Algorithmic work of one pass, from the schedule alone: attention flops (4 n_k L d per
-    slice-step), bytes of K read by scoring, bytes moved by compaction (upper bound: every kept row
-    beyond the untouched prefix is unknown on the host, so all kept rows are counted), append bytes."""
+    """Algorithmic work of one pass, from the schedule alone.
+
+    attend_flop       4 n_k L d per slice-step.
+    attend_min_bytes  what attend must move: K and V of the L entries once, Q and O, plus - since it also
+                      appends - the write of the current map's K/V rows and positions into the pages, and
+                      the write of the w x L window logits.
+    select_bytes      the score + select kernel: w x L logits and L positions in, L scores and the keep
+                      list out.
+    compact_bytes     K and V rows (and positions) of the survivors, read and written (upper bound: which
+                      rows already sit in place is unknown on the host).
+    score_bytes       K read by the stand-alone logits kernel; zero when attend recorded the logits.
+    """
     n = wl.n_tokens
     d = wl.head_dim
     esz = 2 if wl.dtype == "bf16" else 4
     slices = wl.batch * wl.n_heads
+    fused = wl.dtype == "bf16" and d == 128
     out = {"attend_flop": 0, "attend_min_bytes": 0, "score_bytes": 0, "compact_bytes": 0, "append_bytes": 0,
            "select_bytes": 0, "attend_launches": 0}
     per_scale_flop = [0] * wl.n_scales
@@ -112,21 +122,25 @@ def pass_work(wl: synth.Workload, budgets, windows):
         hist = 0
         for k in range(wl.n_scales):
             L = hist + n[k]
+            w = len(windows[k]) if windows[k] is not None else n[k]
             f = 4 * n[k] * L * d * slices
             out["attend_flop"] += f
             per_scale_flop[k] += f
             out["attend_min_bytes"] += (2 * L + 2 * n[k]) * d * esz * slices
-            out["append_bytes"] += 2 * 2 * n[k] * d * esz * slices
+            if fused:
+                out["attend_min_bytes"] += (2 * n[k] * d * esz + 4 * n[k] + 4 * w * L) * slices
+            else:
+                out["append_bytes"] += 2 * 2 * n[k] * d * esz * slices
             out["attend_launches"] += 1
             if k + 1 == wl.n_scales:
                 break
-            w = len(windows[k]) if windows[k] is not None else n[k]
             cand = L - w
             b = budgets[l][k]
             if b != binding.KEEP_ALL and b < cand:
-                out["score_bytes"] += L * d * esz * slices
-                out["select_bytes"] += (4 * L + 4 * (b + w)) * slices
-                out["compact_bytes"] += (b + w) * 2 * 2 * d * esz * slices
+                if not fused:
+                    out["score_bytes"] += L * d * esz * slices
+                out["select_bytes"] += (4 * w * L + 4 * L + 4 * L + 4 * (b + w)) * slices
+                out["compact_bytes"] += (b + w) * (2 * 2 * d * esz + 8) * slices
                 hist = b + w
             else:
                 hist = L
