@@ -192,3 +192,80 @@ def test_layer_stats_matches_oracle_and_recovers_planted_roles():
     for k in range(3, len(sides) - 1):      # scales whose history exceeds K' by a wide margin
         assert np.nonzero(roles[:, k])[0].tolist() == planted
     kv.close()
+
+
+def test_bf16_three_ctas_per_slice_and_window_paths():
+    """n_k up to 576: a slice's queries span three CTAs (two with two query tiles, one with one).  Run
+    once with the window logits recorded by attend and once with the stand-alone logits kernel."""
+    sides = (2, 6, 12, 18, 24)
+    n = orc.scale_token_counts(sides)
+    budgets = [[100] * len(sides), [40] * len(sides)]
+    wl = synth.Workload("t", 2, 1, 2, 128, "bf16", sides, seed=17, n_drafters=1)
+    for patches in (16, 0):
+        kv = binding.ScaleKV(2, 1, 2, 128, "bf16", sides, sides, budgets, max_window=16, window_patches=patches)
+        run = ParityRun(kv, "bf16", sides, budgets, lambda l, k: synth.scale_inputs(wl, l, k),
+                        lambda k: orc.window_centroids(sides[k], sides[k], 16), all_slices(2, 1, 2), compress_last=True).run()
+        assert run.evictions >= 12
+        kv.close()
+
+
+def test_compress_and_export_without_attend():
+    """append -> compress with no attend in between: the library copies the map itself."""
+    sides = (4, 8, 12)
+    n = orc.scale_token_counts(sides)
+    budgets = [[20] * 3]
+    kv = binding.ScaleKV(1, 1, 2, 128, "bf16", sides, sides, budgets, max_window=16)
+    g = torch.Generator().manual_seed(31)
+    caches = [orc.SliceCache(n, 128) for _ in range(2)]
+    for k in range(3):
+        Q, K, V = (torch.randn(1, 2, n[k], 128, generator=g).to(torch.bfloat16) for _ in range(3))
+        Qd, Kd, Vd = Q.cuda(), K.cuda(), V.cuda()
+        torch.cuda.synchronize()
+        kv.scalekv_append(0, k, Kd, Vd)
+        wpos = orc.window_centroids(sides[k], sides[k], 16)
+        if k == 1:
+            pos, Kg, Vg = kv.scalekv_export_slice(0, 0, 1, with_kv=True)      # export straight after append
+            assert len(pos) == caches[1].pos.shape[0] + n[k]
+        kv.scalekv_compress(0, Qd, wpos, qw_is_full_map=True)
+        kv.scalekv_sync()
+        for h in range(2):
+            c = caches[h]
+            c.append(K[0, h].double().numpy(), V[0, h].double().numpy())
+            want, _ = c.compress(Q[0, h].double().numpy()[wpos], wpos, budgets[0][k])
+            pos, Kg, Vg = kv.scalekv_export_slice(0, 0, h, with_kv=True)
+            assert np.array_equal(pos.numpy(), want)
+            assert np.array_equal(Kg.double().numpy(), c.K) and np.array_equal(Vg.double().numpy(), c.V)
+    kv.close()
+
+
+def test_full_size_single_layer_sampled_slices():
+    """configs[1] at full size (B 8, H 16, 13 scales, 10 % budget) in the launch configuration the
+    benchmark uses; the oracle follows three sampled slices through the whole pass."""
+    wl = synth.WORKLOADS["layer2b"]
+    n = wl.n_tokens
+    b10 = orc.budget_tokens(0.10, n)
+    budgets = [[b10] * wl.n_scales]
+    kv = binding.ScaleKV(1, wl.batch, wl.n_heads, 128, "bf16", wl.sides, wl.sides, budgets, max_window=16)
+    slices = [(0, 0, 0), (0, 3, 7), (0, 7, 15)]
+    run = ParityRun(kv, "bf16", wl.sides, budgets, lambda l, k: synth.scale_inputs(wl, l, k, device="cuda"),
+                    lambda k: orc.window_centroids(wl.sides[k], wl.sides[k], 16), slices).run()
+    assert run.evictions == 3 * 5          # compress evicts at scales 8..12 (1-based) of the 13
+    assert kv.scalekv_lengths(0)[7][15] == b10 + 16 + n[-1]
+    kv.close()
+
+
+def test_full_size_pass_sampled_slices():
+    """configs[2] at full size (32 layers, drafter / refiner budgets of 30 % / 3 %, planted roles): all
+    layers run on the GPU, the oracle follows one slice in each of two drafter and two refiner layers."""
+    wl = synth.WORKLOADS["pass2b"]
+    n = wl.n_tokens
+    planted = synth.drafter_layers(wl)
+    bd, br = orc.budget_tokens(0.30, n), orc.budget_tokens(0.03, n)
+    budgets = [[bd if l in planted else br] * wl.n_scales for l in range(wl.n_layers)]
+    kv = binding.ScaleKV(wl.n_layers, wl.batch, wl.n_heads, 128, "bf16", wl.sides, wl.sides, budgets, max_window=16)
+    refiners = [l for l in range(wl.n_layers) if l not in planted]
+    slices = [(planted[0], 0, 0), (planted[-1], 7, 15), (refiners[0], 2, 5), (refiners[-1], 5, 9)]
+    run = ParityRun(kv, "bf16", wl.sides, budgets, lambda l, k: synth.scale_inputs(wl, l, k, device="cuda"),
+                    lambda k: orc.window_centroids(wl.sides[k], wl.sides[k], 16), slices, check_lse=False).run()
+    assert run.evictions > 0
+    kv.close()
