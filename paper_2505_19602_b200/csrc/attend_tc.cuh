@@ -383,6 +383,7 @@ struct Params {
   // observation window (Sec. 3.3): when win_logits is not null, the base-2 logits scale * log2(e) * <q, k>
   // of the w window rows against every cache entry are recorded in win_logits[slice][rank][slot]
   float *win_logits;
+  float *win_lse;      // [slice][rank]: base-2 log-sum-exp of each window row's logits (its softmax normaliser)
   int ld_l;            // leading dimension of a logit row
   int w;
   int win_pos[kMaxWindow];   // ascending raster indices of the window rows inside the current map
@@ -757,6 +758,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       }
       if (prm.lse != nullptr && half == 0 && qi < n_k)
         prm.lse[(size_t)slice * n_k + qi] = (m_used[qt] + log2f(lsum)) * 0.6931471805599453f;
+      if (wrank[qt] >= 0 && half == 0) prm.win_lse[(size_t)slice * prm.w + wrank[qt]] = m_used[qt] + log2f(lsum);
     }
     tc_fence_before();
   }
@@ -828,7 +830,7 @@ struct AttendTc {
   // reads them there and copies them in), else nullptr.
   // win_logits / win_pos / w: where to record the window rows' logits (nullptr: do not).
   bool launch(const LayerView &lv, const TensorView &Q, const TensorView &O, float *lse, int n_k, const TensorView *Kc,
-              const TensorView *Vc, int n_prev, float scale, float *win_logits, int ld_l, const int *win_pos, int w,
+              const TensorView *Vc, int n_prev, float scale, float *win_logits, float *win_lse, int ld_l, const int *win_pos, int w,
               cudaStream_t stream, std::string &err) {
     CUtensorMap tmQ, tmKc, tmVc;
     const int B = lv.n_slices / lv.n_heads;
@@ -847,6 +849,7 @@ struct AttendTc {
     prm.fused_append = fused ? 1 : 0;
     prm.n_prev = n_prev;
     prm.win_logits = win_logits;
+    prm.win_lse = win_lse;
     prm.ld_l = ld_l;
     prm.w = win_logits ? w : 0;
     for (int e = 0; e < kMaxWindow; ++e) prm.win_pos[e] = (win_logits && e < w) ? win_pos[e] : -1;

@@ -313,14 +313,16 @@ __device__ __forceinline__ float block_reduce_sum(float v, float *red) {
 
 // ------------------------------------------------------------------------------------------
 // score, step 2, aggregation and selection in one kernel, one CTA of 1024 threads per slice
-// (Sec. 3.3, Eq. 5 and the selection paragraph).  Input: base-2 logits y[w][L] of the window rows.
-//   1. per window row j: m_j = max_i y_ji and Z_j = sum_i 2^(y_ji - m_j)   (two sweeps, 16 rows at a time)
-//   2. s_i = (1/w) sum_j 2^(y_ji - m_j) / Z_j  -> scores (global, for inspection) and, as the bit
+// (Sec. 3.3, Eq. 5 and the selection paragraph).  Input: base-2 logits y[w][L] of the window rows
+// and, when attend recorded them, the rows' base-2 log-sum-exp lse[w] (then the logits are read once).
+//   1. (without lse) per window row j: m_j = max_i y_ji, Z_j = sum_i 2^(y_ji - m_j), lse_j = m_j + log2 Z_j
+//   2. s_i = (1/w) sum_j 2^(y_ji - lse_j)  -> scores (global, for inspection) and, as the bit
 //      pattern of the non-negative float, the radix key of entry i in shared memory; window entries
 //      get a sentinel and never take part in the selection
 //   3. radix select of the k'-th largest key, 8 bits per pass, warp-aggregated histogram updates
 //   4. ordered emit of the ascending slot list of survivors (selected U window); ties at the
-//      threshold go to the lowest slots = lowest original positions.  Deterministic.
+//      threshold go to the lowest slots = lowest original positions.  Every thread owns a run of
+//      consecutive entries, so two block scans order the whole list.  Deterministic.
 // Dynamic shared memory: 4 * ld_s bytes of keys.
 // ------------------------------------------------------------------------------------------
 constexpr uint32_t kWindowKey = 0xFFFFFFFFu;
@@ -352,11 +354,11 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int *warp_sums, int *
 }
 
 __global__ void __launch_bounds__(1024) score_select_kernel(LayerView lv, WindowArg wa, int budget, const float *logits,
-                                                            int ld_l, float *scores, int ld_s, int *keep_list,
-                                                            int *kept_count) {
+                                                            const float *lse_in, int ld_l, float *scores, int ld_s,
+                                                            int *keep_list, int *kept_count) {
   extern __shared__ uint32_t key[];            // [L]
   __shared__ float part[32][16];               // per-warp partial maxima / sums of 16 rows
-  __shared__ float m_row[kMaxWindow], inv_row[kMaxWindow];
+  __shared__ float m_row[kMaxWindow], lse_row[kMaxWindow];
   __shared__ int hist[256];
   __shared__ int warp_sums[33];
   __shared__ uint32_t sh_prefix;
@@ -368,57 +370,64 @@ __global__ void __launch_bounds__(1024) score_select_kernel(LayerView lv, Window
   const float *y = logits + (size_t)slice * w * ld_l;
   int *out = keep_list + (size_t)slice * ld_s;
 
-  // 1. row maxima and normalisers, 16 rows per round
-  for (int g0 = 0; g0 < w; g0 += 16) {
-    const int nr = w - g0 < 16 ? w - g0 : 16;
-    float acc[16];
-#pragma unroll
-    for (int r = 0; r < 16; ++r) acc[r] = -INFINITY;
-    for (int i = tid; i < L; i += 1024) {
-#pragma unroll
-      for (int r = 0; r < 16; ++r)
-        if (r < nr) acc[r] = fmaxf(acc[r], y[(size_t)(g0 + r) * ld_l + i]);
-    }
-#pragma unroll
-    for (int r = 0; r < 16; ++r) {
-      float v = acc[r];
-      for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
-      if (lane == 0) part[wid][r] = v;
-    }
+  if (lse_in != nullptr) {
+    if (tid < w) lse_row[tid] = lse_in[(size_t)slice * w + tid];
     __syncthreads();
-    if (tid < 16) {
-      float v = part[0][tid];
-      for (int k = 1; k < 32; ++k) v = fmaxf(v, part[k][tid]);
-      if (tid < nr) m_row[g0 + tid] = v;
-    }
-    __syncthreads();
+  } else {
+    // 1. row maxima and normalisers, 16 rows per round
+    for (int g0 = 0; g0 < w; g0 += 16) {
+      const int nr = w - g0 < 16 ? w - g0 : 16;
+      float acc[16];
 #pragma unroll
-    for (int r = 0; r < 16; ++r) acc[r] = 0.f;
-    for (int i = tid; i < L; i += 1024) {
+      for (int r = 0; r < 16; ++r) acc[r] = -INFINITY;
+      for (int i = tid; i < L; i += 1024) {
 #pragma unroll
-      for (int r = 0; r < 16; ++r)
-        if (r < nr) acc[r] += exp2f(y[(size_t)(g0 + r) * ld_l + i] - m_row[g0 + r]);
-    }
+        for (int r = 0; r < 16; ++r)
+          if (r < nr) acc[r] = fmaxf(acc[r], y[(size_t)(g0 + r) * ld_l + i]);
+      }
 #pragma unroll
-    for (int r = 0; r < 16; ++r) {
-      float v = acc[r];
-      for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-      if (lane == 0) part[wid][r] = v;
+      for (int r = 0; r < 16; ++r) {
+        float v = acc[r];
+        for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+        if (lane == 0) part[wid][r] = v;
+      }
+      __syncthreads();
+      if (tid < 16) {
+        float v = part[0][tid];
+        for (int k = 1; k < 32; ++k) v = fmaxf(v, part[k][tid]);
+        if (tid < nr) m_row[g0 + tid] = v;
+      }
+      __syncthreads();
+#pragma unroll
+      for (int r = 0; r < 16; ++r) acc[r] = 0.f;
+      for (int i = tid; i < L; i += 1024) {
+#pragma unroll
+        for (int r = 0; r < 16; ++r)
+          if (r < nr) acc[r] += exp2f(y[(size_t)(g0 + r) * ld_l + i] - m_row[g0 + r]);
+      }
+#pragma unroll
+      for (int r = 0; r < 16; ++r) {
+        float v = acc[r];
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        if (lane == 0) part[wid][r] = v;
+      }
+      __syncthreads();
+      if (tid < 16) {
+        float v = 0.f;
+        for (int k = 0; k < 32; ++k) v += part[k][tid];     // fixed order: deterministic
+        if (tid < nr) lse_row[g0 + tid] = m_row[g0 + tid] + log2f(v);
+      }
+      __syncthreads();
     }
-    __syncthreads();
-    if (tid < 16) {
-      float v = 0.f;
-      for (int k = 0; k < 32; ++k) v += part[k][tid];     // fixed order: deterministic
-      if (tid < nr) inv_row[g0 + tid] = 1.f / (v * (float)w);
-    }
-    __syncthreads();
   }
 
   // 2. scores and keys
+  const float inv_w = 1.f / (float)w;
   int n_win_local = 0;
   for (int i = tid; i < L; i += 1024) {
     float sc = 0.f;
-    for (int j = 0; j < w; ++j) sc += exp2f(y[(size_t)j * ld_l + i] - m_row[j]) * inv_row[j];
+    for (int j = 0; j < w; ++j) sc += exp2f(y[(size_t)j * ld_l + i] - lse_row[j]);
+    sc *= inv_w;
     scores[(size_t)slice * ld_s + i] = sc;
     const bool win = is_window_pos(wa, lv.pos_pool[slot_row(lv, slice, i)]);
     key[i] = win ? kWindowKey : (__float_as_uint(sc) & 0x7FFFFFFFu);
@@ -461,9 +470,9 @@ __global__ void __launch_bounds__(1024) score_select_kernel(LayerView lv, Window
           if (lane >= o) incl += t;
         }
         const int rem = sh_remaining;
-        int before = incl - tot;
-        const bool here = before < rem && incl >= rem;
-        if (here) {
+        const int before = incl - tot;
+        __syncwarp();
+        if (before < rem && incl >= rem) {
           int dsel = 0, r = rem - before;
 #pragma unroll
           for (int e = 0; e < 8; ++e) {
@@ -483,79 +492,103 @@ __global__ void __launch_bounds__(1024) score_select_kernel(LayerView lv, Window
   const bool keep_all = (kprime >= cand);
   const bool keep_none = (kprime == 0);
 
-  // 4. ordered emit
-  int base_out = 0, base_tie = 0;
-  for (int i0 = 0; i0 < L; i0 += 1024) {
-    const int i = i0 + tid;
-    uint32_t k = 0;
-    bool win = false, gt = false, tie = false;
-    if (i < L) {
-      k = key[i];
-      win = (k == kWindowKey);
-      if (!win) {
-        if (keep_all) gt = true;
-        else if (!keep_none) { gt = k > threshold; tie = (k == threshold); }
+  // 4. ordered emit: thread t owns entries [t * E, (t + 1) * E)
+  const int E = (L + 1023) >> 10;
+  const int i_lo = tid * E, i_hi = (i_lo + E < L) ? i_lo + E : L;
+  int n_tie = 0;
+  for (int i = i_lo; i < i_hi; ++i) {
+    const uint32_t k = key[i];
+    n_tie += (k != kWindowKey && !keep_all && !keep_none && k == threshold) ? 1 : 0;
+  }
+  int tie_total, keep_total;
+  int tie_rank = block_exclusive_scan(n_tie, warp_sums, &tie_total);
+  int n_keep = 0;
+  {
+    int tr = tie_rank;
+    for (int i = i_lo; i < i_hi; ++i) {
+      const uint32_t k = key[i];
+      bool keep = (k == kWindowKey);
+      if (!keep) {
+        if (keep_all) keep = true;
+        else if (!keep_none) {
+          if (k > threshold) keep = true;
+          else if (k == threshold) { keep = tr < n_ties_taken; ++tr; }
+        }
+      }
+      n_keep += keep ? 1 : 0;
+    }
+  }
+  int oidx = block_exclusive_scan(n_keep, warp_sums, &keep_total);
+  for (int i = i_lo; i < i_hi; ++i) {
+    const uint32_t k = key[i];
+    bool keep = (k == kWindowKey);
+    if (!keep) {
+      if (keep_all) keep = true;
+      else if (!keep_none) {
+        if (k > threshold) keep = true;
+        else if (k == threshold) { keep = tie_rank < n_ties_taken; ++tie_rank; }
       }
     }
-    int tie_total, keep_total;
-    const int tie_rank = base_tie + block_exclusive_scan(tie ? 1 : 0, warp_sums, &tie_total);
-    const bool keep = win || gt || (tie && tie_rank < n_ties_taken);
-    const int oidx = base_out + block_exclusive_scan(keep ? 1 : 0, warp_sums, &keep_total);
-    if (keep) out[oidx] = i;
-    base_tie += tie_total;
-    base_out += keep_total;
+    if (keep) out[oidx++] = i;
   }
-  if (tid == 0) kept_count[slice] = base_out;
+  if (tid == 0) kept_count[slice] = keep_total;
 }
 
 // ------------------------------------------------------------------------------------------
 // compact: slot j <- old slot keep[j], in place (Sec. 3.3, pruning).  grid (n_slices, 2, 4):
 // blockIdx.y = 0 moves K (and, in column block 0, pos), 1 moves V; blockIdx.z picks a quarter of
 // the row's 16-byte pieces, so that a slice's move is spread over 8 CTAs that touch disjoint bytes.
-// keep is ascending, so keep[j] >= j: within a chunk every source is read before any destination
-// is written, and the sources of later chunks lie beyond every earlier destination.  256 threads,
-// chunks of 256 * 8 / ppq rows (ppq = pieces per row quarter), 8 pieces in flight per thread.
+// The slice's page table and keep list are staged in shared memory first, so that the row moves
+// depend on no further global look-up.  keep is ascending, so keep[j] >= j: within a chunk every
+// source is read before any destination is written, and the sources of later chunks lie beyond
+// every earlier destination.  256 threads, chunks of 2048 / ppq rows (ppq = pieces per row
+// quarter), 8 pieces in flight per thread.  Dynamic shared memory: 4 * (ld_s + pages_per_slice) B.
 // ------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) compact_kernel(LayerView lv, const int *keep_list, int ld_s, const int *kept_count) {
+  extern __shared__ int csm[];
+  int *list = csm;                 // [kept]
+  int *pt = csm + ld_s;            // [pages_per_slice]
   const int slice = blockIdx.x;
   const int which = blockIdx.y;
   const int quarter = blockIdx.z;
   char *pool = which == 0 ? lv.k_pool : lv.v_pool;
-  const int *list = keep_list + (size_t)slice * ld_s;
   const int kept = kept_count[slice];
+  for (int i = threadIdx.x; i < kept; i += 256) list[i] = __ldg(keep_list + (size_t)slice * ld_s + i);
+  for (int i = threadIdx.x; i < lv.pages_per_slice; i += 256) pt[i] = __ldg(lv.page_table + (size_t)slice * lv.pages_per_slice + i);
+  __syncthreads();
+  auto row_of = [&](int slot) { return ((size_t)pt[slot >> lv.page_shift] << lv.page_shift) + (size_t)(slot & lv.page_mask); };
   const int ppr = lv.row_bytes >> 4;       // 16-byte pieces per row
   const int ppq = ppr >> 2;                // pieces of this CTA's quarter (row_bytes is a multiple of 64)
   const int C = 2048 / ppq;                // rows per chunk
   int lo = 0, hi = kept;                   // first j with keep[j] != j (the untouched prefix is skipped)
   while (lo < hi) {
     const int mid = (lo + hi) >> 1;
-    if (__ldg(list + mid) == mid) lo = mid + 1; else hi = mid;
+    if (list[mid] == mid) lo = mid + 1; else hi = mid;
   }
   const bool do_pos_cta = which == 0 && quarter == 0;
+  const int r_in = threadIdx.x / ppq, c = quarter * ppq + threadIdx.x % ppq;   // piece u of a thread: row r_in + u * 256 / ppq
+  const int r_step = 256 / ppq;
+  const bool pos_thread = do_pos_cta && (threadIdx.x % ppq == 0);
   for (int c0 = lo; c0 < kept; c0 += C) {
     uint4 buf[8];
     int pv[8];
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
-      const int piece = threadIdx.x + u * 256;
-      const int r = piece / ppq, c = quarter * ppq + piece % ppq;
-      const int j = c0 + r;
+      const int j = c0 + r_in + u * r_step;
       if (j < kept) {
-        const size_t row = slot_row(lv, slice, __ldg(list + j));
+        const size_t row = row_of(list[j]);
         buf[u] = reinterpret_cast<const uint4 *>(pool + row * lv.row_bytes)[c];
-        if (do_pos_cta && piece % ppq == 0) pv[u] = lv.pos_pool[row];
+        if (pos_thread) pv[u] = lv.pos_pool[row];
       }
     }
     __syncthreads();
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
-      const int piece = threadIdx.x + u * 256;
-      const int r = piece / ppq, c = quarter * ppq + piece % ppq;
-      const int j = c0 + r;
+      const int j = c0 + r_in + u * r_step;
       if (j < kept) {
-        const size_t row = slot_row(lv, slice, j);
+        const size_t row = row_of(j);
         reinterpret_cast<uint4 *>(pool + row * lv.row_bytes)[c] = buf[u];
-        if (do_pos_cta && piece % ppq == 0) lv.pos_pool[row] = pv[u];
+        if (pos_thread) lv.pos_pool[row] = pv[u];
       }
     }
   }

@@ -48,7 +48,7 @@ struct Plan {
   size_t off_k, off_v, off_pos, off_pt, off_len, off_status, pool_bytes;
   size_t pt_elems, logits_elems;
   // workspace layout
-  size_t off_logits, off_scores, off_keys, off_keep, off_kept, off_acc, off_qw, ws_bytes;
+  size_t off_logits, off_wlse, off_scores, off_keys, off_keep, off_kept, off_acc, off_qw, ws_bytes;
 };
 
 // Raster indices of the observation window of an h x w map (see scalekv_window_centroids).
@@ -149,6 +149,7 @@ scalekv_status make_plan(const scalekv_config *c, Plan &p, std::string &err) {
   o = 0;
   p.logits_elems = (size_t)p.n_slices * p.max_window * p.ld_s;   // one buffer per layer parity
   p.off_logits = o; o = align_up(o + 2 * p.logits_elems * 4, 1024);
+  p.off_wlse = o; o = align_up(o + 2 * (size_t)p.n_slices * p.max_window * 4, 1024);   // one per layer parity
   p.off_scores = o; o = align_up(o + (size_t)p.n_slices * p.ld_s * 4, 1024);
   p.off_keys = o; o = align_up(o + (size_t)p.n_slices * p.ld_s * 4, 1024);
   p.off_keep = o; o = align_up(o + (size_t)p.n_slices * p.ld_s * 4, 1024);
@@ -408,6 +409,7 @@ scalekv_status scalekv_init(const scalekv_config *cfg, scalekv_ctx **out) {
     set_smem(layer_stats_kernel<float, 64>, (size_t)(64 + p.ld_s) * 4);
   }
   set_smem(score_select_kernel, (size_t)p.ld_s * 4);
+  set_smem(compact_kernel, (size_t)(p.ld_s + (p.ld_s + p.P - 1) / p.P + 1) * 4);
   cudaGetLastError();
   std::string tc_err;
   if (!ctx->tc.init(cfg->dtype, p.d, ctx->pool + p.off_k, ctx->pool + p.off_v, p.n_pages, p.P, tc_err)) {
@@ -521,8 +523,9 @@ scalekv_status scalekv_attend(scalekv_ctx *ctx, int32_t layer, scalekv_tensor Q,
       const int k = ctx->next_scale[layer] - 1;
       const std::vector<int> &win = p.windows[k];
       float *wl = win.empty() ? nullptr : reinterpret_cast<float *>(ctx->ws + p.off_logits) + (size_t)(layer & 1) * p.logits_elems;
+      float *wlse = reinterpret_cast<float *>(ctx->ws + p.off_wlse) + (size_t)(layer & 1) * p.n_slices * p.max_window;
       if (!ctx->tc.launch(lv, tview(Q), tview(O), lse, nk, fused ? &kc : nullptr, fused ? &vc : nullptr, p.N[k], ctx->scale, wl,
-                          p.ld_s, win.data(), (int)win.size(), ctx->s_main, e))
+                          wlse, p.ld_s, win.data(), (int)win.size(), ctx->s_main, e))
         return fail(ctx, SCALEKV_ERR_CUDA, "attend launch: %s", e.c_str());
       ctx->in_store[layer] = 1;
       ctx->logits_of[layer] = wl ? k : -1;
@@ -590,11 +593,14 @@ scalekv_status scalekv_compress(scalekv_ctx *ctx, int32_t layer, scalekv_tensor 
     ctx->logits_of[layer] = -1;
     {
       Scope sc(ctx, s, kSelect);
-      score_select_kernel<<<p.n_slices, 1024, (size_t)p.ld_s * 4, s>>>(lv, wa, budget, logits, p.ld_s, scores, p.ld_s, keep, kept);
+      const float *wlse = recorded ? reinterpret_cast<float *>(ctx->ws + p.off_wlse) + (size_t)(layer & 1) * p.n_slices * p.max_window
+                                   : nullptr;
+      score_select_kernel<<<p.n_slices, 1024, (size_t)p.ld_s * 4, s>>>(lv, wa, budget, logits, wlse, p.ld_s, scores, p.ld_s, keep,
+                                                                       kept);
     }
     {
       Scope sc(ctx, s, kCompact);
-      compact_kernel<<<dim3(p.n_slices, 2, 4), 256, 0, s>>>(lv, keep, p.ld_s, kept);
+      compact_kernel<<<dim3(p.n_slices, 2, 4), 256, (size_t)(p.ld_s + lv.pages_per_slice) * 4, s>>>(lv, keep, p.ld_s, kept);
     }
     ctx->scores_len = L;
     ctx->hist[layer] = budget + wa.w;
