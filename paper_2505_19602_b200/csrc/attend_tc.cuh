@@ -2,7 +2,7 @@
 // O = softmax(scale * Q K^T) V with online softmax.  One CTA owns up to two 128-query tiles (A, B)
 // of one slice and streams the slice's K/V pages once for both.
 //
-// Roles inside a CTA of 384 threads (three warpgroups):
+// Roles inside a CTA of 128 + 128 * kParts threads:
 //   warp 0 (one thread) : TMA producer.  The query tiles once; then per 128-key tile the K and V rows into
 //                         128B-swizzled shared memory: history tiles page by page through the slice's
 //                         page table, tiles of a not yet appended current map from the caller's tensors.
@@ -11,17 +11,18 @@
 //                         j is  S_A(j), PV_B(j-1), S_B(j), PV_A(j): while one tile's softmax runs, the
 //                         tensor pipe works for the other tile.  With one query tile the two S buffers
 //                         alternate and S(j+1) is issued ahead of PV(j).
-//   warps 4-11          : softmax.  Warps 4-7 own columns 0-63 and warps 8-11 columns 64-127 of every S
-//                         tile; warp w and warp w + 4 share the 32 query rows (TMEM lanes) of quarter
-//                         w % 4, and all eight warps work on tile A's S, then on tile B's.  A thread
-//                         sweeps its half row once (tcgen05.ld): p = exp2(s * c - m) against the running
-//                         reference m with packed f32x2 arithmetic (a share of the exponentials on the
-//                         FMA pipe), the partial row sum, and P as bf16 pairs written back into the first
-//                         columns of its own half of the S buffer (tcgen05.st), from where the PV product
-//                         takes its A operand.  The two warps of a quarter meet on an mbarrier per tile:
-//                         only when a half row's sum shows that an exponent left the lazy band (2^8) do
-//                         both recompute the row against a new reference and rescale O.  At the end the
-//                         same warps normalise and store O, 64 columns each.
+//   warps 4 ..          : softmax, kParts warps per TMEM lane quarter (kParts = 2: warps 4-11).  Warp w takes
+//                         columns kCols * ((w - 4) / 4) .. + kCols - 1 of every S tile; the warps w, w + 4, ..
+//                         share the 32 query rows (TMEM lanes) of quarter w % 4, and all of them work on tile
+//                         A's S, then on tile B's.  A thread sweeps its row part once (tcgen05.ld):
+//                         p = exp2(s * c - m) against the running reference m with packed f32x2 arithmetic
+//                         (a share of the exponentials on the FMA pipe), the partial row sum, and P as bf16
+//                         pairs written back into the first columns of its own part of the S buffer
+//                         (tcgen05.st), from where the PV product takes its A operand.  The warps of a
+//                         quarter meet on an mbarrier per tile: only when a part's sum shows that an
+//                         exponent left the lazy band (2^8) do they recompute the row against a new
+//                         reference and rescale O.  At the end the same warps normalise and store O.
+//                         (Four warps per quarter, 16 softmax warps, measured the same as two.)
 //   warps 2-3           : append.  When the current map has not been copied into the store yet, its K/V
 //                         tiles come from the caller's tensors, and the CTA whose turn it is writes each
 //                         tile's rows from shared memory to the slice's pages (and their original
@@ -40,15 +41,19 @@
 namespace scalekv {
 namespace tc {
 
-constexpr int kThreads = 384;                    // warps: TMA, MMA, 2 x append, 8 x softmax
+constexpr int kParts = 2;                        // softmax warps per TMEM lane quarter: each takes 128 / kParts columns of an S tile
+constexpr int kCols = 128 / kParts;              // S columns per softmax thread and tile
+constexpr int kChunks = kCols / 32;              // tcgen05.ld x32 loads per thread and tile
+constexpr int kThreads = 128 + 128 * kParts;     // warps: TMA, MMA, 2 x append, 4 * kParts x softmax
 constexpr int kStages = 5;                       // one ring for the K and V tiles: K_0, V_0, K_1, V_1, ...
 constexpr uint32_t kTileBytes = 128 * 128 * 2;   // one 128 x 128 bf16 operand tile
 constexpr uint32_t kHalfBytes = kTileBytes / 2;  // 64 head-dim columns = one 128-byte swizzle span
-constexpr uint32_t kOffQ = 0;                    // two query tiles
+constexpr uint32_t kOffQ = 0;                    // two query tiles (the dynamic shared memory must start 1024-byte aligned)
 constexpr uint32_t kOffRing = kOffQ + 2 * kTileBytes;
 constexpr uint32_t kOffBar = kOffRing + kStages * kTileBytes;
-constexpr uint32_t kOffX = kOffBar + 256;           // exchange area of the softmax warp pairs: flags [2][4][2], values [4][2][32]
-constexpr uint32_t kSmemBytes = kOffX + 1280 + 1024;   // + alignment slack
+constexpr uint32_t kOffX = kOffBar + 256;        // exchange area of the softmax warps of a quarter: flags [2][4][kParts], values [4][kParts][32]
+constexpr uint32_t kSmemBytes = kOffX + 128 + 4 * kParts * 32 * 4;
+static_assert(kSmemBytes <= 232448, "more shared memory than a CTA can have");
 // barrier slots (8 bytes each): one full/empty pair per ring stage, one S/P/PV barrier per S buffer or query tile
 enum { bQFull = 0, bFull = 1, bEmpty = bFull + kStages, bSFull = bEmpty + kStages, bPFull = bSFull + 2, bPvDone = bPFull + 2,
        bPair = bPvDone + 2, bFinal = bPair + 4, bCount = bFinal + 2 };
@@ -174,23 +179,25 @@ __device__ __forceinline__ void tc_mma_ss_x8(uint32_t d_tmem, uint32_t a_lo, uin
       "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc)
       : "memory");
 }
-// TS: A = P in TMEM (8 columns per step inside a half of the S buffer, the second half 64 columns
-// further), B = V in shared memory as the MN-major operand (16 keys = 2048 B per step).
+// TS: A = P in TMEM (16 keys = 8 columns per step; every softmax thread's keys sit at the start of its
+// own kCols columns of the S buffer), B = V in shared memory as the MN-major operand (16 keys = 2048 B per step).
+__device__ __forceinline__ constexpr uint32_t p_col(int kk) { return (uint32_t)(((kk * 16) / kCols) * kCols + ((kk * 16) % kCols) / 2); }
 __device__ __forceinline__ void tc_mma_ts_x8(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t hi, uint32_t idesc,
                                              uint32_t accumulate_first) {
   asm volatile(
       "{\n\t.reg .pred e, pf, pt;\n\t.reg .b64 db;\n\t.reg .b32 at, bl;\n\t"
       "elect.sync _|e, 0xffffffff;\n\tsetp.ne.b32 pf, %5, 0;\n\tsetp.eq.b32 pt, 0, 0;\n\t"
       "mov.b64 db, {%2, %3};\n\t@e tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, pf;\n\t"
-      "add.u32 at, %1, 8;\n\tadd.u32 bl, %2, 128;\n\tmov.b64 db, {bl, %3};\n\t@e tcgen05.mma.cta_group::1.kind::f16 [%0], [at], db, %4, pt;\n\t"
-      "add.u32 at, %1, 16;\n\tadd.u32 bl, %2, 256;\n\tmov.b64 db, {bl, %3};\n\t@e tcgen05.mma.cta_group::1.kind::f16 [%0], [at], db, %4, pt;\n\t"
-      "add.u32 at, %1, 24;\n\tadd.u32 bl, %2, 384;\n\tmov.b64 db, {bl, %3};\n\t@e tcgen05.mma.cta_group::1.kind::f16 [%0], [at], db, %4, pt;\n\t"
-      "add.u32 at, %1, 64;\n\tadd.u32 bl, %2, 512;\n\tmov.b64 db, {bl, %3};\n\t@e tcgen05.mma.cta_group::1.kind::f16 [%0], [at], db, %4, pt;\n\t"
-      "add.u32 at, %1, 72;\n\tadd.u32 bl, %2, 640;\n\tmov.b64 db, {bl, %3};\n\t@e tcgen05.mma.cta_group::1.kind::f16 [%0], [at], db, %4, pt;\n\t"
-      "add.u32 at, %1, 80;\n\tadd.u32 bl, %2, 768;\n\tmov.b64 db, {bl, %3};\n\t@e tcgen05.mma.cta_group::1.kind::f16 [%0], [at], db, %4, pt;\n\t"
-      "add.u32 at, %1, 88;\n\tadd.u32 bl, %2, 896;\n\tmov.b64 db, {bl, %3};\n\t@e tcgen05.mma.cta_group::1.kind::f16 [%0], [at], db, %4, pt;\n\t"
+      "add.u32 at, %1, %6;\n\tadd.u32 bl, %2, 128;\n\tmov.b64 db, {bl, %3};\n\t@e tcgen05.mma.cta_group::1.kind::f16 [%0], [at], db, %4, pt;\n\t"
+      "add.u32 at, %1, %7;\n\tadd.u32 bl, %2, 256;\n\tmov.b64 db, {bl, %3};\n\t@e tcgen05.mma.cta_group::1.kind::f16 [%0], [at], db, %4, pt;\n\t"
+      "add.u32 at, %1, %8;\n\tadd.u32 bl, %2, 384;\n\tmov.b64 db, {bl, %3};\n\t@e tcgen05.mma.cta_group::1.kind::f16 [%0], [at], db, %4, pt;\n\t"
+      "add.u32 at, %1, %9;\n\tadd.u32 bl, %2, 512;\n\tmov.b64 db, {bl, %3};\n\t@e tcgen05.mma.cta_group::1.kind::f16 [%0], [at], db, %4, pt;\n\t"
+      "add.u32 at, %1, %10;\n\tadd.u32 bl, %2, 640;\n\tmov.b64 db, {bl, %3};\n\t@e tcgen05.mma.cta_group::1.kind::f16 [%0], [at], db, %4, pt;\n\t"
+      "add.u32 at, %1, %11;\n\tadd.u32 bl, %2, 768;\n\tmov.b64 db, {bl, %3};\n\t@e tcgen05.mma.cta_group::1.kind::f16 [%0], [at], db, %4, pt;\n\t"
+      "add.u32 at, %1, %12;\n\tadd.u32 bl, %2, 896;\n\tmov.b64 db, {bl, %3};\n\t@e tcgen05.mma.cta_group::1.kind::f16 [%0], [at], db, %4, pt;\n\t"
       "}" ::"r"(d_tmem),
-      "r"(a_tmem), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate_first)
+      "r"(a_tmem), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate_first), "n"(p_col(1)), "n"(p_col(2)), "n"(p_col(3)), "n"(p_col(4)),
+      "n"(p_col(5)), "n"(p_col(6)), "n"(p_col(7))
       : "memory");
 }
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
@@ -308,23 +315,23 @@ __host__ __device__ constexpr uint32_t instr_desc(bool b_mn_major) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
 }
 
-// Rare path of the softmax, taken together by the two warps that share a quarter's rows when the fast
-// sweep of one of their half rows overflowed the lazy band (always in the first tile, where no
-// reference exists yet).  The S half row is still intact at s_addr: a first sweep finds its maximum,
-// the two halves exchange theirs through shared memory (mine -> x_mine, the partner's <- x_other, with
-// one rendezvous on pair_bar), the reference moves up to the row maximum if that is larger, the half
-// row's P is recomputed against it and written over the first 32 columns (a chunk's columns are only
-// overwritten after it was read), and this warp's 64 columns of the O accumulator at o_addr are
-// multiplied by 2^(old reference - new reference) once the previous PV product of the tile has landed.
-// `valid` = number of columns of this half that hold keys (may be <= 0).  Returns the half row's sum
+// Rare path of the softmax, taken together by the kParts warps that share a quarter's rows when the
+// fast sweep of one of their row parts overflowed the lazy band (always in the first tile, where no
+// reference exists yet).  The S row part is still intact at s_addr: a first sweep finds its maximum,
+// the parts exchange theirs through shared memory (mine -> x_quarter[part], with one rendezvous on
+// pair_bar), the reference moves up to the row maximum if that is larger, the part's P is recomputed
+// against it and written over the part's first columns (a chunk's columns are only overwritten
+// after it was read), and this warp's kCols columns of the O accumulator at o_addr are multiplied by
+// 2^(old reference - new reference) once the previous PV product of the tile has landed.
+// `valid` = number of columns of this part that hold keys (may be <= 0).  Returns the part's row sum
 // and the new reference; sum < 0 when a wait gave up.
 struct Redo { float sum, m; };
-__device__ __noinline__ Redo redo_half(uint32_t s_addr, uint32_t o_addr, int valid, float c, float m_used, bool with_o,
+__device__ __noinline__ Redo redo_part(uint32_t s_addr, uint32_t o_addr, int valid, float c, float m_used, bool with_o,
                                        uint32_t pv_bar, uint32_t pv_parity, uint32_t pair_bar, uint32_t pair_parity,
-                                       volatile float *x_mine, volatile float *x_other, volatile int *abort_flag, int *status) {
+                                       volatile float *x_quarter, int part, int lane, volatile int *abort_flag, int *status) {
   float mt = -INFINITY;
 #pragma unroll 1
-  for (int cc = 0; cc < 2; ++cc) {
+  for (int cc = 0; cc < kChunks; ++cc) {
     float x[32];
     tc_ld32(s_addr + cc * 32, x);
     tc_wait_ld();
@@ -332,15 +339,16 @@ __device__ __noinline__ Redo redo_half(uint32_t s_addr, uint32_t o_addr, int val
     for (int i = 0; i < 32; ++i)
       if (cc * 32 + i < valid) mt = fmaxf(mt, x[i]);
   }
-  *x_mine = mt;
+  x_quarter[part * 32 + lane] = mt;
   mbar_arrive(pair_bar);
   if (!mbar_wait_warp(pair_bar, pair_parity, abort_flag, status)) return {-1.f, m_used};
-  mt = fmaxf(mt, *x_other);
+#pragma unroll
+  for (int q = 0; q < kParts; ++q) mt = fmaxf(mt, x_quarter[q * 32 + lane]);
   const float m_new = fmaxf(m_used, mt * c);
   const float sc = ex2(m_used - m_new);
   float sum = 0.f;
 #pragma unroll 1
-  for (int cc = 0; cc < 2; ++cc) {
+  for (int cc = 0; cc < kChunks; ++cc) {
     float x[32];
     uint32_t pk[16];
     tc_ld32(s_addr + cc * 32, x);
@@ -358,7 +366,7 @@ __device__ __noinline__ Redo redo_half(uint32_t s_addr, uint32_t o_addr, int val
     if (!mbar_wait_warp(pv_bar, pv_parity, abort_flag, status)) return {-1.f, m_new};
     tc_fence_after();
 #pragma unroll 1
-    for (int cc = 0; cc < 2; ++cc) {
+    for (int cc = 0; cc < kChunks; ++cc) {
       float o[32];
       tc_ld32(o_addr + cc * 32, o);
       tc_wait_ld();
@@ -394,8 +402,8 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                  const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmKc,
                  const __grid_constant__ CUtensorMap tmVc, const Params prm) {
   extern __shared__ uint8_t smem_raw[];
-  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  uint8_t *base_ptr = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t base = smem_u32(smem_raw);
+  uint8_t *base_ptr = smem_raw;
   const uint32_t bars = base + kOffBar;
   volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(base_ptr + kOffBar + 192);
   volatile int *abort_flag = reinterpret_cast<volatile int *>(base_ptr + kOffBar + 196);
@@ -422,6 +430,10 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   };
   int *status = lv.status;
   if (*reinterpret_cast<volatile int *>(status) != 0) return;   // an earlier CTA gave up: do not pile on
+  if (base & 1023u) {                                            // swizzled tiles need the alignment: report, do not fault
+    if (tid == 0) atomicExch(status, kDevCheck);
+    return;
+  }
 
   if (tid == 0) {
     *abort_flag = 0;
@@ -432,10 +444,10 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     }
     for (int s = 0; s < 2; ++s) {
       mbar_init(bar(bSFull + s), 1);
-      mbar_init(bar(bPFull + s), 256);
+      mbar_init(bar(bPFull + s), 128 * kParts);
       mbar_init(bar(bPvDone + s), 1);
     }
-    for (int s = 0; s < 4; ++s) mbar_init(bar(bPair + s), 64);
+    for (int s = 0; s < 4; ++s) mbar_init(bar(bPair + s), 32 * kParts);
     for (int s = 0; s < 2; ++s) mbar_init(bar(bFinal + s), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -591,18 +603,23 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   }
   } else {
     // ------------------------------------------------------------------ softmax + epilogue
-    const int half = (warp - 4) >> 2;            // 0: columns 0-63, 1: columns 64-127 of every S tile
+    const int part = (warp - 4) >> 2;            // which kCols columns of every S tile
     const int quarter = warp & 3;                // the TMEM lane quarter this warp may access
     const int row = quarter * 32 + lane;
     const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
     const float c = prm.scale_log2e;
     const uint64_t c2 = pack2(c, c);
-    volatile int *xflag = reinterpret_cast<volatile int *>(base_ptr + kOffX);           // [2][4][2]
-    volatile float *xval = reinterpret_cast<volatile float *>(base_ptr + kOffX + 64);   // [4][2][32]
-    volatile float *x_mine = xval + (quarter * 2 + half) * 32 + lane;
-    volatile float *x_other = xval + (quarter * 2 + (half ^ 1)) * 32 + lane;
+    volatile int *xflag = reinterpret_cast<volatile int *>(base_ptr + kOffX);                            // [2][4][kParts]
+    volatile float *x_quarter = reinterpret_cast<volatile float *>(base_ptr + kOffX + 128) + quarter * kParts * 32;   // [kParts][32]
     const uint32_t pair_bar = bar(bPair + quarter);
-    uint32_t pair_uses = 0;                      // rendezvous so far of this quarter's two warps (same in both)
+    uint32_t pair_uses = 0;                      // rendezvous so far of this quarter's warps (same in all of them)
+    // rendezvous of the kParts warps of this quarter; false when a wait gave up
+    auto meet = [&]() -> bool {
+      mbar_arrive(pair_bar);
+      const bool r = mbar_wait_warp(pair_bar, pair_uses & 1u, abort_flag, status);
+      ++pair_uses;
+      return r;
+    };
     const int ntile = single ? 1 : 2;
     float m_used[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f};
     // window rows of this thread (rank in the window, or -1) and whether its warp has any
@@ -627,26 +644,26 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         ok = mbar_wait_warp(bar(bSFull + buf), par, abort_flag, status);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t s_addr = lane_addr + kColS + buf * 128 + half * 64;
-        const int valid = tile_valid(j) - half * 64;   // < 64 only in a ragged tile; may be <= 0
-        float v[2][32];
+        const uint32_t s_addr = lane_addr + kColS + buf * 128 + part * kCols;
+        const int valid = tile_valid(j) - part * kCols;   // < kCols only in a ragged tile; may be <= 0
+        float v[kChunks > 1 ? 2 : 1][32];
         tc_ld32(s_addr, v[0]);
         // one sweep: x = s * c - m, p = exp2(x), partial row sum; the bf16 pairs of p stay in registers
-        // until both halves know that no exponent left the lazy band.  (64 values of at most 2^8 sum to
-        // at most 2^14; a larger, infinite or NaN sum means that some x exceeded 8 - or that there is no
-        // reference yet, m = -inf in the first tile.)
+        // until all parts know that no exponent left the lazy band.  (kCols values of at most 2^8 sum to
+        // at most 2^8 kCols; a larger, infinite or NaN sum means that some x exceeded 8 - or that there
+        // is no reference yet, m = -inf in the first tile.)
         const uint64_t negm2 = pack2(-m_used[qt], -m_used[qt]);
         uint64_t sum2a = pack2(0.f, 0.f), sum2b = sum2a;
-        uint32_t pk[32];
+        uint32_t pk[kCols / 2];
 #pragma unroll
-        for (int cc = 0; cc < 2; ++cc) {
+        for (int cc = 0; cc < kChunks; ++cc) {
           tc_wait_ld();
-          if (cc < 1) tc_ld32(s_addr + (cc + 1) * 32, v[(cc + 1) & 1]);
+          if (cc + 1 < kChunks) tc_ld32(s_addr + (cc + 1) * 32, v[(cc + 1) & 1]);
           float *x = v[cc & 1];
           if (wwarp[qt]) {
             if (wrank[qt] >= 0) {
               // slot of this chunk's first column: history tiles start at 128 j, current-map tiles behind the history
-              const int slot0 = (j < Th ? j * 128 : hist + (j - Th) * 128) + half * 64 + cc * 32;
+              const int slot0 = (j < Th ? j * 128 : hist + (j - Th) * 128) + part * kCols + cc * 32;
               float *dst = prm.win_logits + ((size_t)slice * prm.w + wrank[qt]) * prm.ld_l + slot0;
 #pragma unroll
               for (int i = 0; i < 32; ++i)
@@ -654,7 +671,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             }
             __syncwarp();   // the tcgen05 instructions that follow want the warp converged
           }
-          if (valid < 64) {
+          if (valid < kCols) {
 #pragma unroll
             for (int i = 0; i < 32; ++i)
               if (cc * 32 + i >= valid) x[i] = -INFINITY;
@@ -685,25 +702,26 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         unpack2(sum2a, s0, s1);
         unpack2(sum2b, s2, s3);
         const float lt = (s0 + s1) + (s2 + s3);
-        // the two warps of the quarter tell each other whether one of their rows needs the rare path
-        const int mine = __any_sync(0xffffffffu, !(lt <= 16384.f)) ? 1 : 0;
+        // the warps of the quarter tell each other whether one of their rows needs the rare path
+        int mine = __any_sync(0xffffffffu, !(lt <= 256.f * (float)kCols)) ? 1 : 0;
         const int slot = (int)(pair_uses & 1u);
-        if (lane == 0) xflag[(slot * 4 + quarter) * 2 + half] = mine;
-        mbar_arrive(pair_bar);
-        ok = mbar_wait_warp(pair_bar, pair_uses & 1u, abort_flag, status);
-        ++pair_uses;
+        if (lane == 0) xflag[(slot * 4 + quarter) * kParts + part] = mine;
+        ok = meet();
         if (!ok) break;
-        if (mine | xflag[(slot * 4 + quarter) * 2 + (half ^ 1)]) {
-          const Redo r = redo_half(s_addr, lane_addr + kColO + qt * 128 + half * 64, valid, c, m_used[qt], j > 0, bar(bPvDone + qt),
-                                   (j - 1) & 1, pair_bar, pair_uses & 1u, x_mine, x_other, abort_flag, status);
+#pragma unroll
+        for (int q = 0; q < kParts; ++q) mine |= xflag[(slot * 4 + quarter) * kParts + q];
+        if (mine) {
+          const Redo r = redo_part(s_addr, lane_addr + kColO + qt * 128 + part * kCols, valid, c, m_used[qt], j > 0,
+                                   bar(bPvDone + qt), (j - 1) & 1, pair_bar, pair_uses & 1u, x_quarter, part, lane, abort_flag,
+                                   status);
           ++pair_uses;
           ok = __all_sync(0xffffffffu, r.sum >= 0.f);
           if (!ok) break;
           l[qt] = l[qt] * ex2(m_used[qt] - r.m) + r.sum;
           m_used[qt] = r.m;
         } else {
-          tc_st16(s_addr, pk);
-          tc_st16(s_addr + 16, pk + 16);
+#pragma unroll
+          for (int cc = 0; cc < kChunks; ++cc) tc_st16(s_addr + cc * 16, pk + cc * 16);
           l[qt] += lt;
         }
         tc_wait_st();
@@ -711,12 +729,8 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         mbar_arrive(bar(bPFull + buf));
       }
     }
-    if (ok) {
-      // a rendezvous of its own orders the partner's last read of the exchange area before its reuse
-      mbar_arrive(pair_bar);
-      ok = mbar_wait_warp(pair_bar, pair_uses & 1u, abort_flag, status);
-      ++pair_uses;
-    }
+    // a rendezvous of its own orders the other warps' last read of the exchange area before its reuse
+    if (ok) ok = meet();
 #pragma unroll
     for (int qt = 0; qt < 2; ++qt) {
       if (qt >= ntile || !ok) break;
@@ -725,24 +739,22 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       ok = mbar_wait_warp(bar(bFinal + qt), 0, abort_flag, status);
       if (!ok) break;
       tc_fence_after();
-      // the row sum is the sum of the two halves' partial sums
-      *x_mine = l[qt];
-      mbar_arrive(pair_bar);
-      ok = mbar_wait_warp(pair_bar, pair_uses & 1u, abort_flag, status);
-      ++pair_uses;
+      // the row sum is the sum of the parts' partial sums
+      x_quarter[part * 32 + lane] = l[qt];
+      ok = meet();
       if (!ok) break;
-      const float lsum = l[qt] + *x_other;
-      mbar_arrive(pair_bar);                     // second rendezvous: the partner has read before x_mine is reused
-      ok = mbar_wait_warp(pair_bar, pair_uses & 1u, abort_flag, status);
-      ++pair_uses;
+      float lsum = 0.f;
+#pragma unroll
+      for (int q = 0; q < kParts; ++q) lsum += x_quarter[q * 32 + lane];
+      ok = meet();                               // every warp has read before the area is reused
       if (!ok) break;
       const float inv = 1.f / lsum;
       const int qi = q_first + qt * 128 + row;
-      __nv_bfloat16 *orow = const_cast<__nv_bfloat16 *>(row_ptr<__nv_bfloat16>(prm.O, b, h, qi < n_k ? qi : 0)) + half * 64;
+      __nv_bfloat16 *orow = const_cast<__nv_bfloat16 *>(row_ptr<__nv_bfloat16>(prm.O, b, h, qi < n_k ? qi : 0)) + part * kCols;
 #pragma unroll
-      for (int cc = 0; cc < 2; ++cc) {
+      for (int cc = 0; cc < kChunks; ++cc) {
         float o[32];
-        tc_ld32(lane_addr + kColO + qt * 128 + half * 64 + cc * 32, o);
+        tc_ld32(lane_addr + kColO + qt * 128 + part * kCols + cc * 32, o);
         tc_wait_ld();
         if (qi < n_k) {
 #pragma unroll
@@ -756,9 +768,9 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           }
         }
       }
-      if (prm.lse != nullptr && half == 0 && qi < n_k)
+      if (prm.lse != nullptr && part == 0 && qi < n_k)
         prm.lse[(size_t)slice * n_k + qi] = (m_used[qt] + log2f(lsum)) * 0.6931471805599453f;
-      if (wrank[qt] >= 0 && half == 0) prm.win_lse[(size_t)slice * prm.w + wrank[qt]] = m_used[qt] + log2f(lsum);
+      if (wrank[qt] >= 0 && part == 0) prm.win_lse[(size_t)slice * prm.w + wrank[qt]] = m_used[qt] + log2f(lsum);
     }
     tc_fence_before();
   }

@@ -269,3 +269,40 @@ def test_full_size_pass_sampled_slices():
                     lambda k: orc.window_centroids(wl.sides[k], wl.sides[k], 16), slices, check_lse=False).run()
     assert run.evictions > 0
     kv.close()
+
+
+def test_8b_class_shape_full_cache_and_budget_sampled_slices():
+    """configs[3] (B 8, H 32, 13 scales): slices are independent, so two of the 40 layers stand for the
+    pass - one with the full cache, one at the refiner budget; the oracle follows two slices of each."""
+    wl8 = synth.WORKLOADS["pass8b"]
+    wl = synth.Workload("pass8b-2", 2, wl8.batch, wl8.n_heads, 128, "bf16", wl8.sides, seed=wl8.seed, n_drafters=1)
+    n = wl.n_tokens
+    br = orc.budget_tokens(0.03, n)
+    budgets = [[binding.KEEP_ALL] * wl.n_scales, [br] * wl.n_scales]
+    kv = binding.ScaleKV(2, wl.batch, wl.n_heads, 128, "bf16", wl.sides, wl.sides, budgets, max_window=16)
+    slices = [(0, 0, 0), (0, 7, 31), (1, 3, 17), (1, 6, 2)]
+    run = ParityRun(kv, "bf16", wl.sides, budgets, lambda l, k: synth.scale_inputs(wl, l, k, device="cuda"),
+                    lambda k: orc.window_centroids(wl.sides[k], wl.sides[k], 16), slices, check_lse=False,
+                    max_rows=1024).run()
+    assert run.evictions > 0
+    assert kv.scalekv_lengths(0)[7][31] == sum(n)
+    kv.close()
+
+
+def test_hires_16_scales_sampled_slices():
+    """configs[4] (B 4, H 16, 16 scales up to 128 x 128): one drafter and one refiner layer at the 10 %
+    point of the sweep; attention compared on evenly spaced query rows of the large maps."""
+    wlh = synth.WORKLOADS["hires"]
+    wl = synth.Workload("hires-2", 2, wlh.batch, wlh.n_heads, 128, "bf16", wlh.sides, seed=wlh.seed, n_drafters=1)
+    n = wl.n_tokens
+    refiner_pct = 0.10 / 3.25
+    bd, br = orc.budget_tokens(round(10 * refiner_pct, 6), n), orc.budget_tokens(round(refiner_pct, 6), n)
+    planted = synth.drafter_layers(wl)
+    budgets = [[bd if l in planted else br] * wl.n_scales for l in range(2)]
+    kv = binding.ScaleKV(2, wl.batch, wl.n_heads, 128, "bf16", wl.sides, wl.sides, budgets, max_window=16)
+    slices = [(0, 0, 0), (1, 3, 15)]
+    run = ParityRun(kv, "bf16", wl.sides, budgets, lambda l, k: synth.scale_inputs(wl, l, k, device="cuda"),
+                    lambda k: orc.window_centroids(wl.sides[k], wl.sides[k], 16), slices, check_lse=False,
+                    max_rows=512).run()
+    assert run.evictions > 0
+    kv.close()
