@@ -216,6 +216,31 @@ def run_reference(args):
 
 
 # --------------------------------------------------------------------------------------------
+# Multi-rank plumbing (no data-path collective: every rank owns its own batch of images)
+# --------------------------------------------------------------------------------------------
+def rank_workload(wl, rank, world):
+    """The workload of one rank: same shapes, its own seed, so that every rank owns a different batch."""
+    return dataclasses.replace(wl, seed=wl.seed + 1000 * rank) if world > 1 else wl
+
+
+def max_over_ranks(x, world, device="cpu"):
+    """Slowest rank's time: the job is done when the last rank is."""
+    if world <= 1:
+        return float(x)
+    import torch
+    import torch.distributed as dist
+
+    t = torch.tensor([float(x)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_throughput(n_scales, steps, world, ms_max):
+    """Whole-job scale-steps per second: all ranks' scale-steps over the slowest rank's time."""
+    return n_scales * steps * world / (ms_max / 1000.0)
+
+
+# --------------------------------------------------------------------------------------------
 # CUDA arm
 # --------------------------------------------------------------------------------------------
 def run_scalekv(args):
@@ -233,8 +258,7 @@ def run_scalekv(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     wl = workload_from_args(args)
-    if world > 1:
-        wl = dataclasses.replace(wl, seed=wl.seed + 1000 * rank)      # every rank owns a different batch
+    wl = rank_workload(wl, rank, world)
     peaks = load_peaks()
     windows = pipeline.windows_for(wl.sides, wl.window)
 
@@ -298,11 +322,8 @@ def run_scalekv(args):
     ms_events = timed_passes(args.steps)
     prof_timed = kv.scalekv_profile_read()
     clocks = sampler.stop()
-    if world > 1:
-        t = torch.tensor([ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    value = wl.n_scales * args.steps * world / (ms / 1000.0)
+    ms = max_over_ranks(ms, world, "cuda")
+    value = job_throughput(wl.n_scales, args.steps, world, ms)
 
     # the same passes once more with compress serialised onto stream_main: every kernel timed alone
     kv.scalekv_profile_enable(2)
@@ -368,10 +389,7 @@ def run_scalekv(args):
             e2e_pass()
         barrier()
         e2e_s = time.perf_counter() - t0
-        if world > 1:
-            t = torch.tensor([e2e_s], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_s = float(t.item())
+        e2e_s = max_over_ranks(e2e_s, world, "cuda")
         esz = 2 if wl.dtype == "bf16" else 4
         tok_bytes = sum(wl.n_tokens) * wl.batch * wl.n_heads * wl.head_dim * esz * wl.n_layers
         e2e = {"value": wl.n_scales * e2e_steps * world / e2e_s, "unit": UNIT, "h2d_bytes_per_step": 3 * tok_bytes,
