@@ -335,7 +335,7 @@ def run_scalekv(args):
     att_tflops = work["attend_flop"] * args.steps / (att_ms / 1000.0) / 1e12 if att_ms > 0 else 0.0
     peak_tf = peaks["bf16_sustained"] if wl.dtype == "bf16" else None
     kernels = {}
-    for name, key in (("append", "append_bytes"), ("score_logits", "score_bytes"), ("score_select", "select_bytes"),
+    for name, key in (("append", "append_bytes"), ("score", "score_bytes"), ("select", "select_bytes"),
                       ("compact", "compact_bytes")):
         kms, kn = prof_alone[name]
         if kn == 0:

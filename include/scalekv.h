@@ -209,7 +209,7 @@ scalekv_status scalekv_launch_count(scalekv_ctx *ctx, int64_t *count);
  * it runs on (durations of kernels on the two streams may overlap and then include contention).
  * on = 2: compress runs on stream_main as well, so that no two kernels overlap and each duration
  * is the kernel's own.  on = 0: off.  scalekv_profile_read waits for both streams and returns, for
- * class `which` (0 append, 1 attend, 2 score logits, 3 score + select, 4 compact, 5 other), the
+ * class `which` (0 append, 1 attend, 2 score, 3 select, 4 compact, 5 other), the
  * summed milliseconds and the number of launches since profiling was last enabled. */
 scalekv_status scalekv_profile_enable(scalekv_ctx *ctx, int32_t on);
 scalekv_status scalekv_profile_read(scalekv_ctx *ctx, int32_t which, double *ms_total, int64_t *launches);

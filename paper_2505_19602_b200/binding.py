@@ -21,7 +21,7 @@ KEEP_ALL = -1
 MAX_WINDOW = 64
 BF16, F32 = 0, 1
 STATUS_NAMES = ["OK", "INVALID_ARG", "BAD_STATE", "CAPACITY", "UNSUPPORTED", "CUDA", "TIMEOUT", "DEVICE_CHECK"]
-KERNEL_CLASSES = ["append", "attend", "score_logits", "score_select", "compact", "other"]
+KERNEL_CLASSES = ["append", "attend", "score", "select", "compact", "other"]
 
 
 class ScaleKVError(RuntimeError):

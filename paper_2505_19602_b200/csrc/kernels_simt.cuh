@@ -312,18 +312,12 @@ __device__ __forceinline__ float block_reduce_sum(float v, float *red) {
 }
 
 // ------------------------------------------------------------------------------------------
-// score, step 2, aggregation and selection in one kernel, one CTA of 1024 threads per slice
-// (Sec. 3.3, Eq. 5 and the selection paragraph).  Input: base-2 logits y[w][L] of the window rows
-// and, when attend recorded them, the rows' base-2 log-sum-exp lse[w] (then the logits are read once).
-//   1. (without lse) per window row j: m_j = max_i y_ji, Z_j = sum_i 2^(y_ji - m_j), lse_j = m_j + log2 Z_j
-//   2. s_i = (1/w) sum_j 2^(y_ji - lse_j)  -> scores (global, for inspection) and, as the bit
-//      pattern of the non-negative float, the radix key of entry i in shared memory; window entries
-//      get a sentinel and never take part in the selection
-//   3. radix select of the k'-th largest key, 8 bits per pass, warp-aggregated histogram updates
-//   4. ordered emit of the ascending slot list of survivors (selected U window); ties at the
-//      threshold go to the lowest slots = lowest original positions.  Every thread owns a run of
-//      consecutive entries, so two block scans order the whole list.  Deterministic.
-// Dynamic shared memory: 4 * ld_s bytes of keys.
+// score, step 2 (Sec. 3.3, Eq. 5): from the base-2 logits y[w][L] of the window rows to the importance
+// s_i = (1/w) sum_j 2^(y_ji - lse_j), lse_j the base-2 log-sum-exp of row j (recorded by attend, or
+// computed by row_lse_kernel).  Streaming and embarrassingly parallel: grid (ceil(L_max / 256),
+// n_slices), one entry per thread, the w loads of a thread independent and coalesced across the warp.
+// Besides the score (kept for inspection) it writes the entry's radix key: the bit pattern of the
+// non-negative float, or a sentinel for window entries, which never take part in the selection.
 // ------------------------------------------------------------------------------------------
 constexpr uint32_t kWindowKey = 0xFFFFFFFFu;
 
@@ -353,92 +347,123 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int *warp_sums, int *
   return warp_sums[wid] + incl - v;
 }
 
-__global__ void __launch_bounds__(1024) score_select_kernel(LayerView lv, WindowArg wa, int budget, const float *logits,
-                                                            const float *lse_in, int ld_l, float *scores, int ld_s,
-                                                            int *keep_list, int *kept_count) {
-  extern __shared__ uint32_t key[];            // [L]
-  __shared__ float part[32][16];               // per-warp partial maxima / sums of 16 rows
-  __shared__ float m_row[kMaxWindow], lse_row[kMaxWindow];
-  __shared__ int hist[256];
-  __shared__ int warp_sums[33];
-  __shared__ uint32_t sh_prefix;
-  __shared__ int sh_remaining;
+__global__ void __launch_bounds__(256) score_kernel(LayerView lv, WindowArg wa, const float *logits, const float *lse,
+                                                    int ld_l, float *scores, uint32_t *keys, int ld_s) {
+  __shared__ float lse_row[kMaxWindow];
+  const int slice = blockIdx.y;
+  const int L = lv.hist_len[slice] + wa.n_k;
+  const int i = blockIdx.x * 256 + threadIdx.x;
+  if (blockIdx.x * 256 >= L) return;
+  const int w = wa.w;
+  if (threadIdx.x < w) lse_row[threadIdx.x] = lse[(size_t)slice * w + threadIdx.x];
+  __syncthreads();
+  if (i >= L) return;
+  const float *y = logits + (size_t)slice * w * ld_l + i;
+  float sc = 0.f;
+  int j = 0;
+  for (; j + 8 <= w; j += 8) {
+    float t[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) t[e] = __ldg(y + (size_t)(j + e) * ld_l);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) sc += exp2f(t[e] - lse_row[j + e]);
+  }
+  for (; j < w; ++j) sc += exp2f(__ldg(y + (size_t)j * ld_l) - lse_row[j]);
+  sc *= 1.f / (float)w;
+  scores[(size_t)slice * ld_s + i] = sc;
+  const bool win = is_window_pos(wa, lv.pos_pool[slot_row(lv, slice, i)]);
+  keys[(size_t)slice * ld_s + i] = win ? kWindowKey : (__float_as_uint(sc) & 0x7FFFFFFFu);
+}
+
+// Base-2 log-sum-exp of every window row of y[w][L] when attend did not record it: one CTA of 1024
+// threads per slice, 16 rows per round, a maximum sweep and a sum sweep.  lse is [n_slices][w].
+__global__ void __launch_bounds__(1024) row_lse_kernel(LayerView lv, WindowArg wa, const float *logits, int ld_l, float *lse) {
+  __shared__ float part[32][16];
+  __shared__ float m_row[16];
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const int slice = blockIdx.x;
   const int L = lv.hist_len[slice] + wa.n_k;
   const int w = wa.w;
   const float *y = logits + (size_t)slice * w * ld_l;
+  for (int g0 = 0; g0 < w; g0 += 16) {
+    const int nr = w - g0 < 16 ? w - g0 : 16;
+    float acc[16];
+#pragma unroll
+    for (int r = 0; r < 16; ++r) acc[r] = -INFINITY;
+    for (int i = tid; i < L; i += 1024) {
+#pragma unroll
+      for (int r = 0; r < 16; ++r)
+        if (r < nr) acc[r] = fmaxf(acc[r], y[(size_t)(g0 + r) * ld_l + i]);
+    }
+#pragma unroll
+    for (int r = 0; r < 16; ++r) {
+      float v = acc[r];
+      for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+      if (lane == 0) part[wid][r] = v;
+    }
+    __syncthreads();
+    if (tid < 16) {
+      float v = part[0][tid];
+      for (int k = 1; k < 32; ++k) v = fmaxf(v, part[k][tid]);
+      m_row[tid] = v;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int r = 0; r < 16; ++r) acc[r] = 0.f;
+    for (int i = tid; i < L; i += 1024) {
+#pragma unroll
+      for (int r = 0; r < 16; ++r)
+        if (r < nr) acc[r] += exp2f(y[(size_t)(g0 + r) * ld_l + i] - m_row[r]);
+    }
+#pragma unroll
+    for (int r = 0; r < 16; ++r) {
+      float v = acc[r];
+      for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+      if (lane == 0) part[wid][r] = v;
+    }
+    __syncthreads();
+    if (tid < 16) {
+      float v = 0.f;
+      for (int k = 0; k < 32; ++k) v += part[k][tid];     // fixed order: deterministic
+      if (tid < nr) lse[(size_t)slice * w + g0 + tid] = m_row[tid] + log2f(v);
+    }
+    __syncthreads();
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// select: per-slice top-k' of the non-window entries by key (Sec. 3.3), one CTA of 1024 threads per
+// slice with the slice's keys in shared memory:
+//   radix select of the k'-th largest key, 8 bits per pass, warp-aggregated histogram updates; then
+//   the ordered emit of the ascending slot list of survivors (selected U window); ties at the
+//   threshold go to the lowest slots = lowest original positions.  Every thread owns a run of
+//   consecutive entries, so two block scans order the whole list.  Deterministic.
+// Dynamic shared memory: 4 * ld_s bytes of keys.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(1024) select_kernel(LayerView lv, WindowArg wa, int budget, const uint32_t *keys, int ld_s,
+                                                      int *keep_list, int *kept_count) {
+  extern __shared__ uint32_t key[];            // [L]
+  __shared__ int hist[256];
+  __shared__ int warp_sums[33];
+  __shared__ uint32_t sh_prefix;
+  __shared__ int sh_remaining;
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int slice = blockIdx.x;
+  const int L = lv.hist_len[slice] + wa.n_k;
   int *out = keep_list + (size_t)slice * ld_s;
 
-  if (lse_in != nullptr) {
-    if (tid < w) lse_row[tid] = lse_in[(size_t)slice * w + tid];
-    __syncthreads();
-  } else {
-    // 1. row maxima and normalisers, 16 rows per round
-    for (int g0 = 0; g0 < w; g0 += 16) {
-      const int nr = w - g0 < 16 ? w - g0 : 16;
-      float acc[16];
-#pragma unroll
-      for (int r = 0; r < 16; ++r) acc[r] = -INFINITY;
-      for (int i = tid; i < L; i += 1024) {
-#pragma unroll
-        for (int r = 0; r < 16; ++r)
-          if (r < nr) acc[r] = fmaxf(acc[r], y[(size_t)(g0 + r) * ld_l + i]);
-      }
-#pragma unroll
-      for (int r = 0; r < 16; ++r) {
-        float v = acc[r];
-        for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
-        if (lane == 0) part[wid][r] = v;
-      }
-      __syncthreads();
-      if (tid < 16) {
-        float v = part[0][tid];
-        for (int k = 1; k < 32; ++k) v = fmaxf(v, part[k][tid]);
-        if (tid < nr) m_row[g0 + tid] = v;
-      }
-      __syncthreads();
-#pragma unroll
-      for (int r = 0; r < 16; ++r) acc[r] = 0.f;
-      for (int i = tid; i < L; i += 1024) {
-#pragma unroll
-        for (int r = 0; r < 16; ++r)
-          if (r < nr) acc[r] += exp2f(y[(size_t)(g0 + r) * ld_l + i] - m_row[g0 + r]);
-      }
-#pragma unroll
-      for (int r = 0; r < 16; ++r) {
-        float v = acc[r];
-        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-        if (lane == 0) part[wid][r] = v;
-      }
-      __syncthreads();
-      if (tid < 16) {
-        float v = 0.f;
-        for (int k = 0; k < 32; ++k) v += part[k][tid];     // fixed order: deterministic
-        if (tid < nr) lse_row[g0 + tid] = m_row[g0 + tid] + log2f(v);
-      }
-      __syncthreads();
-    }
-  }
-
-  // 2. scores and keys
-  const float inv_w = 1.f / (float)w;
   int n_win_local = 0;
   for (int i = tid; i < L; i += 1024) {
-    float sc = 0.f;
-    for (int j = 0; j < w; ++j) sc += exp2f(y[(size_t)j * ld_l + i] - lse_row[j]);
-    sc *= inv_w;
-    scores[(size_t)slice * ld_s + i] = sc;
-    const bool win = is_window_pos(wa, lv.pos_pool[slot_row(lv, slice, i)]);
-    key[i] = win ? kWindowKey : (__float_as_uint(sc) & 0x7FFFFFFFu);
-    n_win_local += win ? 1 : 0;
+    const uint32_t k = __ldg(keys + (size_t)slice * ld_s + i);
+    key[i] = k;
+    n_win_local += (k == kWindowKey) ? 1 : 0;
   }
   int n_win;
   block_exclusive_scan(n_win_local, warp_sums, &n_win);
   const int cand = L - n_win;
   const int kprime = (budget < 0 || budget > cand) ? cand : budget;
 
-  // 3. radix select of the kprime-th largest key
+  // radix select of the kprime-th largest key
   uint32_t threshold = 0;
   int n_ties_taken = 0;       // how many entries equal to the threshold are kept
   if (kprime > 0 && kprime < cand) {
@@ -492,7 +517,7 @@ __global__ void __launch_bounds__(1024) score_select_kernel(LayerView lv, Window
   const bool keep_all = (kprime >= cand);
   const bool keep_none = (kprime == 0);
 
-  // 4. ordered emit: thread t owns entries [t * E, (t + 1) * E)
+  // ordered emit: thread t owns entries [t * E, (t + 1) * E)
   const int E = (L + 1023) >> 10;
   const int i_lo = tid * E, i_hi = (i_lo + E < L) ? i_lo + E : L;
   int n_tie = 0;

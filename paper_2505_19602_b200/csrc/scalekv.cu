@@ -408,7 +408,7 @@ scalekv_status scalekv_init(const scalekv_config *cfg, scalekv_ctx **out) {
     set_smem(score_logits_kernel<float, 64>, 2 * 64 * 68 * 4);
     set_smem(layer_stats_kernel<float, 64>, (size_t)(64 + p.ld_s) * 4);
   }
-  set_smem(score_select_kernel, (size_t)p.ld_s * 4);
+  set_smem(select_kernel, (size_t)p.ld_s * 4);
   set_smem(compact_kernel, (size_t)(p.ld_s + (p.ld_s + p.P - 1) / p.P + 1) * 4);
   cudaGetLastError();
   std::string tc_err;
@@ -591,12 +591,19 @@ scalekv_status scalekv_compress(scalekv_ctx *ctx, int32_t layer, scalekv_tensor 
                                                                          ctx->scale);
     }
     ctx->logits_of[layer] = -1;
+    float *wlse = reinterpret_cast<float *>(ctx->ws + p.off_wlse) + (size_t)(layer & 1) * p.n_slices * p.max_window;
+    uint32_t *keys = reinterpret_cast<uint32_t *>(ctx->ws + p.off_keys);
+    if (!recorded) {
+      Scope sc(ctx, s, kScore);
+      row_lse_kernel<<<p.n_slices, 1024, 0, s>>>(lv, wa, logits, p.ld_s, wlse);
+    }
+    {
+      Scope sc(ctx, s, kScore);
+      score_kernel<<<dim3((L + 255) / 256, p.n_slices), 256, 0, s>>>(lv, wa, logits, wlse, p.ld_s, scores, keys, p.ld_s);
+    }
     {
       Scope sc(ctx, s, kSelect);
-      const float *wlse = recorded ? reinterpret_cast<float *>(ctx->ws + p.off_wlse) + (size_t)(layer & 1) * p.n_slices * p.max_window
-                                   : nullptr;
-      score_select_kernel<<<p.n_slices, 1024, (size_t)p.ld_s * 4, s>>>(lv, wa, budget, logits, wlse, p.ld_s, scores, p.ld_s, keep,
-                                                                       kept);
+      select_kernel<<<p.n_slices, 1024, (size_t)p.ld_s * 4, s>>>(lv, wa, budget, keys, p.ld_s, keep, kept);
     }
     {
       Scope sc(ctx, s, kCompact);

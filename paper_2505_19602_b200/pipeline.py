@@ -104,11 +104,11 @@ def pass_work(wl: synth.Workload, budgets, windows):
     attend_min_bytes  what attend must move: K and V of the L entries once, Q and O, plus - since it also
                       appends - the write of the current map's K/V rows and positions into the pages, and
                       the write of the w x L window logits.
-    select_bytes      the score + select kernel: w x L logits and L positions in, L scores and the keep
-                      list out.
+    score_bytes       the score kernel: w x L logits and L positions in, L scores and L keys out (plus K read
+                      by the stand-alone logits kernel when attend did not record the logits).
+    select_bytes      the select kernel: L keys in, the keep list out.
     compact_bytes     K and V rows (and positions) of the survivors, read and written (upper bound: which
                       rows already sit in place is unknown on the host).
-    score_bytes       K read by the stand-alone logits kernel; zero when attend recorded the logits.
     """
     n = wl.n_tokens
     d = wl.head_dim
@@ -139,7 +139,8 @@ def pass_work(wl: synth.Workload, budgets, windows):
             if b != binding.KEEP_ALL and b < cand:
                 if not fused:
                     out["score_bytes"] += L * d * esz * slices
-                out["select_bytes"] += (4 * w * L + 4 * L + 4 * L + 4 * (b + w)) * slices
+                out["score_bytes"] += (4 * w * L + 4 * L + 4 * L + 4 * L) * slices
+                out["select_bytes"] += (4 * L + 4 * (b + w)) * slices
                 out["compact_bytes"] += (b + w) * (2 * 2 * d * esz + 8) * slices
                 hist = b + w
             else:
