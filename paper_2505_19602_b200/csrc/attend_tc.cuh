@@ -51,8 +51,8 @@ constexpr uint32_t kHalfBytes = kTileBytes / 2;  // 64 head-dim columns = one 12
 constexpr uint32_t kOffQ = 0;                    // two query tiles (the dynamic shared memory must start 1024-byte aligned)
 constexpr uint32_t kOffRing = kOffQ + 2 * kTileBytes;
 constexpr uint32_t kOffBar = kOffRing + kStages * kTileBytes;
-constexpr uint32_t kOffX = kOffBar + 256;        // exchange area of the softmax warps of a quarter: flags [2][4][kParts], values [4][kParts][32]
-constexpr uint32_t kSmemBytes = kOffX + 128 + 4 * kParts * 32 * 4;
+constexpr uint32_t kOffX = kOffBar + 256;        // exchange area of the softmax warps of a quarter: flags [2][4][kParts], values [2][4][kParts][32]
+constexpr uint32_t kSmemBytes = kOffX + 128 + 2 * 4 * kParts * 32 * 4;
 static_assert(kSmemBytes <= 232448, "more shared memory than a CTA can have");
 // barrier slots (8 bytes each): one full/empty pair per ring stage, one S/P/PV barrier per S buffer or query tile
 enum { bQFull = 0, bFull = 1, bEmpty = bFull + kStages, bSFull = bEmpty + kStages, bPFull = bSFull + 2, bPvDone = bPFull + 2,
@@ -316,8 +316,8 @@ __host__ __device__ constexpr uint32_t instr_desc(bool b_mn_major) {
 }
 
 // Rare path of the softmax, taken together by the kParts warps that share a quarter's rows when the
-// fast sweep of one of their row parts overflowed the lazy band (always in the first tile, where no
-// reference exists yet).  The S row part is still intact at s_addr: a first sweep finds its maximum,
+// fast sweep of one of their row parts overflowed the lazy band (the first tile, where no reference
+// exists yet, has a path of its own).  The S row part is still intact at s_addr: a first sweep finds its maximum,
 // the parts exchange theirs through shared memory (mine -> x_quarter[part], with one rendezvous on
 // pair_bar), the reference moves up to the row maximum if that is larger, the part's P is recomputed
 // against it and written over the part's first columns (a chunk's columns are only overwritten
@@ -610,7 +610,8 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     const float c = prm.scale_log2e;
     const uint64_t c2 = pack2(c, c);
     volatile int *xflag = reinterpret_cast<volatile int *>(base_ptr + kOffX);                            // [2][4][kParts]
-    volatile float *x_quarter = reinterpret_cast<volatile float *>(base_ptr + kOffX + 128) + quarter * kParts * 32;   // [kParts][32]
+    // values [2][4][kParts][32]: x_quarter points at [0][quarter]; the second block is only used by the epilogue
+    volatile float *x_quarter = reinterpret_cast<volatile float *>(base_ptr + kOffX + 128) + quarter * kParts * 32;
     const uint32_t pair_bar = bar(bPair + quarter);
     uint32_t pair_uses = 0;                      // rendezvous so far of this quarter's warps (same in all of them)
     // rendezvous of the kParts warps of this quarter; false when a wait gave up
@@ -647,11 +648,32 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         const uint32_t s_addr = lane_addr + kColS + buf * 128 + part * kCols;
         const int valid = tile_valid(j) - part * kCols;   // < kCols only in a ragged tile; may be <= 0
         float v[kChunks > 1 ? 2 : 1][32];
+        if (j == 0) {
+          // first tile: no reference yet.  A sweep of its own finds the part's row maximum, the parts
+          // exchange theirs, and the ordinary sweep below then runs against the row maximum.
+          float mt = -INFINITY;
+#pragma unroll
+          for (int cc = 0; cc < kChunks; ++cc) {
+            tc_ld32(s_addr + cc * 32, v[0]);
+            tc_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; i += 2) {
+              const float e0 = (cc * 32 + i < valid) ? v[0][i] : -INFINITY;
+              const float e1 = (cc * 32 + i + 1 < valid) ? v[0][i + 1] : -INFINITY;
+              mt = max3(mt, e0, e1);
+            }
+          }
+          x_quarter[part * 32 + lane] = mt;
+          ok = meet();
+          if (!ok) break;
+#pragma unroll
+          for (int q = 0; q < kParts; ++q) mt = fmaxf(mt, x_quarter[q * 32 + lane]);
+          m_used[qt] = mt * c;
+        }
         tc_ld32(s_addr, v[0]);
         // one sweep: x = s * c - m, p = exp2(x), partial row sum; the bf16 pairs of p stay in registers
         // until all parts know that no exponent left the lazy band.  (kCols values of at most 2^8 sum to
-        // at most 2^8 kCols; a larger, infinite or NaN sum means that some x exceeded 8 - or that there
-        // is no reference yet, m = -inf in the first tile.)
+        // at most 2^8 kCols; a larger, infinite or NaN sum means that some x exceeded 8.)
         const uint64_t negm2 = pack2(-m_used[qt], -m_used[qt]);
         uint64_t sum2a = pack2(0.f, 0.f), sum2b = sum2a;
         uint32_t pk[kCols / 2];
@@ -729,41 +751,42 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         mbar_arrive(bar(bPFull + buf));
       }
     }
-    // a rendezvous of its own orders the other warps' last read of the exchange area before its reuse
+    // the row sums are the sums of the parts' partial sums: one exchange for both tiles (the rendezvous
+    // before it orders the other warps' last read of the exchange area before its reuse)
     if (ok) ok = meet();
+    if (ok) {
+#pragma unroll
+      for (int qt = 0; qt < 2; ++qt) x_quarter[(qt * 4 * kParts + part) * 32 + lane] = l[qt];
+      ok = meet();
+    }
 #pragma unroll
     for (int qt = 0; qt < 2; ++qt) {
       if (qt >= ntile || !ok) break;
+      float lsum = 0.f;
+#pragma unroll
+      for (int q = 0; q < kParts; ++q) lsum += x_quarter[(qt * 4 * kParts + q) * 32 + lane];
       // a barrier that completes exactly once, after the last PV product: the per-tile PV barrier will
       // not do, a parity wait cannot tell phases two apart and this warp may be that far behind it
       ok = mbar_wait_warp(bar(bFinal + qt), 0, abort_flag, status);
       if (!ok) break;
       tc_fence_after();
-      // the row sum is the sum of the parts' partial sums
-      x_quarter[part * 32 + lane] = l[qt];
-      ok = meet();
-      if (!ok) break;
-      float lsum = 0.f;
-#pragma unroll
-      for (int q = 0; q < kParts; ++q) lsum += x_quarter[q * 32 + lane];
-      ok = meet();                               // every warp has read before the area is reused
-      if (!ok) break;
       const float inv = 1.f / lsum;
       const int qi = q_first + qt * 128 + row;
       __nv_bfloat16 *orow = const_cast<__nv_bfloat16 *>(row_ptr<__nv_bfloat16>(prm.O, b, h, qi < n_k ? qi : 0)) + part * kCols;
+      float o[kChunks][32];
 #pragma unroll
-      for (int cc = 0; cc < kChunks; ++cc) {
-        float o[32];
-        tc_ld32(lane_addr + kColO + qt * 128 + part * kCols + cc * 32, o);
-        tc_wait_ld();
-        if (qi < n_k) {
+      for (int cc = 0; cc < kChunks; ++cc) tc_ld32(lane_addr + kColO + qt * 128 + part * kCols + cc * 32, o[cc]);
+      tc_wait_ld();
+      if (qi < n_k) {
+#pragma unroll
+        for (int cc = 0; cc < kChunks; ++cc) {
 #pragma unroll
           for (int v4 = 0; v4 < 4; ++v4) {
             uint4 w;
-            w.x = pack_bf16(o[8 * v4 + 0] * inv, o[8 * v4 + 1] * inv);
-            w.y = pack_bf16(o[8 * v4 + 2] * inv, o[8 * v4 + 3] * inv);
-            w.z = pack_bf16(o[8 * v4 + 4] * inv, o[8 * v4 + 5] * inv);
-            w.w = pack_bf16(o[8 * v4 + 6] * inv, o[8 * v4 + 7] * inv);
+            w.x = pack_bf16(o[cc][8 * v4 + 0] * inv, o[cc][8 * v4 + 1] * inv);
+            w.y = pack_bf16(o[cc][8 * v4 + 2] * inv, o[cc][8 * v4 + 3] * inv);
+            w.z = pack_bf16(o[cc][8 * v4 + 4] * inv, o[cc][8 * v4 + 5] * inv);
+            w.w = pack_bf16(o[cc][8 * v4 + 6] * inv, o[cc][8 * v4 + 7] * inv);
             reinterpret_cast<uint4 *>(orow + cc * 32)[v4] = w;
           }
         }
