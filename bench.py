@@ -27,9 +27,12 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 METRIC = "scale_steps_per_sec"
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the attend kernel from the ncu capture summarised under
-# profiles/ (None while the kernel has changed since the counters were taken)
-ATTEND_TRAFFIC = None
+# DRAM traffic of the attend kernel: (dram__bytes_read.sum + dram__bytes_write.sum) / algorithmic bytes over the two
+# launches of the ncu capture summarised in profiles/attend_tc_kernel_pass2b_1layer.md (1539.1 MB measured against
+# 1676 MB algorithmic: part of the appended rows is still in L2 when a launch ends).  The capture runs one layer of the
+# workload; traffic grows in proportion to the bytes a launch must move, so the roofline object reports this ratio times
+# the average algorithmic bytes per launch.  Set to None when the kernel changes after the capture.
+ATTEND_TRAFFIC_RATIO = 1539.1 / 1676.0
 UNIT = "scale-steps/s"
 
 
@@ -349,7 +352,10 @@ def run_scalekv(args):
                          "TFLOPps_alone": work["attend_flop"] * args.steps / (al_ms / 1000.0) / 1e12 if al_ms > 0 else 0.0,
                          "algorithmic_GB_per_pass": work["attend_min_bytes"] / 1e9}
     roofline = {"bound": "tensor", "kernel": "attend_tc_kernel", "achieved": att_tflops, "peak": peak_tf, "unit": "TFLOP/s",
-                "frac": (att_tflops / peak_tf) if peak_tf else None, "traffic": ATTEND_TRAFFIC,
+                "frac": (att_tflops / peak_tf) if peak_tf else None,
+                "traffic": (ATTEND_TRAFFIC_RATIO * work["attend_min_bytes"] / max(work["attend_launches"], 1)
+                            if ATTEND_TRAFFIC_RATIO and wl.dtype == "bf16" else None),
+                "traffic_unit": "bytes per launch (average launch; ncu capture of one layer scaled by algorithmic bytes)",
                 "peak_source": f"{peaks['source']} bf16 sustained (kernel timed inside a long step)",
                 "avg_launch_ms": att_ms / max(att_n, 1),
                 "flop_per_launch_avg": work["attend_flop"] / max(work["attend_launches"], 1),
