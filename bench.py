@@ -274,8 +274,13 @@ def run_scalekv(args):
         asi, roles = pipeline.calibrate_roles(wl, wl.n_drafters, device=local_rank)
         budgets = pipeline.budget_table(wl, roles)
         planted = synth.drafter_layers(wl)
-        hits = sum(int(roles[l][k]) for k in range(1, wl.n_scales - 1) for l in planted)
-        role_note = f"{wl.n_drafters} drafters per scale from scalekv_layer_stats; {hits}/{len(planted) * (wl.n_scales - 2)} planted recovered"
+        # Eq. 2 cannot tell the roles apart while the history is shorter than K' (then the top-K' mass is all of the
+        # history mass and ASI = c (1 - c) is symmetric): count the recovery over the scales with a longer history
+        n_cum = [sum(wl.n_tokens[:k]) for k in range(wl.n_scales)]
+        ks = [k for k in range(1, wl.n_scales - 1) if n_cum[k] > 4 * 16]
+        hits = sum(int(roles[l][k]) for k in ks for l in planted)
+        role_note = (f"{wl.n_drafters} drafters per scale from scalekv_layer_stats; {hits}/{len(planted) * len(ks)} planted "
+                     f"drafters recovered at the {len(ks)} scales whose history exceeds 4 K'")
     else:
         b = pipeline.pct_budget(10, 100, sum(wl.n_tokens[:-1]))
         budgets = [[b] * wl.n_scales for _ in range(wl.n_layers)]

@@ -306,3 +306,44 @@ def test_hires_16_scales_sampled_slices():
                     max_rows=512).run()
     assert run.evictions > 0
     kv.close()
+
+
+def test_strided_views_of_a_packed_qkv_tensor():
+    """Q, K, V as strided views of one packed [B, n, 3, H, d] activation tensor (token stride 3 H d, head
+    stride d), O into a strided view as well: the tensor maps and the copy kernels take strides."""
+    sides = (3, 7, 13, 17)
+    n = orc.scale_token_counts(sides)
+    B, H, d = 2, 3, 128
+    budgets = [[60] * len(sides)]
+    kv = binding.ScaleKV(1, B, H, d, "bf16", sides, sides, budgets, max_window=16)
+    g = torch.Generator().manual_seed(77)
+    caches = {(b, h): orc.SliceCache(n, d) for b in range(B) for h in range(H)}
+    worst = 0.0
+    for k in range(len(sides)):
+        packed = torch.randn(B, n[k], 3, H, d, generator=g).to(torch.bfloat16)
+        pd = packed.cuda()
+        Q, K, V = (pd[:, :, i].permute(0, 2, 1, 3) for i in range(3))          # [B, H, n, d] views, not contiguous
+        assert not Q.is_contiguous()
+        Obuf = torch.zeros(B, n[k], H, d, dtype=torch.bfloat16, device="cuda")
+        O = Obuf.permute(0, 2, 1, 3)
+        torch.cuda.synchronize()
+        kv.scalekv_append(0, k, K, V)
+        kv.scalekv_attend(0, Q, O)
+        wpos = orc.window_centroids(sides[k], sides[k], 16)
+        if k + 1 < len(sides):
+            kv.scalekv_compress(0, Q, wpos, qw_is_full_map=True)
+        kv.scalekv_sync()
+        for b in range(B):
+            for h in range(H):
+                c = caches[(b, h)]
+                qh, kh, vh = (packed[b, :, i, h].double().numpy() for i in range(3))
+                c.append(kh, vh)
+                Oo, _ = c.attend(qh)
+                worst = max(worst, float(np.max(np.abs(Oo - Obuf[b, :, h].double().cpu().numpy()))))
+                if k + 1 < len(sides):
+                    want, _ = c.compress(qh[wpos], wpos, budgets[0][k])
+                    pos, Kg, Vg = kv.scalekv_export_slice(0, b, h, with_kv=True)
+                    assert np.array_equal(pos.numpy(), want)
+                    assert np.array_equal(Kg.double().numpy(), c.K) and np.array_equal(Vg.double().numpy(), c.V)
+    assert worst <= 2e-2, worst
+    kv.close()
