@@ -347,3 +347,16 @@ def test_strided_views_of_a_packed_qkv_tensor():
                     assert np.array_equal(Kg.double().numpy(), c.K) and np.array_equal(Vg.double().numpy(), c.V)
     assert worst <= 2e-2, worst
     kv.close()
+
+
+def test_budget_zero_keeps_only_the_window():
+    """k^l = 0: every candidate is evicted, the window entries alone survive (and still attend correctly)."""
+    sides = (2, 5, 9, 12)
+    n = orc.scale_token_counts(sides)
+    budgets = [[0] * len(sides)]
+    kv = binding.ScaleKV(1, 1, 2, 128, "bf16", sides, sides, budgets, max_window=16)
+    run = ParityRun(kv, "bf16", sides, budgets, randn_inputs(1, 2, 128, n, torch.bfloat16, 41),
+                    lambda k: orc.window_centroids(sides[k], sides[k], 16), all_slices(1, 1, 2), compress_last=True).run()
+    assert run.evictions == 2 * (len(sides) - 1)        # the first map is its own window: nothing to evict
+    assert kv.scalekv_lengths(0) == [[16, 16]]
+    kv.close()
