@@ -425,9 +425,13 @@ scalekv_status scalekv_reset(scalekv_ctx *ctx) {
   if (!ctx) return SCALEKV_ERR_INVALID_ARG;
   const Plan &p = ctx->plan;
   if (ctx->s_side != ctx->s_main) {
-    cudaEvent_t e = ctx->ev_compress[0];
-    CU(cudaEventRecord(e, ctx->s_side));
-    CU(cudaStreamWaitEvent(ctx->s_main, e, 0));
+    // stream_main forks to stream_side and joins it again: everything enqueued on either stream so far
+    // precedes the reset.  (Fork before join, so that the sequence is also legal while stream_main is
+    // being captured into a CUDA graph.)
+    CU(cudaEventRecord(ctx->ev_attend[0], ctx->s_main));
+    CU(cudaStreamWaitEvent(ctx->s_side, ctx->ev_attend[0], 0));
+    CU(cudaEventRecord(ctx->ev_compress[0], ctx->s_side));
+    CU(cudaStreamWaitEvent(ctx->s_main, ctx->ev_compress[0], 0));
   }
   CU(cudaMemsetAsync(ctx->pool + p.off_len, 0, (size_t)p.n_layers * p.n_slices * 4, ctx->s_main));
   if (ctx->s_side != ctx->s_main) {

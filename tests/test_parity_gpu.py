@@ -360,3 +360,57 @@ def test_budget_zero_keeps_only_the_window():
     assert run.evictions == 2 * (len(sides) - 1)        # the first map is its own window: nothing to evict
     assert kv.scalekv_lengths(0) == [[16, 16]]
     kv.close()
+
+
+def test_whole_pass_replays_from_a_cuda_graph():
+    """reset + every append / attend / compress of a pass captured on stream_main (compress forks to
+    stream_side inside the capture) replays to the same outputs and the same kept sets as eager calls."""
+    from paper_2505_19602_b200 import pipeline
+
+    sides = (1, 2, 4, 8, 12, 16, 20)
+    wl = synth.Workload("g", 3, 2, 2, 128, "bf16", sides, seed=23, n_drafters=1)
+    budgets = [[120] * len(sides), [30] * len(sides), [60] * len(sides)]
+    kv = binding.ScaleKV(3, 2, 2, 128, "bf16", sides, sides, budgets, max_window=16)
+    inputs = pipeline.PassInputs(wl)
+    windows = pipeline.windows_for(sides, 16)
+    pipeline.run_pass(kv, inputs, windows)
+    kv.scalekv_sync()
+    want_O = inputs.O.clone()
+    want_pos = [kv.scalekv_export_slice(l, 1, 1).clone() for l in range(3)]
+    g = torch.cuda.CUDAGraph()
+    torch.cuda.synchronize()
+    with torch.cuda.graph(g, stream=kv.stream_main):
+        pipeline.run_pass(kv, inputs, windows)
+        kv.stream_main.wait_stream(kv.stream_side)
+    for _ in range(2):
+        inputs.O.zero_()
+        torch.cuda.synchronize()
+        with torch.cuda.stream(kv.stream_main):
+            g.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(inputs.O, want_O)
+        for l in range(3):
+            assert torch.equal(kv.scalekv_export_slice(l, 1, 1), want_pos[l])
+    kv.close()
+
+
+def test_budget_table_from_eq4_with_global_roles_and_refiner_decay():
+    """Budgets that differ per (layer, scale): roles ranked over all pairs (the printed form of the
+    drafter selection), refiner budgets decaying with the scale, drafters taking what the refiners save."""
+    sides = (1, 2, 4, 6, 8, 12, 16)
+    n = orc.scale_token_counts(sides)
+    L_layers = 4
+    rng = np.random.default_rng(5)
+    asi = rng.random((L_layers, len(sides))) * 0.2
+    roles = binding.scalekv_assign_roles(asi, 7, mode=0)
+    assert np.array_equal(roles, orc.assign_roles(asi, 7, 0))
+    table = binding.scalekv_make_budgets(roles, 40, 30, 3)
+    assert np.array_equal(table, orc.make_budgets(roles, 40, 30, 3))
+    budgets = [[int(x) for x in row] for row in table]
+    assert len({b for row in budgets for b in row}) > 4            # really varies
+    wl = synth.Workload("b", L_layers, 1, 2, 128, "bf16", sides, seed=29, n_drafters=1)
+    kv = binding.ScaleKV(L_layers, 1, 2, 128, "bf16", sides, sides, budgets, max_window=16)
+    run = ParityRun(kv, "bf16", sides, budgets, lambda l, k: synth.scale_inputs(wl, l, k),
+                    lambda k: orc.window_centroids(sides[k], sides[k], 16), all_slices(L_layers, 1, 2)).run()
+    assert run.evictions > 0
+    kv.close()
