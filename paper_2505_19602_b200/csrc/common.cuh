@@ -73,10 +73,4 @@ template <> struct Vec16<__nv_bfloat16> {
   }
 };
 
-// Non-negative-or-any float -> uint32 whose unsigned order equals the float order.
-__device__ __forceinline__ uint32_t orderable(float f) {
-  uint32_t u = __float_as_uint(f);
-  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-}
-
 }  // namespace scalekv

@@ -709,20 +709,4 @@ __global__ void __launch_bounds__(256) layer_stats_kernel(LayerView lv, TensorVi
   }
 }
 
-// rows window_pos[j] of a dense [B*H][n_k][d] tensor -> dense [B*H][w][d] (16-byte pieces)
-__global__ void gather_rows_kernel(const char *src, char *dst, WindowArg wa, int row_bytes, int n_slices) {
-  const int ppr = row_bytes >> 4;
-  const long long total = (long long)n_slices * wa.w * ppr;
-  for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < total;
-       idx += (long long)gridDim.x * blockDim.x) {
-    const int c = (int)(idx % ppr);
-    const long long rj = idx / ppr;
-    const int j = (int)(rj % wa.w);
-    const long long sl = rj / wa.w;
-    const int qi = wa.all ? j : wa.pos[j];
-    reinterpret_cast<uint4 *>(dst + (sl * wa.w + j) * row_bytes)[c] =
-        reinterpret_cast<const uint4 *>(src + (sl * wa.n_k + qi) * row_bytes)[c];
-  }
-}
-
 }  // namespace scalekv

@@ -48,7 +48,7 @@ struct Plan {
   size_t off_k, off_v, off_pos, off_pt, off_len, off_status, pool_bytes;
   size_t pt_elems, logits_elems;
   // workspace layout
-  size_t off_logits, off_wlse, off_scores, off_keys, off_keep, off_kept, off_acc, off_qw, ws_bytes;
+  size_t off_logits, off_wlse, off_scores, off_keys, off_keep, off_kept, off_acc, ws_bytes;
 };
 
 // Raster indices of the observation window of an h x w map (see scalekv_window_centroids).
@@ -155,7 +155,6 @@ scalekv_status make_plan(const scalekv_config *c, Plan &p, std::string &err) {
   p.off_keep = o; o = align_up(o + (size_t)p.n_slices * p.ld_s * 4, 1024);
   p.off_kept = o; o = align_up(o + (size_t)p.n_slices * 4, 1024);
   p.off_acc = o; o = align_up(o + 64, 1024);
-  p.off_qw = o; o = align_up(o + (size_t)p.n_slices * p.max_window * row_bytes, 1024);
   p.ws_bytes = o;
   return SCALEKV_OK;
 }
