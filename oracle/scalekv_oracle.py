@@ -143,6 +143,48 @@ def select(scores, pos, n_prev, window_pos, budget):
     return np.nonzero(keep)[0]
 
 
+def pool_scores(scores, kernel):
+    """1-D average pooling of the importance along the slot axis (Sec. 3.3 speaks of "average pooling",
+    and of the selection being "similar to" SnapKV, which smooths its votes this way).
+
+    Reading: window of odd width `kernel` centred on the entry, zeros beyond both ends, always divided
+    by `kernel` (the usual avg_pool1d with padding kernel // 2); the neighbours are the entries next to
+    it in the cache as it stands (ascending original position), window entries included.  kernel = 1
+    leaves the scores as they are.  This is the alternative to the default reading (no pooling along
+    keys); parity between the two readings is unpinned.
+    """
+    s = np.asarray(scores, dtype=np.float64)
+    k = int(kernel)
+    if k <= 1:
+        return s.copy()
+    assert k % 2 == 1
+    r = k // 2
+    padded = np.concatenate([np.zeros(r), s, np.zeros(r)])
+    out = np.zeros_like(s)
+    for d in range(k):
+        out += padded[d:d + s.shape[0]]
+    return out / k
+
+
+def select_recent(pos, budget, n_sink=0):
+    """Positional keep rule used by the paper's comparison policies (Sec. 4.1: sliding window;
+    sinks + recent tokens): of the L entries keep those whose original position is below n_sink,
+    and of the others the most recent ones, `budget` entries in all (KEEP_ALL keeps everything).
+    Returns the ascending slot indices that are kept."""
+    pos = np.asarray(pos, dtype=np.int64)
+    L = pos.shape[0]
+    if budget == KEEP_ALL or budget >= L:
+        return np.arange(L)
+    sink = pos < int(n_sink)
+    n_recent = max(int(budget) - int(sink.sum()), 0)
+    others = np.nonzero(~sink)[0]
+    order = np.argsort(-pos[others], kind="stable")
+    keep = np.zeros(L, dtype=bool)
+    keep[others[order[:n_recent]]] = True
+    keep |= sink
+    return np.nonzero(keep)[0]
+
+
 # --------------------------------------------------------------------------------------
 # One slice's cache and the per-scale step (call order append -> attend -> compress).
 # --------------------------------------------------------------------------------------
@@ -182,12 +224,17 @@ class SliceCache:
     def scores(self, Qw):
         return window_scores(Qw, self.K, self.scale)
 
-    def compress(self, Qw, window_pos, budget):
-        """Score, select, prune (Sec. 3.3).  Returns (kept original positions, scores)."""
-        s = self.scores(Qw)
+    def compress(self, Qw, window_pos, budget, pool_kernel=1):
+        """Score, (pool,) select, prune (Sec. 3.3).  Returns (kept original positions, scores)."""
+        s = pool_scores(self.scores(Qw), pool_kernel)
         keep = select(s, self.pos, self.N[self.k - 1], window_pos, budget)
         self.adopt(keep)
         return self.pos.copy(), s
+
+    def compress_recent(self, budget, n_sink=0):
+        """Positional pruning (sliding window, sinks + recent).  Returns the kept original positions."""
+        self.adopt(select_recent(self.pos, budget, n_sink))
+        return self.pos.copy()
 
     def adopt(self, keep_slots):
         """Prune to the given ascending slot list."""

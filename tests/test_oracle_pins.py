@@ -385,3 +385,48 @@ def test_make_budgets_satisfies_eq4():
     B0 = orc.make_budgets(roles, bu, br0, 0)
     B70 = orc.make_budgets(roles, bu, br0, 70)
     assert B70[roles].sum() > B0[roles].sum() and B70[~roles].sum() < B0[~roles].sum()
+
+
+# ---- alternative selection rules (pooling along the key axis, positional policies) -------------------
+def test_pool_scores_against_brute_force_and_closed_forms():
+    rng = np.random.default_rng(11)
+    s = rng.random(37)
+    for k in (1, 3, 7, 9):
+        got = orc.pool_scores(s, k)
+        want = np.zeros_like(s)
+        for i in range(len(s)):
+            for d in range(-(k // 2), k // 2 + 1):
+                if 0 <= i + d < len(s):
+                    want[i] += s[i + d]
+            want[i] /= k
+        assert np.allclose(got, want, atol=1e-15)
+    assert np.array_equal(orc.pool_scores(s, 1), s)
+    ones = np.ones(10)
+    p = orc.pool_scores(ones, 5)
+    assert np.allclose(p[2:8], 1.0) and np.allclose(p[[0, 9]], 3 / 5) and np.allclose(p[[1, 8]], 4 / 5)
+    # a single spike spreads evenly over its neighbourhood and keeps its mass
+    e = np.zeros(21); e[10] = 1.0
+    q = orc.pool_scores(e, 7)
+    assert np.allclose(q[7:14], 1 / 7) and np.isclose(q.sum(), 1.0) and q[6] == 0
+
+
+def test_select_recent_brute_force_and_count_rule():
+    rng = np.random.default_rng(12)
+    for trial in range(30):
+        L = int(rng.integers(1, 40))
+        pos = np.sort(rng.choice(200, size=L, replace=False))
+        budget = int(rng.integers(0, L + 3))
+        n_sink = int(rng.integers(0, 6))
+        keep = orc.select_recent(pos, budget, n_sink)
+        if budget >= L:
+            assert np.array_equal(keep, np.arange(L))
+            continue
+        sinks = [i for i in range(L) if pos[i] < n_sink]
+        rest = sorted((i for i in range(L) if pos[i] >= n_sink), key=lambda i: -pos[i])
+        want = sorted(sinks + rest[: max(budget - len(sinks), 0)])
+        assert keep.tolist() == want
+        assert len(keep) == max(budget, len(sinks))
+    assert np.array_equal(orc.select_recent(np.arange(5), orc.KEEP_ALL, 2), np.arange(5))
+    # sliding window: the last entries; sinks + recent: the first n_sink and the last ones
+    assert orc.select_recent(np.arange(10), 3).tolist() == [7, 8, 9]
+    assert orc.select_recent(np.arange(10), 5, 2).tolist() == [0, 1, 7, 8, 9]
