@@ -145,6 +145,28 @@ scalekv_status scalekv_attend(scalekv_ctx *ctx, int32_t layer, scalekv_tensor Q,
 scalekv_status scalekv_compress(scalekv_ctx *ctx, int32_t layer, scalekv_tensor Qw, int32_t w,
                                 const int32_t *window_pos, int32_t qw_is_full_map);
 
+/* Variants of the selection rule (the readings and comparison policies the paper names beside its own).
+ *   policy       SCALEKV_SELECT_SCORE: the observation-window importance of Sec. 3.3 (scalekv_compress).
+ *                SCALEKV_SELECT_RECENT: positional, as in the comparison policies of Sec. 4.1 (sliding
+ *                window; attention sinks + recent tokens): there is no observation window (Qw, w,
+ *                window_pos are ignored), the n_sink lowest original positions always stay and the most
+ *                recent other entries fill the budget; here k^l = budgets[layer][scale] counts the WHOLE
+ *                cache after the call, sinks included.
+ *   pool_kernel  SCORE only.  Odd width (< 64) of a 1-D average pooling of the importance along the slot
+ *                axis before the selection ("average pooling", Sec. 3.3, read as smoothing along keys: zeros
+ *                beyond both ends, always divided by the width; the neighbours are the entries next to it in
+ *                the cache as it stands, window entries included).  0 or 1: none - the default reading.
+ * opts == NULL is scalekv_compress. */
+#define SCALEKV_SELECT_SCORE 0
+#define SCALEKV_SELECT_RECENT 1
+typedef struct {
+  int32_t policy;
+  int32_t pool_kernel;
+  int32_t n_sink;        /* RECENT only */
+} scalekv_select_opts;
+scalekv_status scalekv_compress_ex(scalekv_ctx *ctx, int32_t layer, scalekv_tensor Qw, int32_t w, const int32_t *window_pos,
+                                   int32_t qw_is_full_map, const scalekv_select_opts *opts);
+
 /* One whole step for one layer from HOST memory (pinned memory recommended): copies Q, K, V
  * (dense [B][H][n_k][d]) to `staging`, runs append, attend and compress with the window rows
  * taken from Q (w > 0: explicit window_pos; w < 0: the whole map is the window; w == 0: no

@@ -43,6 +43,10 @@ class scalekv_config(C.Structure):
     ]
 
 
+class scalekv_select_opts(C.Structure):
+    _fields_ = [("policy", C.c_int32), ("pool_kernel", C.c_int32), ("n_sink", C.c_int32)]
+
+
 class scalekv_tensor(C.Structure):
     _fields_ = [("ptr", C.c_void_p), ("stride_b", C.c_int64), ("stride_h", C.c_int64), ("stride_t", C.c_int64)]
 
@@ -88,6 +92,7 @@ def load_library():
         "scalekv_append": [ctx_p, i32, i32, T, T],
         "scalekv_attend": [ctx_p, i32, T, T, C.c_void_p],
         "scalekv_compress": [ctx_p, i32, T, i32, P(i32), i32],
+        "scalekv_compress_ex": [ctx_p, i32, T, i32, P(i32), i32, P(scalekv_select_opts)],
         "scalekv_step_host": [ctx_p, i32, i32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, i32, P(i32)],
         "scalekv_layer_stats": [ctx_p, i32, T, i32, i32, P(f64), P(f64)],
         "scalekv_window_centroids": [i32, i32, i32, P(i32), P(i32)],
@@ -268,6 +273,17 @@ class ScaleKV:
         else:
             wp = _i32_array(window_pos)
             self._check(self.lib.scalekv_compress(self.ctx, layer, tensor_arg(Qw), len(window_pos), wp, int(qw_is_full_map)))
+
+    def scalekv_compress_ex(self, layer, Qw=None, window_pos=None, qw_is_full_map=False, policy="score", pool_kernel=1,
+                            n_sink=0):
+        """scalekv_compress with a selection variant: policy "score" (optionally pooled) or "recent"."""
+        opts = scalekv_select_opts({"score": 0, "recent": 1}[policy], pool_kernel, n_sink)
+        q = tensor_arg(Qw) if Qw is not None else scalekv_tensor(None, 0, 0, 0)
+        if window_pos is None:
+            wp, w = None, 0
+        else:
+            wp, w = _i32_array(window_pos), len(window_pos)
+        self._check(self.lib.scalekv_compress_ex(self.ctx, layer, q, w, wp, int(qw_is_full_map), C.byref(opts)))
 
     def scalekv_step_host(self, layer, scale, Qh, Kh, Vh, Oh, staging, window_pos=None, whole_map=False):
         if whole_map:

@@ -375,6 +375,18 @@ __global__ void __launch_bounds__(256) score_kernel(LayerView lv, WindowArg wa, 
   keys[(size_t)slice * ld_s + i] = win ? kWindowKey : (__float_as_uint(sc) & 0x7FFFFFFFu);
 }
 
+// Keys of the positional keep rule (the comparison policies of Sec. 4.1: sliding window, sinks + recent
+// tokens): entries whose original position is below n_sink carry the sentinel (always kept), every
+// other entry competes on its position, most recent first.  grid (ceil(L_max / 256), n_slices).
+__global__ void __launch_bounds__(256) recent_keys_kernel(LayerView lv, int n_k, int n_sink, uint32_t *keys, int ld_s) {
+  const int slice = blockIdx.y;
+  const int L = lv.hist_len[slice] + n_k;
+  const int i = blockIdx.x * 256 + threadIdx.x;
+  if (i >= L) return;
+  const int pos = lv.pos_pool[slot_row(lv, slice, i)];
+  keys[(size_t)slice * ld_s + i] = pos < n_sink ? kWindowKey : (uint32_t)pos + 1u;
+}
+
 // Base-2 log-sum-exp of every window row of y[w][L] when attend did not record it: one CTA of 1024
 // threads per slice, 16 rows per round, a maximum sweep and a sum sweep.  lse is [n_slices][w].
 __global__ void __launch_bounds__(1024) row_lse_kernel(LayerView lv, WindowArg wa, const float *logits, int ld_l, float *lse) {
@@ -433,15 +445,17 @@ __global__ void __launch_bounds__(1024) row_lse_kernel(LayerView lv, WindowArg w
 
 // ------------------------------------------------------------------------------------------
 // select: per-slice top-k' of the non-window entries by key (Sec. 3.3), one CTA of 1024 threads per
-// slice with the slice's keys in shared memory:
+// slice with the slice's keys in shared memory (with pool > 1 a candidate's key is first replaced by
+// its importance averaged over the neighbouring entries):
 //   radix select of the k'-th largest key, 8 bits per pass, warp-aggregated histogram updates; then
 //   the ordered emit of the ascending slot list of survivors (selected U window); ties at the
 //   threshold go to the lowest slots = lowest original positions.  Every thread owns a run of
 //   consecutive entries, so two block scans order the whole list.  Deterministic.
 // Dynamic shared memory: 4 * ld_s bytes of keys.
 // ------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(1024) select_kernel(LayerView lv, WindowArg wa, int budget, const uint32_t *keys, int ld_s,
-                                                      int *keep_list, int *kept_count) {
+__global__ void __launch_bounds__(1024) select_kernel(LayerView lv, WindowArg wa, int budget, const uint32_t *keys,
+                                                      const float *scores, int pool, int ld_s, int *keep_list,
+                                                      int *kept_count) {
   extern __shared__ uint32_t key[];            // [L]
   __shared__ int hist[256];
   __shared__ int warp_sums[33];
@@ -454,7 +468,16 @@ __global__ void __launch_bounds__(1024) select_kernel(LayerView lv, WindowArg wa
 
   int n_win_local = 0;
   for (int i = tid; i < L; i += 1024) {
-    const uint32_t k = __ldg(keys + (size_t)slice * ld_s + i);
+    uint32_t k = __ldg(keys + (size_t)slice * ld_s + i);
+    if (pool > 1 && k != kWindowKey) {
+      // the importance averaged over `pool` neighbouring entries (zeros beyond both ends), summed in slot order
+      const float *sc = scores + (size_t)slice * ld_s;
+      const int r = pool >> 1;
+      float acc = 0.f;
+      for (int d = -r; d <= r; ++d)
+        if (i + d >= 0 && i + d < L) acc += __ldg(sc + i + d);
+      k = __float_as_uint(acc / (float)pool) & 0x7FFFFFFFu;
+    }
     key[i] = k;
     n_win_local += (k == kWindowKey) ? 1 : 0;
   }

@@ -549,18 +549,42 @@ scalekv_status scalekv_attend(scalekv_ctx *ctx, int32_t layer, scalekv_tensor Q,
 
 scalekv_status scalekv_compress(scalekv_ctx *ctx, int32_t layer, scalekv_tensor Qw, int32_t w, const int32_t *window_pos,
                                 int32_t qw_is_full_map) {
+  return scalekv_compress_ex(ctx, layer, Qw, w, window_pos, qw_is_full_map, nullptr);
+}
+
+scalekv_status scalekv_compress_ex(scalekv_ctx *ctx, int32_t layer, scalekv_tensor Qw, int32_t w, const int32_t *window_pos,
+                                   int32_t qw_is_full_map, const scalekv_select_opts *opts) {
   if (!ctx) return SCALEKV_ERR_INVALID_ARG;
   const Plan &p = ctx->plan;
   if (layer < 0 || layer >= p.n_layers) return fail(ctx, SCALEKV_ERR_INVALID_ARG, "layer %d out of range", layer);
   if (ctx->pending[layer] == 0) return fail(ctx, SCALEKV_ERR_BAD_STATE, "layer %d: compress needs a preceding append", layer);
-  if (!tensor_ok(Qw, p.esize)) return fail(ctx, SCALEKV_ERR_INVALID_ARG, "Qw null or rows not 16-byte aligned");
-  WindowArg wa;
-  scalekv_status st = fill_window(ctx, layer, w, window_pos, wa);
-  if (st != SCALEKV_OK) return st;
+  const int policy = opts ? opts->policy : SCALEKV_SELECT_SCORE;
+  const int pool = (opts && opts->pool_kernel > 1) ? opts->pool_kernel : 1;
+  const int n_sink = opts ? opts->n_sink : 0;
+  if (policy != SCALEKV_SELECT_SCORE && policy != SCALEKV_SELECT_RECENT) return fail(ctx, SCALEKV_ERR_INVALID_ARG, "unknown selection policy %d", policy);
+  if (pool % 2 == 0 || pool > 63) return fail(ctx, SCALEKV_ERR_INVALID_ARG, "pool_kernel must be odd and below 64");
+  if (n_sink < 0) return fail(ctx, SCALEKV_ERR_INVALID_ARG, "n_sink must not be negative");
+  const bool recent = policy == SCALEKV_SELECT_RECENT;
   const int k = ctx->next_scale[layer] - 1;
   const int L = ctx->hist[layer] + ctx->pending[layer];
-  const int cand = L - wa.w;
-  const int budget = p.budgets[(size_t)layer * p.K + k];
+  WindowArg wa;
+  scalekv_status st = SCALEKV_OK;
+  int always_kept;       // entries outside the selection: the window, or the sinks
+  if (recent) {
+    // no observation window: every entry but the sinks competes on its original position
+    wa.w = 0; wa.all = 0; wa.n_prev = p.N[k]; wa.n_k = p.n[k];
+    for (int j = 0; j < kMaxWindow; ++j) wa.pos[j] = 0x7fffffff;
+    always_kept = std::min(n_sink, p.N[k + 1]);          // positions 0 .. n_sink-1 are never evicted once appended
+  } else {
+    if (!tensor_ok(Qw, p.esize)) return fail(ctx, SCALEKV_ERR_INVALID_ARG, "Qw null or rows not 16-byte aligned");
+    st = fill_window(ctx, layer, w, window_pos, wa);
+    if (st != SCALEKV_OK) return st;
+    always_kept = wa.w;
+  }
+  const int cand = L - always_kept;
+  const int table = p.budgets[(size_t)layer * p.K + k];
+  // SCORE: k^l counts the selected entries, the window comes on top.  RECENT: k^l is the whole cache, sinks included.
+  const int budget = (recent && table != SCALEKV_KEEP_ALL) ? std::max(table - always_kept, 0) : table;
   const bool evict = budget != SCALEKV_KEEP_ALL && budget < cand;
   // while per-kernel timing is on, compress runs on stream_main too, so that every kernel is timed alone
   cudaStream_t s = ctx->serialize ? ctx->s_main : ctx->s_side;
@@ -580,9 +604,14 @@ scalekv_status scalekv_compress(scalekv_ctx *ctx, int32_t layer, scalekv_tensor 
     float *scores = reinterpret_cast<float *>(ctx->ws + p.off_scores);
     int *keep = reinterpret_cast<int *>(ctx->ws + p.off_keep);
     int *kept = reinterpret_cast<int *>(ctx->ws + p.off_kept);
+    uint32_t *keys = reinterpret_cast<uint32_t *>(ctx->ws + p.off_keys);
+    if (recent) {
+      Scope sc(ctx, s, kScore);
+      recent_keys_kernel<<<dim3((L + 255) / 256, p.n_slices), 256, 0, s>>>(lv, wa.n_k, n_sink, keys, p.ld_s);
+    }
     // the logits of exactly this window may already be there, recorded by attend
-    bool recorded = ctx->logits_of[layer] == k && (int)p.windows[k].size() == wa.w;
-    for (int j = 0; recorded && j < wa.w; ++j) recorded = p.windows[k][j] == wa.pos[j];
+    bool recorded = recent || (ctx->logits_of[layer] == k && (int)p.windows[k].size() == wa.w);
+    for (int j = 0; !recent && recorded && j < wa.w; ++j) recorded = p.windows[k][j] == wa.pos[j];
     if (!recorded) {
       Scope sc(ctx, s, kScore);
       dim3 grid((L + 63) / 64, p.n_slices);
@@ -595,25 +624,25 @@ scalekv_status scalekv_compress(scalekv_ctx *ctx, int32_t layer, scalekv_tensor 
     }
     ctx->logits_of[layer] = -1;
     float *wlse = reinterpret_cast<float *>(ctx->ws + p.off_wlse) + (size_t)(layer & 1) * p.n_slices * p.max_window;
-    uint32_t *keys = reinterpret_cast<uint32_t *>(ctx->ws + p.off_keys);
     if (!recorded) {
       Scope sc(ctx, s, kScore);
       row_lse_kernel<<<p.n_slices, 1024, 0, s>>>(lv, wa, logits, p.ld_s, wlse);
     }
-    {
+    if (!recent) {
       Scope sc(ctx, s, kScore);
       score_kernel<<<dim3((L + 255) / 256, p.n_slices), 256, 0, s>>>(lv, wa, logits, wlse, p.ld_s, scores, keys, p.ld_s);
     }
     {
       Scope sc(ctx, s, kSelect);
-      select_kernel<<<p.n_slices, 1024, (size_t)p.ld_s * 4, s>>>(lv, wa, budget, keys, p.ld_s, keep, kept);
+      select_kernel<<<p.n_slices, 1024, (size_t)p.ld_s * 4, s>>>(lv, wa, budget, keys, recent ? nullptr : scores, pool, p.ld_s,
+                                                                 keep, kept);
     }
     {
       Scope sc(ctx, s, kCompact);
       compact_kernel<<<dim3(p.n_slices, 2, 4), 256, (size_t)(p.ld_s + lv.pages_per_slice) * 4, s>>>(lv, keep, p.ld_s, kept);
     }
-    ctx->scores_len = L;
-    ctx->hist[layer] = budget + wa.w;
+    ctx->scores_len = recent ? 0 : L;
+    ctx->hist[layer] = budget + always_kept;
     ctx->pending[layer] = 0;
     ctx->attended[layer] = 0;
     st = check_launch(ctx, "compress");

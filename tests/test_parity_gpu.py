@@ -414,3 +414,87 @@ def test_budget_table_from_eq4_with_global_roles_and_refiner_decay():
                     lambda k: orc.window_centroids(sides[k], sides[k], 16), all_slices(L_layers, 1, 2)).run()
     assert run.evictions > 0
     kv.close()
+
+
+def _kept_or_tie(got_pos, cache_pos_before, s, keep_slots, w_abs):
+    """True when got_pos equals the oracle's kept positions or differs only inside the 1e-3 tie band."""
+    want_pos = cache_pos_before[keep_slots]
+    if np.array_equal(got_pos, want_pos):
+        return True
+    sel = np.zeros(len(cache_pos_before), dtype=bool)
+    sel[keep_slots] = True
+    sel &= ~np.isin(cache_pos_before, w_abs)
+    boundary = s[sel].min()
+    diff = np.setxor1d(got_pos, want_pos)
+    idx = np.searchsorted(cache_pos_before, diff)
+    return bool(np.all(np.abs(s[idx] - boundary) / max(abs(boundary), 1e-300) < 1e-3))
+
+
+def test_pooled_importance_matches_oracle():
+    """scalekv_compress_ex with a 7-wide average pooling of the importance along the key axis."""
+    sides = (2, 5, 9, 14, 19)
+    n = orc.scale_token_counts(sides)
+    N = orc.cumulative_token_counts(n)
+    budgets = [[70] * len(sides)]
+    B, H = 1, 3
+    kv = binding.ScaleKV(1, B, H, 128, "bf16", sides, sides, budgets, max_window=16)
+    wl = synth.Workload("p", 1, B, H, 128, "bf16", sides, seed=33)
+    caches = [orc.SliceCache(n, 128) for _ in range(H)]
+    evictions = 0
+    for k in range(len(sides)):
+        Q, K, V = synth.scale_inputs(wl, 0, k)
+        Qd, Kd, Vd = Q.cuda(), K.cuda(), V.cuda()
+        torch.cuda.synchronize()
+        kv.scalekv_append(0, k, Kd, Vd)
+        O = kv.scalekv_attend(0, Qd)
+        wpos = orc.window_centroids(sides[k], sides[k], 16)
+        kv.scalekv_compress_ex(0, Qd, wpos, qw_is_full_map=True, policy="score", pool_kernel=7)
+        kv.scalekv_sync()
+        for h in range(H):
+            c = caches[h]
+            c.append(K[0, h].double().numpy(), V[0, h].double().numpy())
+            Oo, _ = c.attend(Q[0, h].double().numpy())
+            assert np.max(np.abs(Oo - O[0, h].double().cpu().numpy())) <= 2e-2
+            before = c.pos.copy()
+            s = orc.pool_scores(c.scores(Q[0, h].double().numpy()[wpos]), 7)
+            keep = orc.select(s, c.pos, N[k], wpos, budgets[0][k])
+            got = kv.scalekv_export_slice(0, 0, h).numpy().astype(np.int64)
+            assert len(got) == len(keep)
+            evictions += int(len(keep) < len(before))
+            assert _kept_or_tie(got, before, s, keep, [N[k] + p for p in wpos]), (k, h)
+            c.adopt_positions(got)
+    assert evictions >= 6
+    kv.close()
+
+
+@pytest.mark.parametrize("n_sink", [0, 4])
+def test_positional_policy_sliding_window_and_sinks(n_sink):
+    """scalekv_compress_ex with the positional rule: exact (positions are distinct, no ties)."""
+    sides = (2, 5, 9, 14, 19)
+    n = orc.scale_token_counts(sides)
+    budgets = [[50] * len(sides), [13] * len(sides)]
+    B, H = 2, 2
+    kv = binding.ScaleKV(2, B, H, 128, "bf16", sides, sides, budgets, max_window=16)
+    wl = synth.Workload("r", 2, B, H, 128, "bf16", sides, seed=35)
+    caches = {(l, b, h): orc.SliceCache(n, 128) for l in range(2) for b in range(B) for h in range(H)}
+    for k in range(len(sides)):
+        for l in range(2):
+            Q, K, V = synth.scale_inputs(wl, l, k)
+            Qd, Kd, Vd = Q.cuda(), K.cuda(), V.cuda()
+            torch.cuda.synchronize()
+            kv.scalekv_append(l, k, Kd, Vd)
+            O = kv.scalekv_attend(l, Qd)
+            kv.scalekv_compress_ex(l, policy="recent", n_sink=n_sink)
+            kv.scalekv_sync()
+            for b in range(B):
+                for h in range(H):
+                    c = caches[(l, b, h)]
+                    c.append(K[b, h].double().numpy(), V[b, h].double().numpy())
+                    Oo, _ = c.attend(Q[b, h].double().numpy())
+                    assert np.max(np.abs(Oo - O[b, h].double().cpu().numpy())) <= 2e-2
+                    want = c.compress_recent(budgets[l][k], n_sink)
+                    pos, Kg, Vg = kv.scalekv_export_slice(l, b, h, with_kv=True)
+                    assert np.array_equal(pos.numpy(), want), (k, l, b, h)
+                    assert np.array_equal(Kg.double().numpy(), c.K) and np.array_equal(Vg.double().numpy(), c.V)
+    assert kv.scalekv_lengths(1) == [[13, 13], [13, 13]]
+    kv.close()
