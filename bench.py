@@ -379,8 +379,8 @@ def run_scalekv(args):
         host = {}
         for k in range(wl.n_scales):
             host[k] = tuple(t.cpu().pin_memory() for t in inputs.data[(0, k)])
-        Oh = torch.empty(wl.batch, wl.n_heads, n_max, wl.head_dim, dtype=dt).pin_memory()
-        staging = torch.empty(4 * wl.batch * wl.n_heads * n_max * wl.head_dim, dtype=dt, device="cuda")
+        Oh = [torch.empty(wl.batch, wl.n_heads, n_max, wl.head_dim, dtype=dt).pin_memory() for _ in range(2)]
+        staging = torch.empty(8 * wl.batch * wl.n_heads * n_max * wl.head_dim, dtype=dt, device="cuda")
         torch.cuda.synchronize()
 
         def e2e_pass():
@@ -390,8 +390,8 @@ def run_scalekv(args):
                 Qh, Kh, Vh = host[k]
                 last = k + 1 == wl.n_scales
                 for l in range(wl.n_layers):
-                    kv.scalekv_step_host(l, k, Qh, Kh, Vh, Oh, staging, window_pos=None if last else windows[k])
-                    kv.scalekv_sync()          # the host reads the step's output before the next layer
+                    kv.scalekv_step_host(l, k, Qh, Kh, Vh, Oh[(l + k) & 1], staging, window_pos=None if last else windows[k])
+            kv.scalekv_sync()                  # every output has reached the host
         e2e_steps = max(1, min(args.steps, 3))
         e2e_pass()
         barrier()
@@ -405,8 +405,9 @@ def run_scalekv(args):
         tok_bytes = sum(wl.n_tokens) * wl.batch * wl.n_heads * wl.head_dim * esz * wl.n_layers
         e2e = {"value": wl.n_scales * e2e_steps * world / e2e_s, "unit": UNIT, "h2d_bytes_per_step": 3 * tok_bytes,
                "d2h_bytes_per_step": tok_bytes, "steps": e2e_steps,
-               "note": "pinned host Q/K/V -> device, append+attend+compress, O -> host, per layer and scale; "
-                       "layer 0's host tensors are reused for every layer"}
+               "note": "scalekv_step_host per layer and scale: pinned host Q/K/V -> device, append + attend + compress, O -> "
+                       "pinned host; the copies of neighbouring steps overlap the kernels; one sync per pass; layer 0's "
+                       "host tensors are reused for every layer"}
         del staging
 
     cpu = None

@@ -171,8 +171,10 @@ scalekv_status scalekv_compress_ex(scalekv_ctx *ctx, int32_t layer, scalekv_tens
  * (dense [B][H][n_k][d]) to `staging`, runs append, attend and compress with the window rows
  * taken from Q (w > 0: explicit window_pos; w < 0: the whole map is the window; w == 0: no
  * compress), and copies O back to O_host.  staging is device memory of at least
- * 4 * B*H*n_k*d elements.  Everything is enqueued on the context's streams; the host buffers must
- * stay valid until scalekv_sync. */
+ * 8 * B*H*n_k*d elements: consecutive calls alternate between its two halves, and the copies run
+ * on two streams of the library's own (created at the first call), so that a step's input copy, the
+ * previous step's kernels and the output copy before that overlap.  Everything is enqueued; the
+ * host buffers must stay valid, and O_host is complete, once scalekv_sync has returned. */
 scalekv_status scalekv_step_host(scalekv_ctx *ctx, int32_t layer, int32_t scale, const void *Q_host,
                                  const void *K_host, const void *V_host, void *O_host, void *staging,
                                  size_t staging_bytes, int32_t w, const int32_t *window_pos);

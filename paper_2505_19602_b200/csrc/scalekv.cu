@@ -168,6 +168,11 @@ struct scalekv_ctx {
   float scale = 0.f;
   char *pool = nullptr, *ws = nullptr;
   cudaStream_t s_main = nullptr, s_side = nullptr;
+  // scalekv_step_host only: copy streams of the library's own and, per staging half, the events that chain them
+  cudaStream_t s_h2d = nullptr, s_d2h = nullptr;
+  cudaEvent_t ev_in[2] = {nullptr, nullptr}, ev_out[2] = {nullptr, nullptr}, ev_att[2] = {nullptr, nullptr};
+  int set_layer[2] = {-1, -1};     // layer that last used a staging half (-1: unused)
+  long long host_steps = 0;
   std::vector<int> page_table_host;
   // per layer state
   std::vector<int> next_scale;     // scale expected by the next append
@@ -453,6 +458,13 @@ scalekv_status scalekv_destroy(scalekv_ctx *ctx) {
   cudaStreamSynchronize(ctx->s_main);
   if (ctx->s_side != ctx->s_main) cudaStreamSynchronize(ctx->s_side);
   drain_profile(ctx);
+  if (ctx->s_h2d) { cudaStreamSynchronize(ctx->s_h2d); cudaStreamDestroy(ctx->s_h2d); }
+  if (ctx->s_d2h) { cudaStreamSynchronize(ctx->s_d2h); cudaStreamDestroy(ctx->s_d2h); }
+  for (int i = 0; i < 2; ++i) {
+    if (ctx->ev_in[i]) cudaEventDestroy(ctx->ev_in[i]);
+    if (ctx->ev_out[i]) cudaEventDestroy(ctx->ev_out[i]);
+    if (ctx->ev_att[i]) cudaEventDestroy(ctx->ev_att[i]);
+  }
   for (auto e : ctx->ev_attend) cudaEventDestroy(e);
   for (auto e : ctx->ev_compress) cudaEventDestroy(e);
   for (auto e : ctx->event_pool) cudaEventDestroy(e);
@@ -664,11 +676,33 @@ scalekv_status scalekv_step_host(scalekv_ctx *ctx, int32_t layer, int32_t scale,
   if (!Q_host || !K_host || !V_host || !O_host || !staging) return fail(ctx, SCALEKV_ERR_INVALID_ARG, "null buffer");
   const int nk = p.n[scale];
   const size_t bytes = (size_t)p.n_slices * nk * p.d * p.esize;
-  if (staging_bytes < 4 * bytes) return fail(ctx, SCALEKV_ERR_CAPACITY, "staging needs %zu bytes", 4 * bytes);
-  char *dq = static_cast<char *>(staging), *dk = dq + bytes, *dv = dk + bytes, *dout = dv + bytes;
-  CU(cudaMemcpyAsync(dk, K_host, bytes, cudaMemcpyHostToDevice, ctx->s_main));
-  CU(cudaMemcpyAsync(dv, V_host, bytes, cudaMemcpyHostToDevice, ctx->s_main));
-  CU(cudaMemcpyAsync(dq, Q_host, bytes, cudaMemcpyHostToDevice, ctx->s_main));
+  if (staging_bytes < 8 * bytes) return fail(ctx, SCALEKV_ERR_CAPACITY, "staging needs %zu bytes", 8 * bytes);
+  if (!ctx->s_h2d) {
+    // first use: two copy streams of the library's own (input and output copies run in both directions
+    // at once and under the kernels of neighbouring steps) and the events that chain them
+    CU(cudaStreamCreateWithFlags(&ctx->s_h2d, cudaStreamNonBlocking));
+    CU(cudaStreamCreateWithFlags(&ctx->s_d2h, cudaStreamNonBlocking));
+    for (int i = 0; i < 2; ++i) {
+      CU(cudaEventCreateWithFlags(&ctx->ev_in[i], cudaEventDisableTiming));
+      CU(cudaEventCreateWithFlags(&ctx->ev_out[i], cudaEventDisableTiming));
+      CU(cudaEventCreateWithFlags(&ctx->ev_att[i], cudaEventDisableTiming));
+    }
+  }
+  // consecutive steps alternate between the two halves of the staging area
+  const int set = (int)(ctx->host_steps++ & 1);
+  char *dq = static_cast<char *>(staging) + (size_t)set * 4 * bytes, *dk = dq + bytes, *dv = dk + bytes, *dout = dv + bytes;
+  if (ctx->set_layer[set] >= 0) {
+    // the half's previous user must be through: its output copied out, its compress (which may read Q) done
+    CU(cudaStreamWaitEvent(ctx->s_h2d, ctx->ev_out[set], 0));
+    const int pl = ctx->set_layer[set];
+    if (ctx->ev_compress_live[pl]) CU(cudaStreamWaitEvent(ctx->s_h2d, ctx->ev_compress[pl], 0));
+    else CU(cudaStreamWaitEvent(ctx->s_h2d, ctx->ev_att[set], 0));
+  }
+  CU(cudaMemcpyAsync(dk, K_host, bytes, cudaMemcpyHostToDevice, ctx->s_h2d));
+  CU(cudaMemcpyAsync(dv, V_host, bytes, cudaMemcpyHostToDevice, ctx->s_h2d));
+  CU(cudaMemcpyAsync(dq, Q_host, bytes, cudaMemcpyHostToDevice, ctx->s_h2d));
+  CU(cudaEventRecord(ctx->ev_in[set], ctx->s_h2d));
+  CU(cudaStreamWaitEvent(ctx->s_main, ctx->ev_in[set], 0));
   auto dense = [&](const void *ptr) {
     scalekv_tensor t; t.ptr = ptr; t.stride_t = p.d; t.stride_h = (int64_t)nk * p.d; t.stride_b = (int64_t)p.H * nk * p.d;
     return t;
@@ -677,7 +711,11 @@ scalekv_status scalekv_step_host(scalekv_ctx *ctx, int32_t layer, int32_t scale,
   if (st != SCALEKV_OK) return st;
   st = scalekv_attend(ctx, layer, dense(dq), dense(dout), nullptr);
   if (st != SCALEKV_OK) return st;
-  CU(cudaMemcpyAsync(O_host, dout, bytes, cudaMemcpyDeviceToHost, ctx->s_main));
+  CU(cudaEventRecord(ctx->ev_att[set], ctx->s_main));
+  CU(cudaStreamWaitEvent(ctx->s_d2h, ctx->ev_att[set], 0));
+  CU(cudaMemcpyAsync(O_host, dout, bytes, cudaMemcpyDeviceToHost, ctx->s_d2h));
+  CU(cudaEventRecord(ctx->ev_out[set], ctx->s_d2h));
+  ctx->set_layer[set] = layer;
   if (w > 0) {
     st = scalekv_compress(ctx, layer, dense(dq), w, window_pos, 1);
     if (st != SCALEKV_OK) return st;
@@ -785,6 +823,8 @@ scalekv_status scalekv_sync(scalekv_ctx *ctx) {
   if (!ctx) return SCALEKV_ERR_INVALID_ARG;
   CU(cudaStreamSynchronize(ctx->s_main));
   if (ctx->s_side != ctx->s_main) CU(cudaStreamSynchronize(ctx->s_side));
+  if (ctx->s_h2d) CU(cudaStreamSynchronize(ctx->s_h2d));
+  if (ctx->s_d2h) CU(cudaStreamSynchronize(ctx->s_d2h));
   int status = 0;
   CU(cudaMemcpy(&status, ctx->pool + ctx->plan.off_status, 4, cudaMemcpyDeviceToHost));
   if (status == kDevTimeout) return fail(ctx, SCALEKV_ERR_TIMEOUT, "a bounded device-side wait gave up");

@@ -498,3 +498,48 @@ def test_positional_policy_sliding_window_and_sinks(n_sink):
                     assert np.array_equal(Kg.double().numpy(), c.K) and np.array_equal(Vg.double().numpy(), c.V)
     assert kv.scalekv_lengths(1) == [[13, 13], [13, 13]]
     kv.close()
+
+
+def test_step_host_pipeline_matches_device_calls():
+    """scalekv_step_host (pinned host buffers, double-buffered staging, copies on the library's own streams,
+    one sync at the end) gives bit-identical outputs and kept sets to append / attend / compress on
+    device tensors."""
+    sides = (1, 2, 4, 8, 12, 16)
+    n = orc.scale_token_counts(sides)
+    L_layers, B, H, d = 3, 2, 2, 128
+    wl = synth.Workload("e", L_layers, B, H, d, "bf16", sides, seed=37, n_drafters=1)
+    budgets = [[90] * len(sides), [25] * len(sides), [50] * len(sides)]
+    windows = [orc.window_centroids(a, a, 16) for a in sides]
+    data = {(l, k): synth.scale_inputs(wl, l, k) for l in range(L_layers) for k in range(len(sides))}
+    # device path
+    kv = binding.ScaleKV(L_layers, B, H, d, "bf16", sides, sides, budgets, max_window=16)
+    want_O = {}
+    for k in range(len(sides)):
+        for l in range(L_layers):
+            Q, K, V = (t.cuda() for t in data[(l, k)])
+            torch.cuda.synchronize()
+            kv.scalekv_append(l, k, K, V)
+            want_O[(l, k)] = kv.scalekv_attend(l, Q)
+            if k + 1 < len(sides):
+                kv.scalekv_compress(l, Q, windows[k], qw_is_full_map=True)
+    kv.scalekv_sync()
+    want_pos = [kv.scalekv_export_slice(l, 1, 0).clone() for l in range(L_layers)]
+    want_O = {key: t.cpu() for key, t in want_O.items()}
+    kv.close()
+    # host path: everything enqueued, one sync
+    kv = binding.ScaleKV(L_layers, B, H, d, "bf16", sides, sides, budgets, max_window=16)
+    host = {key: tuple(t.pin_memory() for t in qkv) for key, qkv in data.items()}
+    out = {key: torch.empty_like(qkv[0]).pin_memory() for key, qkv in data.items()}
+    staging = torch.empty(8 * B * H * max(n) * d, dtype=torch.bfloat16, device="cuda")
+    torch.cuda.synchronize()
+    for k in range(len(sides)):
+        for l in range(L_layers):
+            Qh, Kh, Vh = host[(l, k)]
+            kv.scalekv_step_host(l, k, Qh, Kh, Vh, out[(l, k)], staging,
+                                 window_pos=windows[k] if k + 1 < len(sides) else None)
+    kv.scalekv_sync()
+    for key in data:
+        assert torch.equal(out[key], want_O[key]), key
+    for l in range(L_layers):
+        assert torch.equal(kv.scalekv_export_slice(l, 1, 0), want_pos[l])
+    kv.close()
