@@ -45,6 +45,9 @@ def parse_args():
     ap.add_argument("--workload", default="pass2b")
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling on a small case)")
     ap.add_argument("--full-cache", action="store_true", help="KEEP_ALL budgets instead of drafter/refiner budgets")
+    ap.add_argument("--overall-pct", type=float, default=0.0,
+                    help="overall budget in per cent of the cached tokens (the 4 / 10 / 20 sweep of the 16-scale workload): "
+                         "refiner budget = overall / 3.25, drafter budget = 10 x refiner; default: 30 %% / 3 %%")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-side-stream", action="store_true")
@@ -272,7 +275,11 @@ def run_scalekv(args):
         role_note = "full cache"
     elif wl.n_drafters > 0:
         asi, roles = pipeline.calibrate_roles(wl, wl.n_drafters, device=local_rank)
-        budgets = pipeline.budget_table(wl, roles)
+        if args.overall_pct > 0:
+            r1000 = max(1, round(args.overall_pct * 1000 / 3.25))          # refiner share in 1/100000 of T_c
+            budgets = pipeline.budget_table(wl, roles, drafter_pct=(10 * r1000, 100000), refiner_pct=(r1000, 100000))
+        else:
+            budgets = pipeline.budget_table(wl, roles)
         planted = synth.drafter_layers(wl)
         # Eq. 2 cannot tell the roles apart while the history is shorter than K' (then the top-K' mass is all of the
         # history mass and ASI = c (1 - c) is symmetric): count the recovery over the scales with a longer history
@@ -422,7 +429,8 @@ def run_scalekv(args):
             "scaling": "weak", "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
             "config": {"workload": wl.name, "layers": wl.n_layers, "batch": wl.batch, "heads": wl.n_heads,
                        "head_dim": wl.head_dim, "scales": wl.n_scales, "tokens": sum(wl.n_tokens),
-                       "budget": role_note, "window": wl.window, "parallelism": f"replica x{world} (batch-sharded, no collective)",
+                       "budget": role_note + (f"; overall {args.overall_pct} %" if args.overall_pct > 0 else ""),
+                       "window": wl.window, "parallelism": f"replica x{world} (batch-sharded, no collective)",
                        "l2_policy": f"inputs larger than L2: {inputs.bytes() / 1e9:.1f} GB of Q/K/V per pass",
                        "side_stream": not args.no_side_stream, "calibration_s": round(calib_s, 1),
                        "attend_kernel": "tcgen05" if os.environ.get("SCALEKV_ATTEND", "") != "simt" else "simt"},
