@@ -414,6 +414,10 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     if (tid == 0) atomicExch(status, kDevCheck);
     return;
   }
+  if (L > (lv.pages_per_slice << lv.page_shift)) {               // the slice would outgrow its page table: report, do not fault
+    if (tid == 0) atomicExch(status, kDevCheck);
+    return;
+  }
 
   if (tid == 0) {
     *abort_flag = 0;

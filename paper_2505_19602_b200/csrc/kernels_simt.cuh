@@ -37,6 +37,10 @@ __global__ void __launch_bounds__(256) append_kernel(LayerView lv, TensorView K,
   const int b = slice / lv.n_heads, h = slice % lv.n_heads;
   const int ppr = lv.row_bytes >> 4;  // 16-byte pieces per row
   const int hist = lv.hist_len[slice];
+  if (hist + n_k > (lv.pages_per_slice << lv.page_shift)) {      // would outgrow the page table: report, do not fault
+    if (threadIdx.x == 0) atomicExch(lv.status, kDevCheck);
+    return;
+  }
   const int rows_per_step = 256 / ppr;
   const int r_in = threadIdx.x / ppr, c = threadIdx.x % ppr;
   const int i0 = blockIdx.x * 64;
@@ -579,7 +583,11 @@ __global__ void __launch_bounds__(1024) select_kernel(LayerView lv, WindowArg wa
     }
     if (keep) out[oidx++] = i;
   }
-  if (tid == 0) kept_count[slice] = keep_total;
+  if (tid == 0) {
+    kept_count[slice] = keep_total;
+    // the count rule of the selection: k' candidates and every sentinel entry survive
+    if (keep_total != kprime + n_win) atomicExch(lv.status, kDevCheck);
+  }
 }
 
 // ------------------------------------------------------------------------------------------

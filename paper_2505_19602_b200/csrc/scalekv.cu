@@ -2,6 +2,7 @@
 // The context plans the paged store, tracks the per-layer call order and lengths, orders the two
 // streams with events and launches the kernels.  Nothing here computes on the CPU.
 #include <cuda_runtime.h>
+#include <nvtx3/nvToolsExt.h>
 
 #include <algorithm>
 #include <cmath>
@@ -241,9 +242,13 @@ bool tensor_ok(const scalekv_tensor &t, int esize) {
   return ((t.stride_b * esize) % 16 == 0) && ((t.stride_h * esize) % 16 == 0) && ((t.stride_t * esize) % 16 == 0);
 }
 
-struct Scope {  // brackets one launch with events when profiling; counts launches
+const char *const kClassNames[kNumClasses] = {"scalekv.append", "scalekv.attend", "scalekv.score", "scalekv.select",
+                                               "scalekv.compact", "scalekv.other"};
+
+struct Scope {  // brackets one launch with an NVTX range and, when profiling, with events; counts launches
   scalekv_ctx *c; cudaStream_t s; int cls; cudaEvent_t a = nullptr, b = nullptr;
   Scope(scalekv_ctx *c_, cudaStream_t s_, int cls_) : c(c_), s(s_), cls(cls_) {
+    nvtxRangePushA(kClassNames[cls]);
     if (c->profile) {
       a = take(); b = take();
       cudaEventRecord(a, s);
@@ -254,6 +259,7 @@ struct Scope {  // brackets one launch with events when profiling; counts launch
     cudaEvent_t e; cudaEventCreate(&e); return e;
   }
   ~Scope() {
+    nvtxRangePop();
     c->launches++;
     if (c->profile) { cudaEventRecord(b, s); c->timed.push_back({a, b, cls}); }
   }
