@@ -223,7 +223,10 @@ class ScaleKV:
             raise ScaleKVError(st, "scalekv_query_sizes")
         self.pool_bytes, self.workspace_bytes = pb.value, wb.value
         with torch.cuda.device(self.device):
-            self.pool = torch.empty(pb.value, dtype=torch.uint8, device=self.device)
+            # the library wants the pool 1024-byte and the workspace 256-byte aligned; the allocator only
+            # promises 512 bytes, so allocate a little more and start at the next boundary
+            self._pool_raw = torch.empty(pb.value + 1024, dtype=torch.uint8, device=self.device)
+            self.pool = self._pool_raw[(-self._pool_raw.data_ptr()) % 1024:][:pb.value]
             self.workspace = torch.empty(wb.value, dtype=torch.uint8, device=self.device)
             self.stream_main = torch.cuda.Stream(device=self.device)
             self.stream_side = torch.cuda.Stream(device=self.device) if side_stream else self.stream_main
