@@ -156,6 +156,14 @@ scalekv_status scalekv_compress(scalekv_ctx *ctx, int32_t layer, scalekv_tensor 
  *                axis before the selection ("average pooling", Sec. 3.3, read as smoothing along keys: zeros
  *                beyond both ends, always divided by the width; the neighbours are the entries next to it in
  *                the cache as it stands, window entries included).  0 or 1: none - the default reading.
+ *   head_shared  SCORE only.  1: one importance for all heads of a batch element ("a unified importance
+ *                metric", Sec. 3.3, read as shared between heads): the mean over the heads of the per-head
+ *                importance, entry by entry, taken before the pooling; every head then keeps the same
+ *                entries.  Needs the heads of a batch element to hold the same original positions, which is
+ *                the case when the layer was compressed this way from its first scale on; otherwise the
+ *                device status turns to SCALEKV_ERR_DEVICE_CHECK (reported by scalekv_sync, sticky) and
+ *                neither the selection nor the compaction runs.
+ *                0: per head - the default reading.
  * opts == NULL is scalekv_compress. */
 #define SCALEKV_SELECT_SCORE 0
 #define SCALEKV_SELECT_RECENT 1
@@ -163,6 +171,7 @@ typedef struct {
   int32_t policy;
   int32_t pool_kernel;
   int32_t n_sink;        /* RECENT only */
+  int32_t head_shared;   /* SCORE only */
 } scalekv_select_opts;
 scalekv_status scalekv_compress_ex(scalekv_ctx *ctx, int32_t layer, scalekv_tensor Qw, int32_t w, const int32_t *window_pos,
                                    int32_t qw_is_full_map, const scalekv_select_opts *opts);

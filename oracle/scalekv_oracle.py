@@ -251,6 +251,23 @@ class SliceCache:
         self.adopt(idx)
 
 
+def compress_head_shared(caches, Qws, window_pos, budget, pool_kernel=1):
+    """Sec. 3.3 with the "unified importance metric" read as shared between heads: the per-head
+    importances of the heads of one batch element are averaged entry by entry, (pooled,) and one
+    selection prunes every head's cache alike.  caches / Qws: one SliceCache / window query block per
+    head; the heads must hold the same original positions.  Returns (kept positions, importance)."""
+    first = caches[0]
+    for c in caches[1:]:
+        if not np.array_equal(c.pos, first.pos):
+            raise ValueError("head-shared selection needs the same entries in every head")
+    per_head = np.stack([c.scores(Qw) for c, Qw in zip(caches, Qws)], axis=0)
+    s = pool_scores(per_head.mean(axis=0), pool_kernel)
+    keep = select(s, first.pos, first.N[first.k - 1], window_pos, budget)
+    for c in caches:
+        c.adopt(keep)
+    return first.pos.copy(), s
+
+
 # --------------------------------------------------------------------------------------
 # Observation window geometry (Sec. 3.3: partition r_k into N patches, take each patch's
 # centroid token; "typically 16 tokens").

@@ -379,6 +379,34 @@ __global__ void __launch_bounds__(256) score_kernel(LayerView lv, WindowArg wa, 
   keys[(size_t)slice * ld_s + i] = win ? kWindowKey : (__float_as_uint(sc) & 0x7FFFFFFFu);
 }
 
+// Head-shared importance (Sec. 3.3, "a unified importance metric" read as shared between the heads of a
+// batch element): every entry's importance becomes the mean over the heads, summed in head order, and
+// the keys follow.  The heads must hold the same entries: equal lengths and equal original positions,
+// else the device status is raised and the selection that follows does not run.
+// grid (ceil(L_max / 256), B), 256 threads; scores and keys are [n_slices][ld_s].
+__global__ void __launch_bounds__(256) head_mean_kernel(LayerView lv, WindowArg wa, float *scores, uint32_t *keys, int ld_s) {
+  const int H = lv.n_heads;
+  const int s0 = blockIdx.y * H;
+  const int L = lv.hist_len[s0] + wa.n_k;
+  const int i = blockIdx.x * 256 + threadIdx.x;
+  if (blockIdx.x == 0 && threadIdx.x < H && lv.hist_len[s0 + threadIdx.x] + wa.n_k != L) atomicExch(lv.status, kDevCheck);
+  if (i >= L) return;
+  const int pos = lv.pos_pool[slot_row(lv, s0, i)];
+  float sum = 0.f;
+  bool same = true;
+  for (int h = 0; h < H; ++h) {
+    sum += scores[(size_t)(s0 + h) * ld_s + i];
+    same = same && (lv.hist_len[s0 + h] + wa.n_k <= i || lv.pos_pool[slot_row(lv, s0 + h, i)] == pos);
+  }
+  if (!same) atomicExch(lv.status, kDevCheck);
+  const float mean = sum * (1.f / (float)H);
+  const uint32_t key = is_window_pos(wa, pos) ? kWindowKey : (__float_as_uint(mean) & 0x7FFFFFFFu);
+  for (int h = 0; h < H; ++h) {
+    scores[(size_t)(s0 + h) * ld_s + i] = mean;
+    keys[(size_t)(s0 + h) * ld_s + i] = key;
+  }
+}
+
 // Keys of the positional keep rule (the comparison policies of Sec. 4.1: sliding window, sinks + recent
 // tokens): entries whose original position is below n_sink carry the sentinel (always kept), every
 // other entry competes on its position, most recent first.  grid (ceil(L_max / 256), n_slices).
@@ -467,6 +495,7 @@ __global__ void __launch_bounds__(1024) select_kernel(LayerView lv, WindowArg wa
   __shared__ int sh_remaining;
   const int tid = threadIdx.x, lane = tid & 31;
   const int slice = blockIdx.x;
+  if (*reinterpret_cast<volatile int *>(lv.status) != 0) return;   // an earlier kernel reported a failed check: leave the store alone
   const int L = lv.hist_len[slice] + wa.n_k;
   int *out = keep_list + (size_t)slice * ld_s;
 
@@ -608,6 +637,7 @@ __global__ void __launch_bounds__(256) compact_kernel(LayerView lv, const int *k
   const int which = blockIdx.y;
   const int quarter = blockIdx.z;
   char *pool = which == 0 ? lv.k_pool : lv.v_pool;
+  if (*reinterpret_cast<volatile int *>(lv.status) != 0) return;   // the selection did not run: nothing to move
   const int kept = kept_count[slice];
   for (int i = threadIdx.x; i < kept; i += 256) list[i] = __ldg(keep_list + (size_t)slice * ld_s + i);
   for (int i = threadIdx.x; i < lv.pages_per_slice; i += 256) pt[i] = __ldg(lv.page_table + (size_t)slice * lv.pages_per_slice + i);

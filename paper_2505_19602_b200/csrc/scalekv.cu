@@ -579,6 +579,7 @@ scalekv_status scalekv_compress_ex(scalekv_ctx *ctx, int32_t layer, scalekv_tens
   const int policy = opts ? opts->policy : SCALEKV_SELECT_SCORE;
   const int pool = (opts && opts->pool_kernel > 1) ? opts->pool_kernel : 1;
   const int n_sink = opts ? opts->n_sink : 0;
+  const bool head_shared = opts && opts->head_shared != 0 && (opts->policy == SCALEKV_SELECT_SCORE);
   if (policy != SCALEKV_SELECT_SCORE && policy != SCALEKV_SELECT_RECENT) return fail(ctx, SCALEKV_ERR_INVALID_ARG, "unknown selection policy %d", policy);
   if (pool % 2 == 0 || pool > 63) return fail(ctx, SCALEKV_ERR_INVALID_ARG, "pool_kernel must be odd and below 64");
   if (n_sink < 0) return fail(ctx, SCALEKV_ERR_INVALID_ARG, "n_sink must not be negative");
@@ -649,6 +650,10 @@ scalekv_status scalekv_compress_ex(scalekv_ctx *ctx, int32_t layer, scalekv_tens
     if (!recent) {
       Scope sc(ctx, s, kScore);
       score_kernel<<<dim3((L + 255) / 256, p.n_slices), 256, 0, s>>>(lv, wa, logits, wlse, p.ld_s, scores, keys, p.ld_s);
+    }
+    if (head_shared) {
+      Scope sc(ctx, s, kScore);
+      head_mean_kernel<<<dim3((L + 255) / 256, p.n_slices / p.H), 256, 0, s>>>(lv, wa, scores, keys, p.ld_s);
     }
     {
       Scope sc(ctx, s, kSelect);

@@ -430,3 +430,61 @@ def test_select_recent_brute_force_and_count_rule():
     # sliding window: the last entries; sinks + recent: the first n_sink and the last ones
     assert orc.select_recent(np.arange(10), 3).tolist() == [7, 8, 9]
     assert orc.select_recent(np.arange(10), 5, 2).tolist() == [0, 1, 7, 8, 9]
+
+
+def test_head_shared_compress_brute_force_and_special_cases():
+    """compress_head_shared against loops written here: attention of every window row to every entry
+    with math.exp, summed over rows and heads; the budget's largest non-window entries stay, ties
+    to the lowest position.  Special cases: one head, and identical heads, reduce to the per-head rule."""
+    rng = np.random.default_rng(21)
+    sides = (2, 3, 5)
+    n = orc.scale_token_counts(sides)
+    N = orc.cumulative_token_counts(n)
+    d, H, budget = 8, 3, 9
+    caches = [orc.SliceCache(n, d) for _ in range(H)]
+    solo = orc.SliceCache(n, d)          # head 0 alone, per-head rule
+    twins = [orc.SliceCache(n, d) for _ in range(2)]   # two copies of head 0, shared rule
+    diverged = False
+    for k in range(len(sides)):
+        Q = rng.normal(size=(H, n[k], d)); K = rng.normal(size=(H, n[k], d)); V = rng.normal(size=(H, n[k], d))
+        for h in range(H):
+            caches[h].append(K[h], V[h])
+        solo.append(K[0], V[0])
+        for c in twins:
+            c.append(K[0], V[0])
+        wpos = orc.window_centroids(sides[k], sides[k], 4)
+        pos = caches[0].pos.copy()
+        L = len(pos)
+        total = [0.0] * L
+        for h in range(H):
+            for i in wpos:
+                z = [sum(Q[h, i, e] * caches[h].K[j, e] for e in range(d)) / math.sqrt(d) for j in range(L)]
+                zmax = max(z)
+                ez = [math.exp(v - zmax) for v in z]
+                den = sum(ez)
+                for j in range(L):
+                    total[j] += ez[j] / den
+        win_abs = {N[k] + i for i in wpos}
+        cand = [j for j in range(L) if int(pos[j]) not in win_abs]
+        cand.sort(key=lambda j: (-total[j], pos[j]))
+        want = sorted(cand[:budget] + [j for j in range(L) if int(pos[j]) in win_abs])
+        got, s = orc.compress_head_shared(caches, [Q[h][wpos] for h in range(H)], wpos, budget)
+        assert got.tolist() == pos[want].tolist()
+        assert np.allclose(s, np.array(total) / (H * len(wpos)), rtol=1e-12, atol=1e-15)
+        for c in caches:
+            assert np.array_equal(c.pos, got)
+        # identical heads and a single head: the per-head rule
+        p_solo, _ = solo.compress(Q[0][wpos], wpos, budget)
+        p_twin, _ = orc.compress_head_shared(twins, [Q[0][wpos]] * 2, wpos, budget)
+        assert np.array_equal(p_solo, p_twin)
+        diverged = diverged or not np.array_equal(p_solo, got)
+    assert diverged          # the shared rule is not the per-head rule in disguise
+    # heads that hold different entries are refused
+    a, b = orc.SliceCache(n, d), orc.SliceCache(n, d)
+    for c in (a, b):
+        c.append(rng.normal(size=(n[0], d)), rng.normal(size=(n[0], d)))
+        c.append(rng.normal(size=(n[1], d)), rng.normal(size=(n[1], d)))
+    a.adopt(np.arange(1, len(a)))
+    b.adopt(np.arange(0, len(b) - 1))
+    with pytest.raises(ValueError):
+        orc.compress_head_shared([a, b], [rng.normal(size=(1, d))] * 2, [0], 2)

@@ -543,3 +543,78 @@ def test_step_host_pipeline_matches_device_calls():
     for l in range(L_layers):
         assert torch.equal(kv.scalekv_export_slice(l, 1, 0), want_pos[l])
     kv.close()
+
+
+@pytest.mark.parametrize("pool_kernel", [1, 5])
+def test_head_shared_importance_matches_oracle(pool_kernel):
+    """scalekv_compress_ex with head_shared: the mean over heads of the per-head importance decides for
+    all heads of a batch element; they keep identical entries, batch elements differ."""
+    sides = (2, 5, 9, 14, 19)
+    n = orc.scale_token_counts(sides)
+    N = orc.cumulative_token_counts(n)
+    budgets = [[60] * len(sides)]
+    B, H = 2, 4
+    kv = binding.ScaleKV(1, B, H, 128, "bf16", sides, sides, budgets, max_window=16)
+    wl = synth.Workload("hs", 1, B, H, 128, "bf16", sides, seed=35)
+    caches = [[orc.SliceCache(n, 128) for _ in range(H)] for _ in range(B)]
+    evictions, batch_differs = 0, False
+    for k in range(len(sides)):
+        Q, K, V = synth.scale_inputs(wl, 0, k)
+        Qd, Kd, Vd = Q.cuda(), K.cuda(), V.cuda()
+        torch.cuda.synchronize()
+        kv.scalekv_append(0, k, Kd, Vd)
+        O = kv.scalekv_attend(0, Qd)
+        wpos = orc.window_centroids(sides[k], sides[k], 16)
+        kv.scalekv_compress_ex(0, Qd, wpos, qw_is_full_map=True, policy="score", pool_kernel=pool_kernel, head_shared=True)
+        kv.scalekv_sync()
+        kept_of_batch = []
+        for b in range(B):
+            for h in range(H):
+                c = caches[b][h]
+                c.append(K[b, h].double().numpy(), V[b, h].double().numpy())
+                Oo, _ = c.attend(Q[b, h].double().numpy())
+                assert np.max(np.abs(Oo - O[b, h].double().cpu().numpy())) <= 2e-2
+            before = caches[b][0].pos.copy()
+            per_head = np.stack([caches[b][h].scores(Q[b, h].double().numpy()[wpos]) for h in range(H)])
+            s = orc.pool_scores(per_head.mean(axis=0), pool_kernel)
+            keep = orc.select(s, before, N[k], wpos, budgets[0][k])
+            got = [kv.scalekv_export_slice(0, b, h).numpy().astype(np.int64) for h in range(H)]
+            for h in range(1, H):
+                assert np.array_equal(got[h], got[0])          # exact: the heads share one decision
+            assert len(got[0]) == len(keep)
+            evictions += int(len(keep) < len(before))
+            assert _kept_or_tie(got[0], before, s, keep, [N[k] + p for p in wpos]), (k, b)
+            for h in range(H):
+                caches[b][h].adopt_positions(got[0])
+                pos, Kg, Vg = kv.scalekv_export_slice(0, b, h, with_kv=True)
+                assert np.array_equal(Kg.double().numpy(), caches[b][h].K) and np.array_equal(Vg.double().numpy(), caches[b][h].V)
+            kept_of_batch.append(got[0])
+        batch_differs = batch_differs or not np.array_equal(kept_of_batch[0], kept_of_batch[1])
+    assert evictions >= 4 and batch_differs
+    kv.close()
+
+
+def test_head_shared_importance_refuses_heads_that_diverged():
+    """After a per-head compress the heads hold different entries: the head-shared rule reports a
+    device check through the status word and leaves the store as it was."""
+    sides = (2, 5, 9, 14)
+    n = orc.scale_token_counts(sides)
+    budgets = [[40] * len(sides)]
+    kv = binding.ScaleKV(1, 1, 3, 128, "bf16", sides, sides, budgets, max_window=16)
+    wl = synth.Workload("hd", 1, 1, 3, 128, "bf16", sides, seed=36)
+    for k in range(len(sides)):
+        Q, K, V = synth.scale_inputs(wl, 0, k, device="cuda")
+        torch.cuda.synchronize()
+        kv.scalekv_append(0, k, K, V)
+        kv.scalekv_attend(0, Q)
+        wpos = orc.window_centroids(sides[k], sides[k], 16)
+        if k < 3:
+            kv.scalekv_compress(0, Q, wpos, qw_is_full_map=True)
+            kv.scalekv_sync()
+    kept = [kv.scalekv_export_slice(0, 0, h).numpy() for h in range(3)]
+    assert any(not np.array_equal(kept[0], kept[h]) for h in (1, 2))
+    kv.scalekv_compress_ex(0, Q, wpos, qw_is_full_map=True, policy="score", head_shared=True)
+    with pytest.raises(binding.ScaleKVError) as e:
+        kv.scalekv_sync()
+    assert e.value.status == binding.STATUS_NAMES.index("DEVICE_CHECK")
+    kv.close()
