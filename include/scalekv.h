@@ -163,7 +163,12 @@ scalekv_status scalekv_compress(scalekv_ctx *ctx, int32_t layer, scalekv_tensor 
  *                the case when the layer was compressed this way from its first scale on; otherwise the
  *                device status turns to SCALEKV_ERR_DEVICE_CHECK (reported by scalekv_sync, sticky) and
  *                neither the selection nor the compaction runs.
- *                0: per head - the default reading.
+ *                0: per head - the default reading.  At most 256 heads.
+ *   head_budgets HOST array [n_heads] or NULL.  Budgets of this call per head (the same for every batch
+ *                element) in place of budgets[layer][scale]: the store is ragged, so heads may keep
+ *                different numbers of entries.  Each value must lie in [0, budgets[layer][scale]] (the
+ *                pages were sized for the table's value); any value >= 0 when the table says KEEP_ALL.
+ *                With head_shared the heads must agree.  At most 128 heads.
  * opts == NULL is scalekv_compress. */
 #define SCALEKV_SELECT_SCORE 0
 #define SCALEKV_SELECT_RECENT 1
@@ -172,6 +177,7 @@ typedef struct {
   int32_t pool_kernel;
   int32_t n_sink;        /* RECENT only */
   int32_t head_shared;   /* SCORE only */
+  const int32_t *head_budgets;
 } scalekv_select_opts;
 scalekv_status scalekv_compress_ex(scalekv_ctx *ctx, int32_t layer, scalekv_tensor Qw, int32_t w, const int32_t *window_pos,
                                    int32_t qw_is_full_map, const scalekv_select_opts *opts);

@@ -44,7 +44,8 @@ class scalekv_config(C.Structure):
 
 
 class scalekv_select_opts(C.Structure):
-    _fields_ = [("policy", C.c_int32), ("pool_kernel", C.c_int32), ("n_sink", C.c_int32), ("head_shared", C.c_int32)]
+    _fields_ = [("policy", C.c_int32), ("pool_kernel", C.c_int32), ("n_sink", C.c_int32), ("head_shared", C.c_int32),
+                ("head_budgets", C.POINTER(C.c_int32))]
 
 
 class scalekv_tensor(C.Structure):
@@ -278,9 +279,10 @@ class ScaleKV:
             self._check(self.lib.scalekv_compress(self.ctx, layer, tensor_arg(Qw), len(window_pos), wp, int(qw_is_full_map)))
 
     def scalekv_compress_ex(self, layer, Qw=None, window_pos=None, qw_is_full_map=False, policy="score", pool_kernel=1,
-                            n_sink=0, head_shared=False):
+                            n_sink=0, head_shared=False, head_budgets=None):
         """scalekv_compress with a selection variant: policy "score" (optionally pooled) or "recent"."""
-        opts = scalekv_select_opts({"score": 0, "recent": 1}[policy], pool_kernel, n_sink, int(head_shared))
+        hb = _i32_array(head_budgets) if head_budgets is not None else None
+        opts = scalekv_select_opts({"score": 0, "recent": 1}[policy], pool_kernel, n_sink, int(head_shared), hb)
         q = tensor_arg(Qw) if Qw is not None else scalekv_tensor(None, 0, 0, 0)
         if window_pos is None:
             wp, w = None, 0

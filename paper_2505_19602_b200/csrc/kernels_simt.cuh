@@ -485,7 +485,12 @@ __global__ void __launch_bounds__(1024) row_lse_kernel(LayerView lv, WindowArg w
 //   consecutive entries, so two block scans order the whole list.  Deterministic.
 // Dynamic shared memory: 4 * ld_s bytes of keys.
 // ------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(1024) select_kernel(LayerView lv, WindowArg wa, int budget, const uint32_t *keys,
+constexpr int kMaxHeadBudgets = 128;
+struct HeadBudgets {     // per-head budgets of one compress call; on = 0: every slice takes the call's common budget
+  int on;
+  int v[kMaxHeadBudgets];
+};
+__global__ void __launch_bounds__(1024) select_kernel(LayerView lv, WindowArg wa, int budget, HeadBudgets hb, const uint32_t *keys,
                                                       const float *scores, int pool, int ld_s, int *keep_list,
                                                       int *kept_count) {
   extern __shared__ uint32_t key[];            // [L]
@@ -517,6 +522,7 @@ __global__ void __launch_bounds__(1024) select_kernel(LayerView lv, WindowArg wa
   int n_win;
   block_exclusive_scan(n_win_local, warp_sums, &n_win);
   const int cand = L - n_win;
+  if (hb.on) budget = hb.v[slice % lv.n_heads];
   const int kprime = (budget < 0 || budget > cand) ? cand : budget;
 
   // radix select of the kprime-th largest key

@@ -583,6 +583,9 @@ scalekv_status scalekv_compress_ex(scalekv_ctx *ctx, int32_t layer, scalekv_tens
   if (policy != SCALEKV_SELECT_SCORE && policy != SCALEKV_SELECT_RECENT) return fail(ctx, SCALEKV_ERR_INVALID_ARG, "unknown selection policy %d", policy);
   if (pool % 2 == 0 || pool > 63) return fail(ctx, SCALEKV_ERR_INVALID_ARG, "pool_kernel must be odd and below 64");
   if (n_sink < 0) return fail(ctx, SCALEKV_ERR_INVALID_ARG, "n_sink must not be negative");
+  if (head_shared && p.H > 256) return fail(ctx, SCALEKV_ERR_UNSUPPORTED, "head_shared supports at most 256 heads");
+  const int32_t *head_budgets = opts ? opts->head_budgets : nullptr;
+  if (head_budgets && p.H > kMaxHeadBudgets) return fail(ctx, SCALEKV_ERR_UNSUPPORTED, "head_budgets supports at most %d heads", kMaxHeadBudgets);
   const bool recent = policy == SCALEKV_SELECT_RECENT;
   const int k = ctx->next_scale[layer] - 1;
   const int L = ctx->hist[layer] + ctx->pending[layer];
@@ -603,8 +606,25 @@ scalekv_status scalekv_compress_ex(scalekv_ctx *ctx, int32_t layer, scalekv_tens
   const int cand = L - always_kept;
   const int table = p.budgets[(size_t)layer * p.K + k];
   // SCORE: k^l counts the selected entries, the window comes on top.  RECENT: k^l is the whole cache, sinks included.
-  const int budget = (recent && table != SCALEKV_KEEP_ALL) ? std::max(table - always_kept, 0) : table;
-  const bool evict = budget != SCALEKV_KEEP_ALL && budget < cand;
+  int budget = (recent && table != SCALEKV_KEEP_ALL) ? std::max(table - always_kept, 0) : table;
+  HeadBudgets hb{};
+  if (head_budgets) {
+    // per-head budgets of this call: the same conversion as for the table's value; the call's common
+    // budget becomes their maximum, which bounds the lengths the host assumes afterwards
+    int lo = 0x7fffffff, hi = 0;
+    for (int h = 0; h < p.H; ++h) {
+      const int b = head_budgets[h];
+      if (b < 0 || (table != SCALEKV_KEEP_ALL && b > table))
+        return fail(ctx, SCALEKV_ERR_INVALID_ARG, "head_budgets[%d] = %d outside [0, %d]", h, b, table);
+      hb.v[h] = recent ? std::max(b - always_kept, 0) : b;
+      lo = std::min(lo, hb.v[h]); hi = std::max(hi, hb.v[h]);
+    }
+    if (head_shared && lo != hi) return fail(ctx, SCALEKV_ERR_INVALID_ARG, "head_shared needs equal head_budgets");
+    hb.on = 1;
+    budget = std::min(hi, cand);
+    if (lo >= cand) hb.on = 0, budget = SCALEKV_KEEP_ALL;      // no head evicts anything
+  }
+  const bool evict = budget != SCALEKV_KEEP_ALL && (budget < cand || (hb.on != 0));
   // while per-kernel timing is on, compress runs on stream_main too, so that every kernel is timed alone
   cudaStream_t s = ctx->serialize ? ctx->s_main : ctx->s_side;
   const bool copy_now = !ctx->in_store[layer];
@@ -657,7 +677,7 @@ scalekv_status scalekv_compress_ex(scalekv_ctx *ctx, int32_t layer, scalekv_tens
     }
     {
       Scope sc(ctx, s, kSelect);
-      select_kernel<<<p.n_slices, 1024, (size_t)p.ld_s * 4, s>>>(lv, wa, budget, keys, recent ? nullptr : scores, pool, p.ld_s,
+      select_kernel<<<p.n_slices, 1024, (size_t)p.ld_s * 4, s>>>(lv, wa, budget, hb, keys, recent ? nullptr : scores, pool, p.ld_s,
                                                                  keep, kept);
     }
     {

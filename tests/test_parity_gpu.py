@@ -618,3 +618,62 @@ def test_head_shared_importance_refuses_heads_that_diverged():
         kv.scalekv_sync()
     assert e.value.status == binding.STATUS_NAMES.index("DEVICE_CHECK")
     kv.close()
+
+
+@pytest.mark.parametrize("policy", ["score", "recent"])
+def test_per_head_budgets_leave_a_ragged_store(policy):
+    """scalekv_compress_ex with head_budgets: every head prunes to its own budget (0 keeps only the
+    window, the table's value is the largest allowed), lengths differ between heads from then on and
+    the next scales' attention and selection still match the oracle slice by slice."""
+    sides = (2, 5, 9, 14, 19)
+    n = orc.scale_token_counts(sides)
+    N = orc.cumulative_token_counts(n)
+    table = 70
+    budgets = [[table] * len(sides)]
+    per_scale = [[10, 40, 70, 0], [10, 40, 70, 0], [30, 30, 70, 5], [5, 40, 60, 0], [70, 1, 20, 33]]
+    B, H = 2, 4
+    kv = binding.ScaleKV(1, B, H, 128, "bf16", sides, sides, budgets, max_window=16)
+    wl = synth.Workload("hb", 1, B, H, 128, "bf16", sides, seed=37)
+    caches = [[orc.SliceCache(n, 128) for _ in range(H)] for _ in range(B)]
+    ragged = False
+    for k in range(len(sides)):
+        Q, K, V = synth.scale_inputs(wl, 0, k)
+        Qd, Kd, Vd = Q.cuda(), K.cuda(), V.cuda()
+        torch.cuda.synchronize()
+        kv.scalekv_append(0, k, Kd, Vd)
+        O = kv.scalekv_attend(0, Qd)
+        wpos = orc.window_centroids(sides[k], sides[k], 16)
+        if policy == "score":
+            kv.scalekv_compress_ex(0, Qd, wpos, qw_is_full_map=True, policy="score", head_budgets=per_scale[k])
+        else:
+            kv.scalekv_compress_ex(0, policy="recent", n_sink=3, head_budgets=per_scale[k])
+        kv.scalekv_sync()
+        lens = kv.scalekv_lengths(0)
+        for b in range(B):
+            for h in range(H):
+                c = caches[b][h]
+                c.append(K[b, h].double().numpy(), V[b, h].double().numpy())
+                Oo, _ = c.attend(Q[b, h].double().numpy())
+                assert np.max(np.abs(Oo - O[b, h].double().cpu().numpy())) <= 2e-2, (k, b, h)
+                before = c.pos.copy()
+                got = kv.scalekv_export_slice(0, b, h).numpy().astype(np.int64)
+                if policy == "score":
+                    s = c.scores(Q[b, h].double().numpy()[wpos])
+                    keep = orc.select(s, before, N[k], wpos, per_scale[k][h])
+                    assert len(got) == len(keep) == min(per_scale[k][h] + len(wpos), len(before))
+                    assert _kept_or_tie(got, before, s, keep, [N[k] + p for p in wpos]), (k, b, h)
+                else:
+                    keep = orc.select_recent(before, per_scale[k][h], 3)
+                    assert np.array_equal(got, before[keep]), (k, b, h)
+                assert int(lens[b][h]) == len(got)
+                c.adopt_positions(got)
+                pos, Kg, Vg = kv.scalekv_export_slice(0, b, h, with_kv=True)
+                assert np.array_equal(Kg.double().numpy(), c.K) and np.array_equal(Vg.double().numpy(), c.V)
+        ragged = ragged or len({int(x) for x in lens[0]}) > 1
+    assert ragged
+    with pytest.raises(binding.ScaleKVError):      # above the table's value: the pages were not sized for it
+        kv.scalekv_reset()
+        Q, K, V = synth.scale_inputs(wl, 0, 0, device="cuda")
+        kv.scalekv_append(0, 0, K, V)
+        kv.scalekv_compress_ex(0, Q, [0, 1, 2, 3], qw_is_full_map=True, head_budgets=[71, 1, 1, 1])
+    kv.close()
