@@ -204,6 +204,16 @@ scalekv_status scalekv_step_host(scalekv_ctx *ctx, int32_t layer, int32_t scale,
 scalekv_status scalekv_layer_stats(scalekv_ctx *ctx, int32_t layer, scalekv_tensor Q, int32_t topk_prime,
                                    int32_t query_stride, double *car, double *htk);
 
+/* The same statistics, also per slice.  car_slices / htk_slices (HOST, [batch * n_heads], either may be
+ * NULL) receive the means of c_i and t_i over the sampled rows of each slice.  nca_slices (HOST,
+ * [batch * n_heads] or NULL) receives the "normalized current scale attention" of Sec. 4.3 per slice:
+ * the average attention a query gives to one token of the current map, c_i / n_k, over the average
+ * it gives to one entry of the whole sequence, 1 / L, averaged over the sampled rows, i.e.
+ * car_slice * L / n_k with L the slice's length (the distribution the paper plots over scales). */
+scalekv_status scalekv_layer_stats_ex(scalekv_ctx *ctx, int32_t layer, scalekv_tensor Q, int32_t topk_prime,
+                                      int32_t query_stride, double *car, double *htk, double *car_slices,
+                                      double *htk_slices, double *nca_slices);
+
 /* Sec. 3.3: the observation window = centroid token of each of N patches of an h x w map.
  * g = floor(sqrt(N)) patches per side, patch (a,b) = rows [a*h/g, (a+1)*h/g) x cols alike, centroid =
  * lower-middle cell; a map with at most N tokens is its own window.  pos (HOST, room for N entries)

@@ -325,6 +325,20 @@ def layer_stats_slice(Q, K, pos, n_prev, topk_prime, query_stride=1, softmax_sca
     return float(c.sum()), float(t.sum()), int(Q.shape[0])
 
 
+def normalized_current_attention(Q, K, pos, n_prev, query_stride=1, softmax_scale=None):
+    """Sec. 4.3, "normalized current scale attention" of one slice: for each sampled query the average
+    attention per token of the current map over the average attention per entry of the whole sequence,
+    (sum_{j in r_k} alpha_ij / n_k) / (sum_j alpha_ij / L), then the mean over the sampled queries."""
+    Q = np.asarray(Q, dtype=np.float64)[:: int(query_stride)]
+    K = np.asarray(K, dtype=np.float64)
+    pos = np.asarray(pos, dtype=np.int64)
+    scale = 1.0 / math.sqrt(Q.shape[1]) if not softmax_scale else float(softmax_scale)
+    A, _ = softmax_rows(scale * (Q @ K.T))
+    cur = pos >= int(n_prev)
+    per_query = (A[:, cur].sum(axis=1) / cur.sum()) / (A.sum(axis=1) / A.shape[1])
+    return float(per_query.mean())
+
+
 def asi_from_sums(sum_c, sum_t, count):
     """ASI = (mean current-attention ratio) * (mean history top-K' ratio)  (Eq. 2)."""
     car = sum_c / count

@@ -96,6 +96,7 @@ def load_library():
         "scalekv_compress_ex": [ctx_p, i32, T, i32, P(i32), i32, P(scalekv_select_opts)],
         "scalekv_step_host": [ctx_p, i32, i32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, i32, P(i32)],
         "scalekv_layer_stats": [ctx_p, i32, T, i32, i32, P(f64), P(f64)],
+        "scalekv_layer_stats_ex": [ctx_p, i32, T, i32, i32, P(f64), P(f64), P(f64), P(f64), P(f64)],
         "scalekv_window_centroids": [i32, i32, i32, P(i32), P(i32)],
         "scalekv_assign_roles": [P(f64), i32, i32, i32, i32, f64, P(C.c_uint8)],
         "scalekv_make_budgets": [P(C.c_uint8), i32, i32, f64, f64, f64, P(i32)],
@@ -306,6 +307,16 @@ class ScaleKV:
         self._check(self.lib.scalekv_layer_stats(self.ctx, layer, tensor_arg(Q), topk_prime, query_stride,
                                                  C.byref(car), C.byref(htk)))
         return car.value, htk.value
+
+    def scalekv_layer_stats_ex(self, layer, Q, topk_prime=16, query_stride=1):
+        """(car, htk, car per slice, htk per slice, normalized current attention per slice); lists are [B][H]."""
+        car, htk = C.c_double(0), C.c_double(0)
+        n = self.batch * self.n_heads
+        cs, ts, ns = (C.c_double * n)(), (C.c_double * n)(), (C.c_double * n)()
+        self._check(self.lib.scalekv_layer_stats_ex(self.ctx, layer, tensor_arg(Q), topk_prime, query_stride,
+                                                    C.byref(car), C.byref(htk), cs, ts, ns))
+        shape = lambda a: [[a[b * self.n_heads + h] for h in range(self.n_heads)] for b in range(self.batch)]
+        return car.value, htk.value, shape(cs), shape(ts), shape(ns)
 
     def scalekv_lengths(self, layer):
         out = (C.c_int32 * (self.batch * self.n_heads))()

@@ -773,6 +773,9 @@ __global__ void __launch_bounds__(256) layer_stats_kernel(LayerView lv, TensorVi
   if (threadIdx.x == 0) {
     atomicAdd(&acc[0], (double)cur);
     atomicAdd(&acc[1], (double)top);
+    // the same sums per slice, behind the two totals
+    atomicAdd(&acc[2 + 2 * blockIdx.y], (double)cur);
+    atomicAdd(&acc[3 + 2 * blockIdx.y], (double)top);
   }
 }
 

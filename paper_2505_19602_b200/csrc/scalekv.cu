@@ -155,7 +155,7 @@ scalekv_status make_plan(const scalekv_config *c, Plan &p, std::string &err) {
   p.off_keys = o; o = align_up(o + (size_t)p.n_slices * p.ld_s * 4, 1024);
   p.off_keep = o; o = align_up(o + (size_t)p.n_slices * p.ld_s * 4, 1024);
   p.off_kept = o; o = align_up(o + (size_t)p.n_slices * 4, 1024);
-  p.off_acc = o; o = align_up(o + 64, 1024);
+  p.off_acc = o; o = align_up(o + 16 + (size_t)p.n_slices * 16, 1024);
   p.ws_bytes = o;
   return SCALEKV_OK;
 }
@@ -759,6 +759,12 @@ scalekv_status scalekv_step_host(scalekv_ctx *ctx, int32_t layer, int32_t scale,
 
 scalekv_status scalekv_layer_stats(scalekv_ctx *ctx, int32_t layer, scalekv_tensor Q, int32_t topk_prime,
                                    int32_t query_stride, double *car, double *htk) {
+  return scalekv_layer_stats_ex(ctx, layer, Q, topk_prime, query_stride, car, htk, nullptr, nullptr, nullptr);
+}
+
+scalekv_status scalekv_layer_stats_ex(scalekv_ctx *ctx, int32_t layer, scalekv_tensor Q, int32_t topk_prime,
+                                      int32_t query_stride, double *car, double *htk, double *car_slices,
+                                      double *htk_slices, double *nca_slices) {
   if (!ctx || !car || !htk) return SCALEKV_ERR_INVALID_ARG;
   const Plan &p = ctx->plan;
   if (layer < 0 || layer >= p.n_layers) return fail(ctx, SCALEKV_ERR_INVALID_ARG, "layer %d out of range", layer);
@@ -772,7 +778,8 @@ scalekv_status scalekv_layer_stats(scalekv_ctx *ctx, int32_t layer, scalekv_tens
   const int L = ctx->hist[layer] + nk;
   const int rows = (nk + query_stride - 1) / query_stride;
   double *acc = reinterpret_cast<double *>(ctx->ws + p.off_acc);
-  CU(cudaMemsetAsync(acc, 0, 16, ctx->s_main));
+  const size_t acc_bytes = 16 + (size_t)p.n_slices * 16;
+  CU(cudaMemsetAsync(acc, 0, acc_bytes, ctx->s_main));
   {
     Scope sc(ctx, ctx->s_main, kOther);
     dim3 grid(rows, p.n_slices);
@@ -785,12 +792,22 @@ scalekv_status scalekv_layer_stats(scalekv_ctx *ctx, int32_t layer, scalekv_tens
   }
   scalekv_status st = check_launch(ctx, "layer_stats");
   if (st != SCALEKV_OK) return st;
-  double host[2];
-  CU(cudaMemcpyAsync(host, acc, 16, cudaMemcpyDeviceToHost, ctx->s_main));
+  std::vector<double> host(2 + 2 * (size_t)p.n_slices);
+  std::vector<int> len(p.n_slices);
+  CU(cudaMemcpyAsync(host.data(), acc, acc_bytes, cudaMemcpyDeviceToHost, ctx->s_main));
+  CU(cudaMemcpyAsync(len.data(), ctx->pool + p.off_len + (size_t)layer * p.n_slices * 4, (size_t)p.n_slices * 4,
+                     cudaMemcpyDeviceToHost, ctx->s_main));
   CU(cudaStreamSynchronize(ctx->s_main));
   const double cnt = (double)rows * p.n_slices;
   *car = host[0] / cnt;
   *htk = host[1] / cnt;
+  for (int s = 0; s < p.n_slices; ++s) {
+    const double c_s = host[2 + 2 * s] / rows, t_s = host[3 + 2 * s] / rows;
+    if (car_slices) car_slices[s] = c_s;
+    if (htk_slices) htk_slices[s] = t_s;
+    // the stored length does not count the map just appended until a compress commits it
+    if (nca_slices) nca_slices[s] = c_s * (double)(len[s] + nk) / (double)nk;
+  }
   return SCALEKV_OK;
 }
 

@@ -70,6 +70,9 @@ WORKLOADS = {
     "pass8b": Workload("pass8b", 40, 8, 32, 128, "bf16", SIDES_13, seed=4, n_drafters=10),
     # configs[4]: 16-scale stress
     "hires": Workload("hires", 32, 4, 16, 128, "bf16", SIDES_16, seed=5, n_drafters=8),
+    # the headline pass with the batch doubled, as under classifier-free guidance (a conditional and an
+    # unconditional branch per image run through the same layers)
+    "pass2b_cfg": Workload("pass2b_cfg", 32, 16, 16, 128, "bf16", SIDES_13, seed=6, n_drafters=8),
 }
 
 

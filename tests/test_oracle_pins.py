@@ -488,3 +488,29 @@ def test_head_shared_compress_brute_force_and_special_cases():
     b.adopt(np.arange(0, len(b) - 1))
     with pytest.raises(ValueError):
         orc.compress_head_shared([a, b], [rng.normal(size=(1, d))] * 2, [0], 2)
+
+
+def test_normalized_current_attention_closed_forms():
+    """Uniform attention gives 1; all mass on the current map gives L / n_k; none gives 0; and the
+    value is CAR * L / n_k computed with plain loops."""
+    rng = np.random.default_rng(8)
+    d, n_prev, nk = 8, 30, 12
+    L = n_prev + nk
+    pos = np.arange(L)
+    K = rng.normal(size=(L, d))
+    assert abs(orc.normalized_current_attention(np.zeros((nk, d)), K, pos, n_prev) - 1.0) < 1e-13
+    # keys of the current map aligned with the queries, scaled up: the mass moves onto the current map
+    big = np.zeros((L, d)); big[n_prev:, 0] = 50.0; big[:n_prev, 0] = -50.0
+    q = np.zeros((nk, d)); q[:, 0] = 10.0
+    assert abs(orc.normalized_current_attention(q, big, pos, n_prev) - L / nk) < 1e-9
+    assert orc.normalized_current_attention(-q, big, pos, n_prev) < 1e-9
+    Q = rng.normal(size=(nk, d))
+    total = 0.0
+    for i in range(0, nk, 3):
+        z = [sum(Q[i, e] * K[j, e] for e in range(d)) / math.sqrt(d) for j in range(L)]
+        zmax = max(z)
+        ez = [math.exp(v - zmax) for v in z]
+        total += sum(ez[n_prev:]) / sum(ez) * L / nk
+    assert abs(orc.normalized_current_attention(Q, K, pos, n_prev, query_stride=3) - total / 4) < 1e-12
+    sc, _, cnt = orc.layer_stats_slice(Q, K, pos, n_prev, 4, query_stride=3)
+    assert abs(orc.normalized_current_attention(Q, K, pos, n_prev, query_stride=3) - sc / cnt * L / nk) < 1e-12

@@ -1,6 +1,8 @@
 """GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same seeded
 inputs - attention outputs within the dtype's bound, kept index sets exact (or inside the stated
 tie band), compacted rows bit-exact."""
+import dataclasses
+
 import numpy as np
 import pytest
 import torch
@@ -177,6 +179,8 @@ def test_layer_stats_matches_oracle_and_recovers_planted_roles():
             torch.cuda.synchronize()
             kv.scalekv_append(l, k, Kd, Vd)
             car, htk = kv.scalekv_layer_stats(l, Qd, topk_prime=4, query_stride=2)
+            car2, htk2, car_s, htk_s, nca_s = kv.scalekv_layer_stats_ex(l, Qd, topk_prime=4, query_stride=2)
+            assert abs(car2 - car) < 1e-6 and abs(htk2 - htk) < 1e-6
             sc = st = cnt = 0
             for b in range(B):
                 for h in range(H):
@@ -184,6 +188,10 @@ def test_layer_stats_matches_oracle_and_recovers_planted_roles():
                     c.append(K[b, h].double().numpy(), V[b, h].double().numpy())
                     a = orc.layer_stats_slice(Q[b, h].double().numpy(), c.K, c.pos, N[k], 4, 2)
                     sc, st, cnt = sc + a[0], st + a[1], cnt + a[2]
+                    # per slice, and the normalized current attention of Sec. 4.3 (at most L / n_k)
+                    assert abs(car_s[b][h] - a[0] / a[2]) < 1e-4 and abs(htk_s[b][h] - a[1] / a[2]) < 1e-4
+                    nca = orc.normalized_current_attention(Q[b, h].double().numpy(), c.K, c.pos, N[k], 2)
+                    assert abs(nca_s[b][h] - nca) <= 1e-4 * len(c) / n[k]
             want_asi, want_car, want_htk = orc.asi_from_sums(sc, st, cnt)
             assert abs(car - want_car) < 1e-4 and abs(htk - want_htk) < 1e-4
             asi[l, k] = car * htk
@@ -676,4 +684,22 @@ def test_per_head_budgets_leave_a_ragged_store(policy):
         Q, K, V = synth.scale_inputs(wl, 0, 0, device="cuda")
         kv.scalekv_append(0, 0, K, V)
         kv.scalekv_compress_ex(0, Q, [0, 1, 2, 3], qw_is_full_map=True, head_budgets=[71, 1, 1, 1])
+    kv.close()
+
+
+def test_doubled_batch_two_layers_sampled_slices():
+    """The headline shape with the batch doubled (16 x 16 slices per layer), one drafter and one
+    refiner layer at full size; the oracle follows slices from both halves of the batch."""
+    wl = dataclasses.replace(synth.WORKLOADS["pass2b_cfg"], n_layers=2, n_drafters=1)
+    n = wl.n_tokens
+    planted = synth.drafter_layers(wl)
+    bd, br = orc.budget_tokens(0.30, n), orc.budget_tokens(0.03, n)
+    budgets = [[bd if l in planted else br] * wl.n_scales for l in range(wl.n_layers)]
+    kv = binding.ScaleKV(wl.n_layers, wl.batch, wl.n_heads, 128, "bf16", wl.sides, wl.sides, budgets, max_window=16)
+    slices = [(0, 1, 3), (0, 15, 15), (1, 8, 0), (1, 12, 9)]
+    run = ParityRun(kv, "bf16", wl.sides, budgets, lambda l, k: synth.scale_inputs(wl, l, k, device="cuda"),
+                    lambda k: orc.window_centroids(wl.sides[k], wl.sides[k], 16), slices, check_lse=False).run()
+    assert run.evictions > 0
+    lens = kv.scalekv_lengths(planted[0])
+    assert all(lens[b][h] == bd + 16 + n[-1] for b in (0, 15) for h in (0, 15))
     kv.close()
