@@ -313,7 +313,7 @@ def run_scalekv(args):
             ev0.record()
         for _ in range(n_pass):
             pipeline.run_pass(kv, inputs, windows)
-        kv.stream_main.wait_stream(kv.stream_side)
+        kv.scalekv_join()
         with torch.cuda.stream(kv.stream_main):
             ev1.record()
         kv.scalekv_sync()
@@ -339,6 +339,25 @@ def run_scalekv(args):
     clocks = sampler.stop()
     ms = max_over_ranks(ms, world, "cuda")
     value = job_throughput(wl.n_scales, args.steps, world, ms)
+
+    # per-scale-step latency: events on stream_main at the scale boundaries of the same passes (a scale-step's
+    # compress of its last layers may still run on the side stream when the next scale-step starts)
+    kv.scalekv_profile_enable(0)
+    per_pass = []
+    for _ in range(args.steps):
+        marks = []
+        pipeline.run_pass(kv, inputs, windows, marks=marks)
+        kv.scalekv_sync()
+        per_pass.append([marks[i].elapsed_time(marks[i + 1]) for i in range(len(marks) - 1)])
+    cols = list(zip(*per_pass))
+    scale_flop = work["per_scale_flop"]
+    per_scale = {"reset_ms_median": statistics.median(cols[0]),
+                 "scale_steps": [{"scale": k + 1, "n_k": wl.n_tokens[k], "ms_median": statistics.median(cols[k + 1]),
+                                  "ms_min": min(cols[k + 1]),
+                                  "attend_TFLOPps": scale_flop[k] / (statistics.median(cols[k + 1]) / 1e3) / 1e12}
+                                 for k in range(wl.n_scales)],
+                 "note": "CUDA events on stream_main at scale boundaries; one scale-step = append + attend + compress of "
+                         "every layer at that scale; attend_TFLOPps = the scale's attention flop over the step's time"}
 
     # the same passes once more with compress serialised onto stream_main: every kernel timed alone
     kv.scalekv_profile_enable(2)
@@ -434,7 +453,7 @@ def run_scalekv(args):
                        "l2_policy": f"inputs larger than L2: {inputs.bytes() / 1e9:.1f} GB of Q/K/V per pass",
                        "side_stream": not args.no_side_stream, "calibration_s": round(calib_s, 1),
                        "attend_kernel": "tcgen05" if os.environ.get("SCALEKV_ATTEND", "") != "simt" else "simt"},
-            "roofline": roofline, "kernels": kernels, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches,
+            "roofline": roofline, "kernels": kernels, "per_scale": per_scale, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches,
             "clocks": clocks, "work_per_pass": {k: v for k, v in work.items() if k != "per_scale_flop"},
         }
         print(json.dumps(line))

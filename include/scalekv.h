@@ -102,8 +102,12 @@ scalekv_status scalekv_init(const scalekv_config *cfg, scalekv_ctx **out);
 /* Empties every slice (start of a new image batch).  Enqueued on stream_main after both streams'
  * pending work.  The hot calls only enqueue kernels, memsets and event fork/joins between the two
  * streams, so a sequence reset, {append, attend, compress}... can be captured on stream_main into a
- * CUDA graph and replayed (join stream_side back into stream_main before ending the capture). */
+ * CUDA graph and replayed (call scalekv_join before ending the capture). */
 scalekv_status scalekv_reset(scalekv_ctx *ctx);
+
+/* Makes stream_main wait for everything enqueued so far on stream_side.  Only enqueues an event record
+ * and a wait: legal during a capture. */
+scalekv_status scalekv_join(scalekv_ctx *ctx);
 
 /* Waits for both streams and frees the host context.  Device memory stays with the caller. */
 scalekv_status scalekv_destroy(scalekv_ctx *ctx);

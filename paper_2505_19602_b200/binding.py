@@ -104,6 +104,7 @@ def load_library():
         "scalekv_export_slice": [ctx_p, i32, i32, i32, P(i32), C.c_void_p, C.c_void_p, i32, P(i32)],
         "scalekv_export_scores": [ctx_p, i32, i32, P(C.c_float), i32, P(i32)],
         "scalekv_sync": [ctx_p],
+        "scalekv_join": [ctx_p],
         "scalekv_launch_count": [ctx_p, P(i64)],
         "scalekv_profile_enable": [ctx_p, i32],
         "scalekv_profile_read": [ctx_p, i32, P(f64), P(i64)],
@@ -347,6 +348,9 @@ class ScaleKV:
 
     def scalekv_sync(self):
         self._check(self.lib.scalekv_sync(self.ctx))
+
+    def scalekv_join(self):
+        self._check(self.lib.scalekv_join(self.ctx))
 
     def scalekv_launch_count(self):
         n = C.c_int64(0)

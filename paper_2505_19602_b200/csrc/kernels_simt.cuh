@@ -500,8 +500,9 @@ __global__ void __launch_bounds__(1024) select_kernel(LayerView lv, WindowArg wa
   __shared__ int sh_remaining;
   const int tid = threadIdx.x, lane = tid & 31;
   const int slice = blockIdx.x;
-  if (*reinterpret_cast<volatile int *>(lv.status) != 0) return;   // an earlier kernel reported a failed check: leave the store alone
+  const int dev_status = *reinterpret_cast<volatile int *>(lv.status);   // both loads in flight before the test
   const int L = lv.hist_len[slice] + wa.n_k;
+  if (dev_status != 0) return;                 // an earlier kernel reported a failed check: leave the store alone
   int *out = keep_list + (size_t)slice * ld_s;
 
   int n_win_local = 0;
@@ -643,8 +644,9 @@ __global__ void __launch_bounds__(256) compact_kernel(LayerView lv, const int *k
   const int which = blockIdx.y;
   const int quarter = blockIdx.z;
   char *pool = which == 0 ? lv.k_pool : lv.v_pool;
-  if (*reinterpret_cast<volatile int *>(lv.status) != 0) return;   // the selection did not run: nothing to move
+  const int dev_status = *reinterpret_cast<volatile int *>(lv.status);   // both loads in flight before the test
   const int kept = kept_count[slice];
+  if (dev_status != 0) return;                 // the selection did not run: nothing to move
   for (int i = threadIdx.x; i < kept; i += 256) list[i] = __ldg(keep_list + (size_t)slice * ld_s + i);
   for (int i = threadIdx.x; i < lv.pages_per_slice; i += 256) pt[i] = __ldg(lv.page_table + (size_t)slice * lv.pages_per_slice + i);
   __syncthreads();

@@ -169,6 +169,7 @@ struct scalekv_ctx {
   float scale = 0.f;
   char *pool = nullptr, *ws = nullptr;
   cudaStream_t s_main = nullptr, s_side = nullptr;
+  cudaEvent_t ev_join = nullptr;   // scalekv_join: marks the side stream's progress
   // scalekv_step_host only: copy streams of the library's own and, per staging half, the events that chain them
   cudaStream_t s_h2d = nullptr, s_d2h = nullptr;
   cudaEvent_t ev_in[2] = {nullptr, nullptr}, ev_out[2] = {nullptr, nullptr}, ev_att[2] = {nullptr, nullptr};
@@ -374,6 +375,7 @@ scalekv_status scalekv_init(const scalekv_config *cfg, scalekv_ctx **out) {
   ctx->s_side = cfg->stream_side ? static_cast<cudaStream_t>(cfg->stream_side) : ctx->s_main;
   auto bail = [&](scalekv_status s) { delete ctx; return s; };
   if (cudaSetDevice(cfg->device) != cudaSuccess) return bail(SCALEKV_ERR_CUDA);
+  if (cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming) != cudaSuccess) return bail(SCALEKV_ERR_CUDA);
   int major = 0, minor = 0;
   cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, cfg->device);
   cudaDeviceGetAttribute(&minor, cudaDevAttrComputeCapabilityMinor, cfg->device);
@@ -464,6 +466,7 @@ scalekv_status scalekv_destroy(scalekv_ctx *ctx) {
   cudaStreamSynchronize(ctx->s_main);
   if (ctx->s_side != ctx->s_main) cudaStreamSynchronize(ctx->s_side);
   drain_profile(ctx);
+  if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
   if (ctx->s_h2d) { cudaStreamSynchronize(ctx->s_h2d); cudaStreamDestroy(ctx->s_h2d); }
   if (ctx->s_d2h) { cudaStreamSynchronize(ctx->s_d2h); cudaStreamDestroy(ctx->s_d2h); }
   for (int i = 0; i < 2; ++i) {
@@ -863,6 +866,15 @@ scalekv_status scalekv_make_budgets(const uint8_t *is_drafter, int32_t L, int32_
     const double bd = (b_uniform * L - nr * br) / nd;
     for (int l = 0; l < L; ++l)
       budgets_out[(size_t)l * K + k] = (int32_t)std::floor((is_drafter[(size_t)l * K + k] ? bd : br) + 0.5);
+  }
+  return SCALEKV_OK;
+}
+
+scalekv_status scalekv_join(scalekv_ctx *ctx) {
+  if (!ctx) return SCALEKV_ERR_INVALID_ARG;
+  if (ctx->s_side != ctx->s_main) {
+    CU(cudaEventRecord(ctx->ev_join, ctx->s_side));
+    CU(cudaStreamWaitEvent(ctx->s_main, ctx->ev_join, 0));
   }
   return SCALEKV_OK;
 }

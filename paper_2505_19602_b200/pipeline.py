@@ -78,10 +78,24 @@ class PassInputs:
         return total
 
 
-def run_pass(kv: binding.ScaleKV, inputs: PassInputs, windows, compress_last=False):
-    """One pass: reset, then for every scale and layer append -> attend -> compress."""
+def run_pass(kv: binding.ScaleKV, inputs: PassInputs, windows, compress_last=False, marks=None):
+    """One pass: reset, then for every scale and layer append -> attend -> compress.
+
+    marks: a list that receives CUDA events recorded on stream_main before the reset, after it, and after
+    every scale-step (2 + n_scales events), for per-scale-step latencies.
+    """
     wl = inputs.wl
+
+    def mark():
+        if marks is not None:
+            ev = torch.cuda.Event(enable_timing=True)
+            with torch.cuda.stream(kv.stream_main):
+                ev.record()
+            marks.append(ev)
+
+    mark()
     kv.scalekv_reset()
+    mark()
     for k in range(wl.n_scales):
         nk = wl.n_tokens[k]
         O = inputs.O[:, :, :nk, :]
@@ -95,6 +109,7 @@ def run_pass(kv: binding.ScaleKV, inputs: PassInputs, windows, compress_last=Fal
                     kv.scalekv_compress(l, Q, None)
                 else:
                     kv.scalekv_compress(l, Q, windows[k], qw_is_full_map=True)
+        mark()
 
 
 def pass_work(wl: synth.Workload, budgets, windows):

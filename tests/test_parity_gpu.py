@@ -389,7 +389,7 @@ def test_whole_pass_replays_from_a_cuda_graph():
     torch.cuda.synchronize()
     with torch.cuda.graph(g, stream=kv.stream_main):
         pipeline.run_pass(kv, inputs, windows)
-        kv.stream_main.wait_stream(kv.stream_side)
+        kv.scalekv_join()
     for _ in range(2):
         inputs.O.zero_()
         torch.cuda.synchronize()
