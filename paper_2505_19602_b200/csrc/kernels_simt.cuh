@@ -486,11 +486,17 @@ __global__ void __launch_bounds__(1024) row_lse_kernel(LayerView lv, WindowArg w
 // Dynamic shared memory: 4 * ld_s bytes of keys.
 // ------------------------------------------------------------------------------------------
 constexpr int kMaxHeadBudgets = 128;
-struct HeadBudgets {     // per-head budgets of one compress call; on = 0: every slice takes the call's common budget
-  int on;
+struct HeadBudgets {     // per-head budgets of one compress call
   int v[kMaxHeadBudgets];
 };
-__global__ void __launch_bounds__(1024) select_kernel(LayerView lv, WindowArg wa, int budget, HeadBudgets hb, const uint32_t *keys,
+// Spreads the per-head budgets of a compress call over the slices (slice = b * n_heads + h), so that the
+// select kernel reads its budget with one load instead of indexing a by-value table.
+__global__ void head_budget_kernel(HeadBudgets hb, int n_heads, int n_slices, int *slice_budget) {
+  const int s = blockIdx.x * blockDim.x + threadIdx.x;
+  if (s < n_slices) slice_budget[s] = hb.v[s % n_heads];
+}
+// slice_budget: per-slice budgets (nullptr: every slice takes `budget`).
+__global__ void __launch_bounds__(1024) select_kernel(LayerView lv, WindowArg wa, int budget, const int *slice_budget, const uint32_t *keys,
                                                       const float *scores, int pool, int ld_s, int *keep_list,
                                                       int *kept_count) {
   extern __shared__ uint32_t key[];            // [L]
@@ -523,7 +529,7 @@ __global__ void __launch_bounds__(1024) select_kernel(LayerView lv, WindowArg wa
   int n_win;
   block_exclusive_scan(n_win_local, warp_sums, &n_win);
   const int cand = L - n_win;
-  if (hb.on) budget = hb.v[slice % lv.n_heads];
+  if (slice_budget != nullptr) budget = slice_budget[slice];
   const int kprime = (budget < 0 || budget > cand) ? cand : budget;
 
   // radix select of the kprime-th largest key

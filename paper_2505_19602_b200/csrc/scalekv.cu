@@ -49,7 +49,7 @@ struct Plan {
   size_t off_k, off_v, off_pos, off_pt, off_len, off_status, pool_bytes;
   size_t pt_elems, logits_elems;
   // workspace layout
-  size_t off_logits, off_wlse, off_scores, off_keys, off_keep, off_kept, off_acc, ws_bytes;
+  size_t off_logits, off_wlse, off_scores, off_keys, off_keep, off_kept, off_hbud, off_acc, ws_bytes;
 };
 
 // Raster indices of the observation window of an h x w map (see scalekv_window_centroids).
@@ -155,6 +155,7 @@ scalekv_status make_plan(const scalekv_config *c, Plan &p, std::string &err) {
   p.off_keys = o; o = align_up(o + (size_t)p.n_slices * p.ld_s * 4, 1024);
   p.off_keep = o; o = align_up(o + (size_t)p.n_slices * p.ld_s * 4, 1024);
   p.off_kept = o; o = align_up(o + (size_t)p.n_slices * 4, 1024);
+  p.off_hbud = o; o = align_up(o + (size_t)p.n_slices * 4, 1024);
   p.off_acc = o; o = align_up(o + 16 + (size_t)p.n_slices * 16, 1024);
   p.ws_bytes = o;
   return SCALEKV_OK;
@@ -611,6 +612,7 @@ scalekv_status scalekv_compress_ex(scalekv_ctx *ctx, int32_t layer, scalekv_tens
   // SCORE: k^l counts the selected entries, the window comes on top.  RECENT: k^l is the whole cache, sinks included.
   int budget = (recent && table != SCALEKV_KEEP_ALL) ? std::max(table - always_kept, 0) : table;
   HeadBudgets hb{};
+  bool hb_on = false;
   if (head_budgets) {
     // per-head budgets of this call: the same conversion as for the table's value; the call's common
     // budget becomes their maximum, which bounds the lengths the host assumes afterwards
@@ -623,11 +625,11 @@ scalekv_status scalekv_compress_ex(scalekv_ctx *ctx, int32_t layer, scalekv_tens
       lo = std::min(lo, hb.v[h]); hi = std::max(hi, hb.v[h]);
     }
     if (head_shared && lo != hi) return fail(ctx, SCALEKV_ERR_INVALID_ARG, "head_shared needs equal head_budgets");
-    hb.on = 1;
+    hb_on = true;
     budget = std::min(hi, cand);
-    if (lo >= cand) hb.on = 0, budget = SCALEKV_KEEP_ALL;      // no head evicts anything
+    if (lo >= cand) hb_on = false, budget = SCALEKV_KEEP_ALL;      // no head evicts anything
   }
-  const bool evict = budget != SCALEKV_KEEP_ALL && (budget < cand || (hb.on != 0));
+  const bool evict = budget != SCALEKV_KEEP_ALL && (budget < cand || hb_on);
   // while per-kernel timing is on, compress runs on stream_main too, so that every kernel is timed alone
   cudaStream_t s = ctx->serialize ? ctx->s_main : ctx->s_side;
   const bool copy_now = !ctx->in_store[layer];
@@ -678,9 +680,15 @@ scalekv_status scalekv_compress_ex(scalekv_ctx *ctx, int32_t layer, scalekv_tens
       Scope sc(ctx, s, kScore);
       head_mean_kernel<<<dim3((L + 255) / 256, p.n_slices / p.H), 256, 0, s>>>(lv, wa, scores, keys, p.ld_s);
     }
+    int *slice_budget = nullptr;
+    if (hb_on) {
+      slice_budget = reinterpret_cast<int *>(ctx->ws + p.off_hbud);
+      Scope sc(ctx, s, kSelect);
+      head_budget_kernel<<<(p.n_slices + 255) / 256, 256, 0, s>>>(hb, p.H, p.n_slices, slice_budget);
+    }
     {
       Scope sc(ctx, s, kSelect);
-      select_kernel<<<p.n_slices, 1024, (size_t)p.ld_s * 4, s>>>(lv, wa, budget, hb, keys, recent ? nullptr : scores, pool, p.ld_s,
+      select_kernel<<<p.n_slices, 1024, (size_t)p.ld_s * 4, s>>>(lv, wa, budget, slice_budget, keys, recent ? nullptr : scores, pool, p.ld_s,
                                                                  keep, kept);
     }
     {
