@@ -22,12 +22,12 @@ class ParityRun:
     """
 
     def __init__(self, kv, dtype, sides, budgets, inputs_fn, window_fn, slices, compress_last=False,
-                 check_lse=True, max_rows=None):
+                 check_lse=True, max_rows=None, sides_w=None):
         self.kv, self.dtype, self.sides = kv, dtype, list(sides)
         self.budgets, self.inputs_fn, self.window_fn = budgets, inputs_fn, window_fn
         self.slices, self.compress_last, self.check_lse = slices, compress_last, check_lse
         self.max_rows = max_rows      # attention is compared on at most this many evenly spaced query rows per map
-        self.n = orc.scale_token_counts(self.sides)
+        self.n = orc.scale_token_counts(self.sides, sides_w)      # sides = heights when sides_w is given
         self.caches = {s: orc.SliceCache(self.n, kv.head_dim) for s in slices}
         self.resyncs = 0
         self.max_err = 0.0

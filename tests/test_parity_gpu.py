@@ -703,3 +703,47 @@ def test_doubled_batch_two_layers_sampled_slices():
     lens = kv.scalekv_lengths(planted[0])
     assert all(lens[b][h] == bd + 16 + n[-1] for b in (0, 15) for h in (0, 15))
     kv.close()
+
+
+def run_random_configuration(seed, max_side=20):
+    """One configuration drawn from a seeded generator, every slice followed by the oracle."""
+    rng = np.random.default_rng(4000 + seed)
+    K = int(rng.integers(3, 7))
+    sides_h = sorted(int(x) for x in rng.choice(np.arange(1, max_side + 1), size=K, replace=False))
+    if rng.random() < 0.5:
+        sides_w = list(sides_h)
+    else:
+        sides_w = [max(1, h + int(rng.integers(-2, 4))) for h in sides_h]
+    dtype, d = ("bf16", 128) if rng.random() < 0.75 else ("f32", 64)
+    n_layers, B, H = int(rng.integers(1, 4)), int(rng.integers(1, 3)), int(rng.integers(1, 4))
+    page_tokens = int(rng.choice([0, 16, 32, 64]))
+    patches = int(rng.choice([4, 9, 16]))
+    choices = [0, 3, 17, 50, 130, 400, binding.KEEP_ALL]
+    budgets = [[int(rng.choice(choices)) for _ in range(K)] for _ in range(n_layers)]
+    gain = float(rng.choice([1.0, 1.0, 3.0]))          # some runs with peaked attention
+    kv = binding.ScaleKV(n_layers, B, H, d, dtype, sides_h, sides_w, budgets, max_window=16, page_tokens=page_tokens,
+                         window_patches=patches)
+    n = orc.scale_token_counts(sides_h, sides_w)
+    gen = torch.Generator().manual_seed(9000 + seed)
+    tdt = synth.torch_dtype(dtype)
+
+    def inputs(l, k):
+        Q = (gain * torch.randn(B, H, n[k], d, generator=gen)).to(tdt)
+        Kt = torch.randn(B, H, n[k], d, generator=gen).to(tdt)
+        V = torch.randn(B, H, n[k], d, generator=gen).to(tdt)
+        return Q, Kt, V
+
+    slices = [(l, b, h) for l in range(n_layers) for b in range(B) for h in range(H)]
+    run = ParityRun(kv, dtype, sides_h, budgets, inputs, lambda k: orc.window_centroids(sides_h[k], sides_w[k], patches),
+                    slices, compress_last=bool(rng.random() < 0.5), sides_w=sides_w).run()
+    assert run.max_err <= {"bf16": 2e-2, "f32": 1e-4}[dtype]
+    kv.close()
+    return run
+
+
+@pytest.mark.parametrize("seed", range(10))
+def test_seeded_random_configurations(seed):
+    """Shapes drawn from a seeded generator: number of scales, square and rectangular maps, layers, batch,
+    heads, dtype, page size, window size, and a budget per (layer, scale) anywhere between 0 and KEEP_ALL
+    (also growing again after a small one)."""
+    run_random_configuration(seed)
