@@ -747,3 +747,20 @@ def test_seeded_random_configurations(seed):
     heads, dtype, page size, window size, and a budget per (layer, scale) anywhere between 0 and KEEP_ALL
     (also growing again after a small one)."""
     run_random_configuration(seed)
+
+
+@pytest.mark.parametrize("dtype,d", [("bf16", 128), ("f32", 64)])
+def test_largest_window_of_64_centroids(dtype, d):
+    """The largest observation window the library takes (64 rows = 8 x 8 patches), recorded by attend."""
+    sides = (4, 10, 17, 24)
+    n = orc.scale_token_counts(sides)
+    budgets = [[100] * len(sides), [binding.KEEP_ALL, 30, 30, 30]]
+    kv = binding.ScaleKV(2, 1, 2, d, dtype, sides, sides, budgets, max_window=64, window_patches=64)
+    gen = torch.Generator().manual_seed(77)
+    tdt = synth.torch_dtype(dtype)
+    inputs = lambda l, k: tuple(torch.randn(1, 2, n[k], d, generator=gen).to(tdt) for _ in range(3))
+    slices = [(l, 0, h) for l in range(2) for h in range(2)]
+    run = ParityRun(kv, dtype, sides, budgets, inputs, lambda k: orc.window_centroids(sides[k], sides[k], 64), slices,
+                    compress_last=True).run()
+    assert len(orc.window_centroids(24, 24, 64)) == 64 and run.evictions >= 8
+    kv.close()
