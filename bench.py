@@ -307,17 +307,22 @@ def run_scalekv(args):
             dist.barrier()
         torch.cuda.synchronize()
 
+    pass_marks = []
+
     def timed_passes(n_pass):
-        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        with torch.cuda.stream(kv.stream_main):
-            ev0.record()
-        for _ in range(n_pass):
+        # one event per pass boundary on stream_main (a pass starts with a reset, which joins the side
+        # stream): the region as a whole gives the reported time, the boundaries its spread
+        marks = [torch.cuda.Event(enable_timing=True) for _ in range(n_pass + 1)]
+        for i in range(n_pass):
+            with torch.cuda.stream(kv.stream_main):
+                marks[i].record()
             pipeline.run_pass(kv, inputs, windows)
         kv.scalekv_join()
         with torch.cuda.stream(kv.stream_main):
-            ev1.record()
+            marks[n_pass].record()
         kv.scalekv_sync()
-        return ev0.elapsed_time(ev1)
+        pass_marks[:] = [marks[i].elapsed_time(marks[i + 1]) for i in range(n_pass)]
+        return marks[0].elapsed_time(marks[n_pass])
 
     for _ in range(args.warmup):
         pipeline.run_pass(kv, inputs, windows)
@@ -329,6 +334,7 @@ def run_scalekv(args):
     ms = timed_passes(args.steps)
     barrier()
     launches = kv.scalekv_launch_count() - launches0
+    pass_spread = {"min": min(pass_marks), "median": statistics.median(pass_marks), "max": max(pass_marks)}
     # the same region again with CUDA events around every launch, each on the stream it is launched on:
     # the attend durations measured here (compress overlapping on the side stream, as in the timed
     # passes) feed the roofline object; the events themselves cost a few per cent, so `value` comes
@@ -444,7 +450,7 @@ def run_scalekv(args):
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-            "ms_per_step": pass_ms, "passes_per_sec": args.steps * world / (ms / 1000.0), "higher_is_better": True,
+            "ms_per_step": pass_ms, "ms_per_step_spread": pass_spread, "passes_per_sec": args.steps * world / (ms / 1000.0), "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
             "config": {"workload": wl.name, "layers": wl.n_layers, "batch": wl.batch, "heads": wl.n_heads,
                        "head_dim": wl.head_dim, "scales": wl.n_scales, "tokens": sum(wl.n_tokens),
