@@ -374,7 +374,13 @@ scalekv_status scalekv_init(const scalekv_config *cfg, scalekv_ctx **out) {
   ctx->pool = static_cast<char *>(cfg->pool); ctx->ws = static_cast<char *>(cfg->workspace);
   ctx->s_main = static_cast<cudaStream_t>(cfg->stream_main);
   ctx->s_side = cfg->stream_side ? static_cast<cudaStream_t>(cfg->stream_side) : ctx->s_main;
-  auto bail = [&](scalekv_status s) { delete ctx; return s; };
+  auto bail = [&](scalekv_status s) {     // a failed init gives back what it had created so far
+    if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
+    for (auto e : ctx->ev_attend) if (e) cudaEventDestroy(e);
+    for (auto e : ctx->ev_compress) if (e) cudaEventDestroy(e);
+    delete ctx;
+    return s;
+  };
   if (cudaSetDevice(cfg->device) != cudaSuccess) return bail(SCALEKV_ERR_CUDA);
   if (cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming) != cudaSuccess) return bail(SCALEKV_ERR_CUDA);
   int major = 0, minor = 0;
