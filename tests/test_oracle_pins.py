@@ -41,6 +41,9 @@ def test_token_count_closed_forms():
     N = orc.cumulative_token_counts(n13)
     assert sum(n * Nk for n, Nk in zip(n13, N[1:])) == 68484681
     assert sum(n * n for n in n13) == 26277921
+    # rectangular maps: h_k * w_k tokens per scale (Sec. 3.1 writes r_k as an h_k x w_k map)
+    assert orc.scale_token_counts((1, 2, 3, 5), (2, 3, 5, 4)) == [2, 6, 15, 20]
+    assert orc.cumulative_token_counts([2, 6, 15, 20]) == [0, 2, 8, 23, 43]
 
 
 def test_table1_accounting():
