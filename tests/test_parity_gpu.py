@@ -764,3 +764,30 @@ def test_largest_window_of_64_centroids(dtype, d):
                     compress_last=True).run()
     assert len(orc.window_centroids(24, 24, 64)) == 64 and run.evictions >= 8
     kv.close()
+
+
+@pytest.mark.parametrize("name,wrong", [("attend", "attend_without_scale"), ("select", "select_smallest"),
+                                        ("window_scores", "scores_sum_not_mean")])
+def test_parity_harness_notices_a_wrong_oracle(monkeypatch, name, wrong):
+    """The comparison itself must bite: with a mistake planted in the oracle (CPU side only) the same
+    run that passes otherwise has to fail."""
+    import test_oracle_mutations as mut
+    sides = (2, 5, 9, 14)
+    n = orc.scale_token_counts(sides)
+    budgets = [[40] * len(sides)]
+
+    def run():
+        kv = binding.ScaleKV(1, 1, 2, 128, "bf16", sides, sides, budgets, max_window=16)
+        gen = torch.Generator().manual_seed(5)
+        inputs = lambda l, k: tuple(torch.randn(1, 2, n[k], 128, generator=gen).to(torch.bfloat16) for _ in range(3))
+        try:
+            ParityRun(kv, "bf16", sides, budgets, inputs, lambda k: orc.window_centroids(sides[k], sides[k], 16),
+                      [(0, 0, 0), (0, 0, 1)]).run()
+        finally:
+            kv.close()
+
+    run()                                            # passes against the oracle as it stands
+    fn = mut.select_variant(smallest=True) if wrong == "select_smallest" else getattr(mut, wrong)
+    monkeypatch.setattr(orc, name, fn)
+    with pytest.raises(AssertionError):
+        run()
