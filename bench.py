@@ -51,6 +51,8 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-side-stream", action="store_true")
+    ap.add_argument("--no-graph", action="store_true",
+                    help="launch the timed passes call by call instead of replaying a CUDA graph of one pass")
     ap.add_argument("--cpu-sample-slices", type=int, default=16)
     return ap.parse_args()
 
@@ -309,14 +311,17 @@ def run_scalekv(args):
 
     pass_marks = []
 
-    def timed_passes(n_pass):
+    def timed_passes(n_pass, graph=None):
         # one event per pass boundary on stream_main (a pass starts with a reset, which joins the side
         # stream): the region as a whole gives the reported time, the boundaries its spread
         marks = [torch.cuda.Event(enable_timing=True) for _ in range(n_pass + 1)]
         for i in range(n_pass):
             with torch.cuda.stream(kv.stream_main):
                 marks[i].record()
-            pipeline.run_pass(kv, inputs, windows)
+                if graph is not None:
+                    graph.replay()
+            if graph is None:
+                pipeline.run_pass(kv, inputs, windows)
         kv.scalekv_join()
         with torch.cuda.stream(kv.stream_main):
             marks[n_pass].record()
@@ -327,13 +332,28 @@ def run_scalekv(args):
     for _ in range(args.warmup):
         pipeline.run_pass(kv, inputs, windows)
     kv.scalekv_sync()
+    # A pass is the same sequence of launches every time (the schedule, the budgets and the buffers are
+    # fixed), so it is captured once into a CUDA graph - stream_main plus the side stream that compress
+    # forks to - and the timed region replays it: the GPU is then never waiting for the host.
+    graph = None
+    launches0 = kv.scalekv_launch_count()
+    if not args.no_graph:
+        graph = torch.cuda.CUDAGraph()
+        torch.cuda.synchronize()
+        with torch.cuda.graph(graph, stream=kv.stream_main):
+            pipeline.run_pass(kv, inputs, windows)
+            kv.scalekv_join()
+        with torch.cuda.stream(kv.stream_main):
+            graph.replay()                         # one untimed replay
+        kv.scalekv_sync()
+    launches_per_pass = kv.scalekv_launch_count() - launches0
     launches0 = kv.scalekv_launch_count()
     sampler = ClockSampler(local_rank)
     barrier()
     sampler.start()
-    ms = timed_passes(args.steps)
+    ms = timed_passes(args.steps, graph)
     barrier()
-    launches = kv.scalekv_launch_count() - launches0
+    launches = launches_per_pass * args.steps if graph is not None else kv.scalekv_launch_count() - launches0
     pass_spread = {"min": min(pass_marks), "median": statistics.median(pass_marks), "max": max(pass_marks)}
     # the same region again with CUDA events around every launch, each on the stream it is launched on:
     # the attend durations measured here (compress overlapping on the side stream, as in the timed
@@ -457,7 +477,7 @@ def run_scalekv(args):
                        "budget": role_note + (f"; overall {args.overall_pct} %" if args.overall_pct > 0 else ""),
                        "window": wl.window, "parallelism": f"replica x{world} (batch-sharded, no collective)",
                        "l2_policy": f"inputs larger than L2: {inputs.bytes() / 1e9:.1f} GB of Q/K/V per pass",
-                       "side_stream": not args.no_side_stream, "calibration_s": round(calib_s, 1),
+                       "side_stream": not args.no_side_stream, "cuda_graph": not args.no_graph, "calibration_s": round(calib_s, 1),
                        "attend_kernel": "tcgen05" if os.environ.get("SCALEKV_ATTEND", "") != "simt" else "simt"},
             "roofline": roofline, "kernels": kernels, "per_scale": per_scale, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches,
             "clocks": clocks, "work_per_pass": {k: v for k, v in work.items() if k != "per_scale_flop"},
