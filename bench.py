@@ -296,9 +296,12 @@ def run_scalekv(args):
         role_note = "uniform 10%"
     calib_s = time.perf_counter() - t0
 
-    kv = binding.ScaleKV(wl.n_layers, wl.batch, wl.n_heads, wl.head_dim, wl.dtype, wl.sides, wl.sides, budgets,
-                         max_window=min(wl.window, binding.MAX_WINDOW), device=local_rank,
-                         side_stream=not args.no_side_stream)
+    def make_kv():
+        return binding.ScaleKV(wl.n_layers, wl.batch, wl.n_heads, wl.head_dim, wl.dtype, wl.sides, wl.sides, budgets,
+                               max_window=min(wl.window, binding.MAX_WINDOW), device=local_rank,
+                               side_stream=not args.no_side_stream)
+
+    kv = make_kv()
     inputs = pipeline.PassInputs(wl, device=local_rank)
     work = pipeline.pass_work(wl, budgets, windows)
     torch.cuda.synchronize()
@@ -335,17 +338,28 @@ def run_scalekv(args):
     # A pass is the same sequence of launches every time (the schedule, the budgets and the buffers are
     # fixed), so it is captured once into a CUDA graph - stream_main plus the side stream that compress
     # forks to - and the timed region replays it: the GPU is then never waiting for the host.
-    graph = None
+    graph, graph_note = None, "off (--no-graph)"
     launches0 = kv.scalekv_launch_count()
     if not args.no_graph:
-        graph = torch.cuda.CUDAGraph()
-        torch.cuda.synchronize()
-        with torch.cuda.graph(graph, stream=kv.stream_main):
+        try:
+            graph = torch.cuda.CUDAGraph()
+            torch.cuda.synchronize()
+            # thread_local: other threads (a process group's watchdog under torchrun) may call CUDA meanwhile
+            with torch.cuda.graph(graph, stream=kv.stream_main, capture_error_mode="thread_local"):
+                pipeline.run_pass(kv, inputs, windows)
+                kv.scalekv_join()
+            with torch.cuda.stream(kv.stream_main):
+                graph.replay()                         # one untimed replay
+            kv.scalekv_sync()
+            graph_note = "on"
+        except Exception as exc:                       # a capture that did not go through: start over, call by call
+            graph, graph_note = None, f"off (capture failed: {type(exc).__name__})"
+            torch.cuda.synchronize()
+            kv.close()
+            kv = make_kv()
             pipeline.run_pass(kv, inputs, windows)
-            kv.scalekv_join()
-        with torch.cuda.stream(kv.stream_main):
-            graph.replay()                         # one untimed replay
-        kv.scalekv_sync()
+            kv.scalekv_sync()
+            launches0 = kv.scalekv_launch_count()
     launches_per_pass = kv.scalekv_launch_count() - launches0
     launches0 = kv.scalekv_launch_count()
     sampler = ClockSampler(local_rank)
@@ -477,7 +491,7 @@ def run_scalekv(args):
                        "budget": role_note + (f"; overall {args.overall_pct} %" if args.overall_pct > 0 else ""),
                        "window": wl.window, "parallelism": f"replica x{world} (batch-sharded, no collective)",
                        "l2_policy": f"inputs larger than L2: {inputs.bytes() / 1e9:.1f} GB of Q/K/V per pass",
-                       "side_stream": not args.no_side_stream, "cuda_graph": not args.no_graph, "calibration_s": round(calib_s, 1),
+                       "side_stream": not args.no_side_stream, "cuda_graph": graph_note, "calibration_s": round(calib_s, 1),
                        "attend_kernel": "tcgen05" if os.environ.get("SCALEKV_ATTEND", "") != "simt" else "simt"},
             "roofline": roofline, "kernels": kernels, "per_scale": per_scale, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches,
             "clocks": clocks, "work_per_pass": {k: v for k, v in work.items() if k != "per_scale_flop"},
