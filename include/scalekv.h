@@ -186,6 +186,13 @@ typedef struct {
 scalekv_status scalekv_compress_ex(scalekv_ctx *ctx, int32_t layer, scalekv_tensor Qw, int32_t w, const int32_t *window_pos,
                                    int32_t qw_is_full_map, const scalekv_select_opts *opts);
 
+/* One whole step for one layer from DEVICE tensors, in one call: scalekv_append(K, V), scalekv_attend(Q -> O
+ * [, lse]) and, with the window rows taken from Q (the full current map), scalekv_compress.
+ * w > 0: window_pos holds w raster indices; w < 0: the whole current map is the window; w == 0: no
+ * compress.  Same contracts as the three calls; saves two trips through the binding per step. */
+scalekv_status scalekv_step(scalekv_ctx *ctx, int32_t layer, int32_t scale, scalekv_tensor Q, scalekv_tensor K,
+                            scalekv_tensor V, scalekv_tensor O, float *lse, int32_t w, const int32_t *window_pos);
+
 /* One whole step for one layer from HOST memory (pinned memory recommended): copies Q, K, V
  * (dense [B][H][n_k][d]) to `staging`, runs append, attend and compress with the window rows
  * taken from Q (w > 0: explicit window_pos; w < 0: the whole map is the window; w == 0: no

@@ -94,6 +94,7 @@ def load_library():
         "scalekv_attend": [ctx_p, i32, T, T, C.c_void_p],
         "scalekv_compress": [ctx_p, i32, T, i32, P(i32), i32],
         "scalekv_compress_ex": [ctx_p, i32, T, i32, P(i32), i32, P(scalekv_select_opts)],
+        "scalekv_step": [ctx_p, i32, i32, T, T, T, T, P(C.c_float), i32, P(i32)],
         "scalekv_step_host": [ctx_p, i32, i32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, i32, P(i32)],
         "scalekv_layer_stats": [ctx_p, i32, T, i32, i32, P(f64), P(f64)],
         "scalekv_layer_stats_ex": [ctx_p, i32, T, i32, i32, P(f64), P(f64), P(f64), P(f64), P(f64)],
@@ -291,6 +292,25 @@ class ScaleKV:
         else:
             wp, w = _i32_array(window_pos), len(window_pos)
         self._check(self.lib.scalekv_compress_ex(self.ctx, layer, q, w, wp, int(qw_is_full_map), C.byref(opts)))
+
+    def scalekv_step(self, layer, scale, Q, K, V, O, window_pos=None, whole_map=False, lse=None):
+        """append + attend + compress (window rows taken from Q) in one call; window_pos None and not whole_map: no compress.
+        window_pos may be a prepared ctypes int32 array (see window_array)."""
+        if whole_map:
+            w, wp = -1, None
+        elif window_pos is None:
+            w, wp = 0, None
+        else:
+            wp = window_pos if isinstance(window_pos, C.Array) else _i32_array(window_pos)
+            w = len(wp)
+        lp = C.cast(lse.data_ptr(), C.POINTER(C.c_float)) if lse is not None else None
+        self._check(self.lib.scalekv_step(self.ctx, layer, scale, tensor_arg(Q), tensor_arg(K), tensor_arg(V), tensor_arg(O),
+                                          lp, w, wp))
+
+    @staticmethod
+    def window_array(window_pos):
+        """The window as the ctypes array the calls take, so that a loop need not rebuild it."""
+        return _i32_array(window_pos)
 
     def scalekv_step_host(self, layer, scale, Qh, Kh, Vh, Oh, staging, window_pos=None, whole_map=False):
         if whole_map:

@@ -774,6 +774,17 @@ scalekv_status scalekv_step_host(scalekv_ctx *ctx, int32_t layer, int32_t scale,
   return SCALEKV_OK;
 }
 
+scalekv_status scalekv_step(scalekv_ctx *ctx, int32_t layer, int32_t scale, scalekv_tensor Q, scalekv_tensor K, scalekv_tensor V,
+                            scalekv_tensor O, float *lse, int32_t w, const int32_t *window_pos) {
+  scalekv_status st = scalekv_append(ctx, layer, scale, K, V);
+  if (st != SCALEKV_OK) return st;
+  st = scalekv_attend(ctx, layer, Q, O, lse);
+  if (st != SCALEKV_OK) return st;
+  if (w > 0) return scalekv_compress(ctx, layer, Q, w, window_pos, 1);
+  if (w < 0) return scalekv_compress(ctx, layer, Q, 0, nullptr, 1);
+  return SCALEKV_OK;
+}
+
 scalekv_status scalekv_layer_stats(scalekv_ctx *ctx, int32_t layer, scalekv_tensor Q, int32_t topk_prime,
                                    int32_t query_stride, double *car, double *htk) {
   return scalekv_layer_stats_ex(ctx, layer, Q, topk_prime, query_stride, car, htk, nullptr, nullptr, nullptr);

@@ -78,8 +78,9 @@ class PassInputs:
         return total
 
 
-def run_pass(kv: binding.ScaleKV, inputs: PassInputs, windows, compress_last=False, marks=None):
-    """One pass: reset, then for every scale and layer append -> attend -> compress.
+def run_pass(kv: binding.ScaleKV, inputs: PassInputs, windows, compress_last=False, marks=None, three_calls=False):
+    """One pass: reset, then for every scale and layer append -> attend -> compress (one scalekv_step per
+    layer and scale, or the three calls one by one with three_calls=True: the same launches either way).
 
     marks: a list that receives CUDA events recorded on stream_main before the reset, after it, and after
     every scale-step (2 + n_scales events), for per-scale-step latencies.
@@ -100,8 +101,13 @@ def run_pass(kv: binding.ScaleKV, inputs: PassInputs, windows, compress_last=Fal
         nk = wl.n_tokens[k]
         O = inputs.O[:, :, :nk, :]
         last = k + 1 == wl.n_scales
+        do_compress = not last or compress_last
+        wp = kv.window_array(windows[k]) if (do_compress and windows[k] is not None) else None
         for l in range(wl.n_layers):
             Q, K, V = inputs.data[(l, k)]
+            if not three_calls:
+                kv.scalekv_step(l, k, Q, K, V, O, window_pos=wp, whole_map=do_compress and wp is None)
+                continue
             kv.scalekv_append(l, k, K, V)
             kv.scalekv_attend(l, Q, O)
             if not last or compress_last:

@@ -791,3 +791,25 @@ def test_parity_harness_notices_a_wrong_oracle(monkeypatch, name, wrong):
     monkeypatch.setattr(orc, name, fn)
     with pytest.raises(AssertionError):
         run()
+
+
+def test_one_call_step_equals_the_three_calls():
+    """scalekv_step (append + attend + compress in one call) leaves exactly what the three calls leave."""
+    from paper_2505_19602_b200 import pipeline
+    sides = (2, 4, 7, 11, 16)
+    wl = synth.Workload("st", 2, 2, 2, 128, "bf16", sides, seed=41)
+    budgets = [[60] * len(sides), [25] * len(sides)]
+    windows = pipeline.windows_for(sides, 16)
+    results = []
+    for three in (True, False):
+        kv = binding.ScaleKV(2, 2, 2, 128, "bf16", sides, sides, budgets, max_window=16)
+        inputs = pipeline.PassInputs(wl)
+        pipeline.run_pass(kv, inputs, windows, compress_last=True, three_calls=three)
+        kv.scalekv_sync()
+        kept = [kv.scalekv_export_slice(l, b, h, with_kv=True) for l in range(2) for b in range(2) for h in range(2)]
+        results.append((inputs.O.clone(), kept, kv.scalekv_launch_count()))
+        kv.close()
+    (O3, kept3, n3), (O1, kept1, n1) = results
+    assert torch.equal(O3, O1) and n3 == n1
+    for a, b in zip(kept3, kept1):
+        assert all(torch.equal(x, y) for x, y in zip(a, b))
