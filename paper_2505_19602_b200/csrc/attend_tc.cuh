@@ -368,8 +368,8 @@ struct Params {
   int box_rows;        // rows per K/V TMA box = min(page_tokens, 128)
   int fused_append;    // 1: the current map's K/V rows are still in the caller's tensors; read them there and copy them in
   int n_prev;          // original position of the current map's first token
-  // observation window (Sec. 3.3): when win_logits is not null, the base-2 logits scale * log2(e) * <q, k>
-  // of the w window rows against every cache entry are recorded in win_logits[slice][rank][slot]
+  // observation window (Sec. 3.3): when win_logits is not null, the raw products <q, k> of the w window rows
+  // against every cache entry are recorded in win_logits[slice][rank][column], column = 128 j + position in key tile j
   float *win_logits;
   float *win_lse;      // [slice][rank]: base-2 log-sum-exp of each window row's logits (its softmax normaliser)
   int ld_l;            // leading dimension of a logit row
@@ -668,12 +668,14 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           float *x = v[cc & 1];
           if (wwarp[qt]) {
             if (wrank[qt] >= 0) {
-              // slot of this chunk's first column: history tiles start at 128 j, current-map tiles behind the history
-              const int slot0 = (j < Th ? j * 128 : hist + (j - Th) * 128) + part * kCols + cc * 32;
-              float *dst = prm.win_logits + ((size_t)slice * prm.w + wrank[qt]) * prm.ld_l + slot0;
+              // The row's raw products go out as they are (the score kernel applies the softmax scale), 32
+              // columns as eight 16-byte stores, at column 128 j + ...: key tile j owns columns [128 j, 128 j + 128)
+              // of a logit row, so the current map starts at the next multiple of 128 behind the history and
+              // every store is aligned.  Columns of a ragged tile beyond its keys hold finite values nobody reads.
+              const int col0 = j * 128 + part * kCols + cc * 32;
+              float4 *dst = reinterpret_cast<float4 *>(prm.win_logits + ((size_t)slice * prm.w + wrank[qt]) * prm.ld_l + col0);
 #pragma unroll
-              for (int i = 0; i < 32; ++i)
-                if (cc * 32 + i < valid) dst[i] = x[i] * c;
+              for (int i = 0; i < 8; ++i) dst[i] = make_float4(x[4 * i], x[4 * i + 1], x[4 * i + 2], x[4 * i + 3]);
             }
             __syncwarp();   // the tcgen05 instructions that follow want the warp converged
           }

@@ -351,18 +351,24 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int *warp_sums, int *
   return warp_sums[wid] + incl - v;
 }
 
+// logit_scale: what turns a stored logit into a base-2 logit (1 when the logits kernel wrote them, softmax scale *
+// log2(e) when attend recorded raw products).  tile_padded: attend recorded them while the current map was
+// not in the store yet, so its entries sit behind the history rounded up to a multiple of 128 columns.
 __global__ void __launch_bounds__(256) score_kernel(LayerView lv, WindowArg wa, const float *logits, const float *lse,
-                                                    int ld_l, float *scores, uint32_t *keys, int ld_s) {
+                                                    int ld_l, float logit_scale, int tile_padded, float *scores, uint32_t *keys,
+                                                    int ld_s) {
   __shared__ float lse_row[kMaxWindow];
   const int slice = blockIdx.y;
-  const int L = lv.hist_len[slice] + wa.n_k;
+  const int hist = lv.hist_len[slice];
+  const int L = hist + wa.n_k;
   const int i = blockIdx.x * 256 + threadIdx.x;
   if (blockIdx.x * 256 >= L) return;
   const int w = wa.w;
   if (threadIdx.x < w) lse_row[threadIdx.x] = lse[(size_t)slice * w + threadIdx.x];
   __syncthreads();
   if (i >= L) return;
-  const float *y = logits + (size_t)slice * w * ld_l + i;
+  const int col = (tile_padded && i >= hist) ? (((hist + 127) >> 7) << 7) + (i - hist) : i;
+  const float *y = logits + (size_t)slice * w * ld_l + col;
   float sc = 0.f;
   int j = 0;
   for (; j + 8 <= w; j += 8) {
@@ -370,9 +376,9 @@ __global__ void __launch_bounds__(256) score_kernel(LayerView lv, WindowArg wa, 
 #pragma unroll
     for (int e = 0; e < 8; ++e) t[e] = __ldg(y + (size_t)(j + e) * ld_l);
 #pragma unroll
-    for (int e = 0; e < 8; ++e) sc += exp2f(t[e] - lse_row[j + e]);
+    for (int e = 0; e < 8; ++e) sc += exp2f(fmaf(t[e], logit_scale, -lse_row[j + e]));
   }
-  for (; j < w; ++j) sc += exp2f(__ldg(y + (size_t)j * ld_l) - lse_row[j]);
+  for (; j < w; ++j) sc += exp2f(fmaf(__ldg(y + (size_t)j * ld_l), logit_scale, -lse_row[j]));
   sc *= 1.f / (float)w;
   scores[(size_t)slice * ld_s + i] = sc;
   const bool win = is_window_pos(wa, lv.pos_pool[slot_row(lv, slice, i)]);

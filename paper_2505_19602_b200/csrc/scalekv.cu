@@ -44,6 +44,7 @@ struct Plan {
   int trans_first[2] = {0, 0};
   long long n_pages = 0;
   int ld_s = 0;                     // padded max length (leading dimension of per-slice scratch)
+  int ld_l = 0;                     // leading dimension of a logit row: room for the history rounded up to a key tile and a ragged last tile
   int n_max = 0;
   // pool layout (byte offsets)
   size_t off_k, off_v, off_pos, off_pt, off_len, off_status, pool_bytes;
@@ -138,6 +139,7 @@ scalekv_status make_plan(const scalekv_config *c, Plan &p, std::string &err) {
   p.n_pages = page;
   p.pt_elems = pt;
   p.ld_s = (int)align_up((size_t)len_max, 64);
+  p.ld_l = (int)align_up((size_t)len_max + 256, 64);
   const size_t row_bytes = (size_t)p.d * p.esize;
   size_t o = 0;
   p.off_k = o; o = align_up(o + (size_t)p.n_pages * p.P * row_bytes, 1024);
@@ -148,7 +150,7 @@ scalekv_status make_plan(const scalekv_config *c, Plan &p, std::string &err) {
   p.off_status = o; o = align_up(o + 256, 1024);
   p.pool_bytes = o;
   o = 0;
-  p.logits_elems = (size_t)p.n_slices * p.max_window * p.ld_s;   // one buffer per layer parity
+  p.logits_elems = (size_t)p.n_slices * p.max_window * p.ld_l;   // one buffer per layer parity
   p.off_logits = o; o = align_up(o + 2 * p.logits_elems * 4, 1024);
   p.off_wlse = o; o = align_up(o + 2 * (size_t)p.n_slices * p.max_window * 4, 1024);   // one per layer parity
   p.off_scores = o; o = align_up(o + (size_t)p.n_slices * p.ld_s * 4, 1024);
@@ -183,6 +185,7 @@ struct scalekv_ctx {
   std::vector<int> pending;        // n_k of an appended, not yet committed current map (0 = none)
   std::vector<int> attended;       // attend ran for the pending map
   std::vector<char> in_store;      // the pending map's rows have been copied into the pages
+  std::vector<char> logits_padded; // attend recorded the logits while the current map was still outside the store
   std::vector<int> logits_of;      // scale whose window logits attend recorded for this layer (-1: none)
   std::vector<scalekv_tensor> pend_k, pend_v;   // the caller's tensors of a pending map that is not in the store yet
   std::vector<cudaEvent_t> ev_attend, ev_compress;
@@ -411,6 +414,7 @@ scalekv_status scalekv_init(const scalekv_config *cfg, scalekv_ctx **out) {
   ctx->attended.assign(p.n_layers, 0);
   ctx->in_store.assign(p.n_layers, 1);
   ctx->logits_of.assign(p.n_layers, -1);
+  ctx->logits_padded.assign(p.n_layers, 0);
   ctx->pend_k.resize(p.n_layers); ctx->pend_v.resize(p.n_layers);
   ctx->ev_attend.resize(p.n_layers); ctx->ev_compress.resize(p.n_layers);
   ctx->ev_compress_live.assign(p.n_layers, 0);
@@ -556,10 +560,11 @@ scalekv_status scalekv_attend(scalekv_ctx *ctx, int32_t layer, scalekv_tensor Q,
       float *wl = win.empty() ? nullptr : reinterpret_cast<float *>(ctx->ws + p.off_logits) + (size_t)(layer & 1) * p.logits_elems;
       float *wlse = reinterpret_cast<float *>(ctx->ws + p.off_wlse) + (size_t)(layer & 1) * p.n_slices * p.max_window;
       if (!ctx->tc.launch(lv, tview(Q), tview(O), lse, nk, fused ? &kc : nullptr, fused ? &vc : nullptr, p.N[k], ctx->scale, wl,
-                          wlse, p.ld_s, win.data(), (int)win.size(), ctx->s_main, e))
+                          wlse, p.ld_l, win.data(), (int)win.size(), ctx->s_main, e))
         return fail(ctx, SCALEKV_ERR_CUDA, "attend launch: %s", e.c_str());
       ctx->in_store[layer] = 1;
       ctx->logits_of[layer] = wl ? k : -1;
+      ctx->logits_padded[layer] = fused ? 1 : 0;
     } else {
       dim3 grid((nk + 63) / 64, p.n_slices);
       if (ctx->dtype == SCALEKV_BF16)
@@ -667,20 +672,22 @@ scalekv_status scalekv_compress_ex(scalekv_ctx *ctx, int32_t layer, scalekv_tens
       dim3 grid((L + 63) / 64, p.n_slices);
       if (ctx->dtype == SCALEKV_BF16)
         score_logits_kernel<__nv_bfloat16, 128><<<grid, 256, 2 * 64 * 132 * 4, s>>>(lv, tview(Qw), wa, qw_is_full_map, logits,
-                                                                                  p.ld_s, ctx->scale);
+                                                                                  p.ld_l, ctx->scale);
       else
-        score_logits_kernel<float, 64><<<grid, 256, 2 * 64 * 68 * 4, s>>>(lv, tview(Qw), wa, qw_is_full_map, logits, p.ld_s,
+        score_logits_kernel<float, 64><<<grid, 256, 2 * 64 * 68 * 4, s>>>(lv, tview(Qw), wa, qw_is_full_map, logits, p.ld_l,
                                                                          ctx->scale);
     }
     ctx->logits_of[layer] = -1;
     float *wlse = reinterpret_cast<float *>(ctx->ws + p.off_wlse) + (size_t)(layer & 1) * p.n_slices * p.max_window;
     if (!recorded) {
       Scope sc(ctx, s, kScore);
-      row_lse_kernel<<<p.n_slices, 1024, 0, s>>>(lv, wa, logits, p.ld_s, wlse);
+      row_lse_kernel<<<p.n_slices, 1024, 0, s>>>(lv, wa, logits, p.ld_l, wlse);
     }
     if (!recent) {
       Scope sc(ctx, s, kScore);
-      score_kernel<<<dim3((L + 255) / 256, p.n_slices), 256, 0, s>>>(lv, wa, logits, wlse, p.ld_s, scores, keys, p.ld_s);
+      // logits recorded by attend are raw products in the tile-aligned layout; the logits kernel writes base-2 logits by slot
+      score_kernel<<<dim3((L + 255) / 256, p.n_slices), 256, 0, s>>>(lv, wa, logits, wlse, p.ld_l, recorded ? ctx->scale * 1.4426950408889634f : 1.f,
+                                                                     (recorded && ctx->logits_padded[layer]) ? 1 : 0, scores, keys, p.ld_s);
     }
     if (head_shared) {
       Scope sc(ctx, s, kScore);
