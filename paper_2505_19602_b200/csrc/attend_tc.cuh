@@ -56,8 +56,9 @@ constexpr uint32_t kSmemBytes = kOffX + 128 + 2 * 4 * kParts * 32 * 4;
 static_assert(kSmemBytes <= 232448, "more shared memory than a CTA can have");
 // barrier slots (8 bytes each): one full/empty pair per ring stage, one S/P/PV barrier per S buffer or query tile
 enum { bQFull = 0, bFull = 1, bEmpty = bFull + kStages, bSFull = bEmpty + kStages, bPFull = bSFull + 2, bPvDone = bPFull + 2,
-       bPair = bPvDone + 2, bFinal = bPair + 4, bCount = bFinal + 2 };
-static_assert(bCount * 8 <= 192, "barriers overlap the TMEM slot");
+       bPair = bPvDone + 2, bFinal = bPair + 4, bOut = bFinal + 2, bCount = bOut + 2 };
+constexpr uint32_t kOffTmemSlot = 208;            // inside the barrier area, behind the barriers
+static_assert(bCount * 8 <= kOffTmemSlot, "barriers overlap the TMEM slot");
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColS = 0, kColO = 256;       // S/P buffers at 0 and 128, O accumulators at 256 and 384
 constexpr int kPolyPairs = 1;                   // of every 4 pairs of exponentials, this many run on the FMA pipe
@@ -125,6 +126,16 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *tm,
       "l"(tm), "r"(x), "r"(y), "r"(z), "r"(w), "r"(bar)
       : "memory");
 }
+
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap *tm, uint32_t src, int x, int y, int z, int w) {
+  asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];" ::"l"(tm), "r"(src), "r"(x), "r"(y),
+               "r"(z), "r"(w)
+               : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+// orders this thread's shared-memory writes before later reads of the asynchronous (TMA) proxy
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 // True in exactly one lane of a converged warp.
 __device__ __forceinline__ bool elect_one() {
@@ -380,13 +391,13 @@ struct Params {
 __global__ void __launch_bounds__(kThreads, 1)
 attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                  const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmKc,
-                 const __grid_constant__ CUtensorMap tmVc, const Params prm) {
+                 const __grid_constant__ CUtensorMap tmVc, const __grid_constant__ CUtensorMap tmO, const Params prm) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = smem_u32(smem_raw);
   uint8_t *base_ptr = smem_raw;
   const uint32_t bars = base + kOffBar;
-  volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(base_ptr + kOffBar + 192);
-  volatile int *abort_flag = reinterpret_cast<volatile int *>(base_ptr + kOffBar + 196);
+  volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(base_ptr + kOffBar + kOffTmemSlot);
+  volatile int *abort_flag = reinterpret_cast<volatile int *>(base_ptr + kOffBar + kOffTmemSlot + 4);
   auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -433,10 +444,11 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     }
     for (int s = 0; s < 4; ++s) mbar_init(bar(bPair + s), 32 * kParts);
     for (int s = 0; s < 2; ++s) mbar_init(bar(bFinal + s), 1);
+    for (int s = 0; s < 2; ++s) mbar_init(bar(bOut + s), 128 * kParts);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(base + kOffBar + 192), "r"(kTmemCols)
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(base + kOffBar + kOffTmemSlot), "r"(kTmemCols)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -758,29 +770,47 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       tc_fence_after();
       const float inv = 1.f / lsum;
       const int qi = q_first + qt * 128 + row;
-      __nv_bfloat16 *orow = const_cast<__nv_bfloat16 *>(row_ptr<__nv_bfloat16>(prm.O, b, h, qi < n_k ? qi : 0)) + part * kCols;
       float o[kChunks][32];
 #pragma unroll
       for (int cc = 0; cc < kChunks; ++cc) tc_ld32(lane_addr + kColO + qt * 128 + part * kCols + cc * 32, o[cc]);
       tc_wait_ld();
-      if (qi < n_k) {
+      // The normalised rows go to the query tile's shared memory (no product reads it any more) in the layout
+      // of a TMA box - two halves of 64 columns, rows of 128 bytes, 128-byte swizzle - and one thread sends the
+      // tile out with two bulk tensor stores: a row written by its own thread straight to global memory costs a
+      // 128-byte line per lane and store instruction.  The tensor map clips the rows beyond n_k.
+      static_assert(kCols == 64, "one softmax part = one 64-column half of the output tile");
+      const uint32_t stage = base + kOffQ + qt * kTileBytes + part * kHalfBytes + row * 128;
 #pragma unroll
-        for (int cc = 0; cc < kChunks; ++cc) {
+      for (int cc = 0; cc < kChunks; ++cc) {
 #pragma unroll
-          for (int v4 = 0; v4 < 4; ++v4) {
-            uint4 w;
-            w.x = pack_bf16(o[cc][8 * v4 + 0] * inv, o[cc][8 * v4 + 1] * inv);
-            w.y = pack_bf16(o[cc][8 * v4 + 2] * inv, o[cc][8 * v4 + 3] * inv);
-            w.z = pack_bf16(o[cc][8 * v4 + 4] * inv, o[cc][8 * v4 + 5] * inv);
-            w.w = pack_bf16(o[cc][8 * v4 + 6] * inv, o[cc][8 * v4 + 7] * inv);
-            reinterpret_cast<uint4 *>(orow + cc * 32)[v4] = w;
-          }
+        for (int v4 = 0; v4 < 4; ++v4) {
+          const uint32_t wx = pack_bf16(o[cc][8 * v4 + 0] * inv, o[cc][8 * v4 + 1] * inv);
+          const uint32_t wy = pack_bf16(o[cc][8 * v4 + 2] * inv, o[cc][8 * v4 + 3] * inv);
+          const uint32_t wz = pack_bf16(o[cc][8 * v4 + 4] * inv, o[cc][8 * v4 + 5] * inv);
+          const uint32_t ww = pack_bf16(o[cc][8 * v4 + 6] * inv, o[cc][8 * v4 + 7] * inv);
+          const uint32_t addr = stage + ((uint32_t)((cc * 4 + v4) ^ (row & 7)) << 4);
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(wx), "r"(wy), "r"(wz), "r"(ww) : "memory");
         }
+      }
+      fence_proxy_async();
+      mbar_arrive(bar(bOut + qt));
+      if (warp == 4) {
+        // one warp waits until all rows of the tile are staged; one of its lanes issues the stores
+        ok = mbar_wait_warp(bar(bOut + qt), 0, abort_flag, status);
+        if (!ok) break;
+        if (elect_one()) {
+          const uint32_t src = base + kOffQ + qt * kTileBytes;
+          tma_store_4d(&tmO, src, 0, q_first + qt * 128, h, b);
+          tma_store_4d(&tmO, src + kHalfBytes, 64, q_first + qt * 128, h, b);
+          tma_store_commit();
+        }
+        __syncwarp();
       }
       if (prm.lse != nullptr && part == 0 && qi < n_k)
         prm.lse[(size_t)slice * n_k + qi] = (m_used[qt] + log2f(lsum)) * 0.6931471805599453f;
       if (wrank[qt] >= 0 && part == 0) prm.win_lse[(size_t)slice * prm.w + wrank[qt]] = m_used[qt] + log2f(lsum);
     }
+    if (warp == 4) tma_store_wait_all();      // (a lane that issued nothing has nothing to wait for)
     tc_fence_before();
   }
   __syncthreads();
@@ -853,9 +883,10 @@ struct AttendTc {
   bool launch(const LayerView &lv, const TensorView &Q, const TensorView &O, float *lse, int n_k, const TensorView *Kc,
               const TensorView *Vc, int n_prev, float scale, float *win_logits, float *win_lse, int ld_l, const int *win_pos, int w,
               cudaStream_t stream, std::string &err) {
-    CUtensorMap tmQ, tmKc, tmVc;
+    CUtensorMap tmQ, tmKc, tmVc, tmO;
     const int B = lv.n_slices / lv.n_heads;
     if (!map_rows(&tmQ, Q, n_k, lv.n_heads, B, "Q", err)) return false;
+    if (!map_rows(&tmO, O, n_k, lv.n_heads, B, "O", err)) return false;
     const bool fused = Kc != nullptr && Vc != nullptr;
     if (fused) {
       if (!map_rows(&tmKc, *Kc, n_k, lv.n_heads, B, "K", err) || !map_rows(&tmVc, *Vc, n_k, lv.n_heads, B, "V", err)) return false;
@@ -875,7 +906,7 @@ struct AttendTc {
     prm.w = win_logits ? w : 0;
     for (int e = 0; e < kMaxWindow; ++e) prm.win_pos[e] = (win_logits && e < w) ? win_pos[e] : -1;
     dim3 grid((n_k + 255) / 256, lv.n_slices);
-    tc::attend_tc_kernel<<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(tmQ, tmK, tmV, tmKc, tmVc, prm);
+    tc::attend_tc_kernel<<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(tmQ, tmK, tmV, tmKc, tmVc, tmO, prm);
     return true;
   }
 };
