@@ -6,6 +6,7 @@ import torch
 from oracle import scalekv_oracle as orc
 
 TOL = {"bf16": 2e-2, "f32": 1e-4}   # max-abs bound on attention outputs
+REL = {"bf16": 2.0 ** -7, "f32": 0.0}    # relative part of the bound (see _compare_slice)
 TIE_BAND = 1e-3                     # relative score band inside which either choice is accepted
 
 
@@ -31,6 +32,7 @@ class ParityRun:
         self.caches = {s: orc.SliceCache(self.n, kv.head_dim) for s in slices}
         self.resyncs = 0
         self.max_err = 0.0
+        self.max_tol = 0.0
         self.max_lse_err = 0.0
         self.evictions = 0
 
@@ -81,7 +83,11 @@ class ParityRun:
             O, lse = cache.attend(Q)
         err = float(np.max(np.abs(O - O_gpu)))
         self.max_err = max(self.max_err, err)
-        assert err <= TOL[self.dtype], f"slice {key} scale {k}: attention max-abs error {err}"
+        # bf16: two roundings to 8 significant bits (P, then O), each at most 2^-9 relative: beyond |O| = 2.56 the
+        # bound that follows from the arithmetic, 2^-7 max|O|, is larger than the 2e-2 quoted for unit-scale outputs
+        tol = max(TOL[self.dtype], REL[self.dtype] * float(np.max(np.abs(O))))
+        self.max_tol = max(self.max_tol, tol)
+        assert err <= tol, f"slice {key} scale {k}: attention max-abs error {err} (bound {tol})"
         if self.check_lse:
             le = float(np.max(np.abs(lse - lse_gpu)))
             self.max_lse_err = max(self.max_lse_err, le)
