@@ -21,7 +21,10 @@
 //                         (tcgen05.st), from where the PV product takes its A operand.  The warps of a
 //                         quarter meet on an mbarrier per tile: only when a part's sum shows that an
 //                         exponent left the lazy band (2^8) do they recompute the row against a new
-//                         reference and rescale O.  At the end the same warps normalise and store O.
+//                         reference and rescale O.  Threads that own a row of the observation window also
+//                         store that row's raw products (16-byte stores, key tile j in columns 128 j ..) for
+//                         the compress that follows.  At the end the same warps normalise O, stage each tile
+//                         in the query tile's shared memory and one thread sends it out with TMA stores.
 //                         (Four warps per quarter, 16 softmax warps, measured the same as two.)
 //   warps 2-3           : append.  When the current map has not been copied into the store yet, its K/V
 //                         tiles come from the caller's tensors, and the CTA whose turn it is writes each
