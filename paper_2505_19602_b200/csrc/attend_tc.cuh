@@ -310,8 +310,8 @@ __host__ __device__ constexpr uint32_t instr_desc(bool b_mn_major) {
 }
 
 // Rare path of the softmax, taken together by the kParts warps that share a quarter's rows when the
-// fast sweep of one of their row parts overflowed the lazy band (the first tile, where no reference
-// exists yet, has a path of its own).  The S row part is still intact at s_addr: a first sweep finds its maximum,
+// fast sweep of one of their row parts overflowed the lazy band (the first tile takes its first
+// reference from its first columns and comes here as well if that was too low).  The S row part is still intact at s_addr: a first sweep finds its maximum,
 // the parts exchange theirs through shared memory (mine -> x_quarter[part], with one rendezvous on
 // pair_bar), the reference moves up to the row maximum if that is larger, the part's P is recomputed
 // against it and written over the part's first columns (a chunk's columns are only overwritten
@@ -647,20 +647,19 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         const uint32_t s_addr = lane_addr + kColS + buf * 128 + part * kCols;
         const int valid = tile_valid(j) - part * kCols;   // < kCols only in a ragged tile; may be <= 0
         float v[kChunks > 1 ? 2 : 1][32];
+        tc_ld32(s_addr, v[0]);
         if (j == 0) {
-          // first tile: no reference yet.  A sweep of its own finds the part's row maximum, the parts
-          // exchange theirs, and the ordinary sweep below then runs against the row maximum.
+          // first tile: no reference yet.  The largest of the first 32 columns of every part serves (the
+          // parts exchange theirs): the lazy band absorbs a row maximum up to 2^8 above it, and a row that
+          // exceeds the band takes the rare path below like in any other tile.  Column 0 of the first tile
+          // always holds a key, so the reference is finite; the chunk stays in registers for the sweep.
+          tc_wait_ld();
           float mt = -INFINITY;
 #pragma unroll
-          for (int cc = 0; cc < kChunks; ++cc) {
-            tc_ld32(s_addr + cc * 32, v[0]);
-            tc_wait_ld();
-#pragma unroll
-            for (int i = 0; i < 32; i += 2) {
-              const float e0 = (cc * 32 + i < valid) ? v[0][i] : -INFINITY;
-              const float e1 = (cc * 32 + i + 1 < valid) ? v[0][i + 1] : -INFINITY;
-              mt = max3(mt, e0, e1);
-            }
+          for (int i = 0; i < 32; i += 2) {
+            const float e0 = (i < valid) ? v[0][i] : -INFINITY;
+            const float e1 = (i + 1 < valid) ? v[0][i + 1] : -INFINITY;
+            mt = max3(mt, e0, e1);
           }
           x_quarter[part * 32 + lane] = mt;
           ok = meet();
@@ -669,7 +668,6 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           for (int q = 0; q < kParts; ++q) mt = fmaxf(mt, x_quarter[q * 32 + lane]);
           m_used[qt] = mt * c;
         }
-        tc_ld32(s_addr, v[0]);
         // one sweep: x = s * c - m, p = exp2(x), partial row sum; the bf16 pairs of p stay in registers
         // until all parts know that no exponent left the lazy band.  (kCols values of at most 2^8 sum to
         // at most 2^8 kCols; a larger, infinite or NaN sum means that some x exceeded 8.)
