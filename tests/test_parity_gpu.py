@@ -813,3 +813,39 @@ def test_one_call_step_equals_the_three_calls():
     assert torch.equal(O3, O1) and n3 == n1
     for a, b in zip(kept3, kept1):
         assert all(torch.equal(x, y) for x, y in zip(a, b))
+
+
+@pytest.mark.parametrize("amp", [6.0, 12.0])
+def test_dominant_keys_anywhere_in_the_first_tiles(amp):
+    """Rows whose logit towards one key is 70 or 140 nats above the rest, that key sitting in the first
+    columns of the first key tile, further inside it, in its second half, or in later tiles: whatever
+    the kernel took as its first reference, the output is that key's value row (the second amplitude
+    is beyond what exp2 can hold against a low reference)."""
+    sides = (4, 20)
+    n = orc.scale_token_counts(sides)
+    d = 128
+    budgets = [[binding.KEEP_ALL] * 2]
+    kv = binding.ScaleKV(1, 1, 2, d, "bf16", sides, sides, budgets, max_window=16)
+    gen = torch.Generator().manual_seed(123)
+    hot_slots = [5, 40, 70, 100, 130, 300]            # cache slots: 5 lies in the first map, the others in the second
+    dirs = torch.randn(len(hot_slots), d, generator=gen)
+    dirs = dirs / dirs.norm(dim=1, keepdim=True) * (d ** 0.5)      # |u|^2 = d: logit of a * u against u is a * sqrt(d)
+
+    def inputs(l, k):
+        Q = torch.randn(1, 2, n[k], d, generator=gen)
+        K = torch.randn(1, 2, n[k], d, generator=gen)
+        V = torch.randn(1, 2, n[k], d, generator=gen)
+        if k == 1:
+            for i in range(n[k]):
+                Q[0, :, i] = dirs[i % len(hot_slots)]
+        for s, u in zip(hot_slots, dirs):
+            if k == 0 and s < n[0]:
+                K[0, :, s] = amp * u
+            if k == 1 and s >= n[0]:
+                K[0, :, s - n[0]] = amp * u
+        return Q.to(torch.bfloat16), K.to(torch.bfloat16), V.to(torch.bfloat16)
+
+    run = ParityRun(kv, "bf16", sides, budgets, inputs, lambda k: orc.window_centroids(sides[k], sides[k], 16),
+                    [(0, 0, 0), (0, 0, 1)], check_lse=True).run()
+    assert run.max_err <= run.max_tol
+    kv.close()
