@@ -28,11 +28,11 @@ if ROOT not in sys.path:
 
 METRIC = "scale_steps_per_sec"
 # DRAM traffic of the attend kernel: (dram__bytes_read.sum + dram__bytes_write.sum) / algorithmic bytes over the two
-# launches of an ncu capture of one layer of the headline workload, its two largest scales (1546.7 MB measured against
+# launches of an ncu capture of one layer of the headline workload, its two largest scales (1548.8 MB measured against
 # 1676 MB algorithmic: part of the appended rows is still in L2 when a launch ends).  The capture runs one layer of the
 # workload; traffic grows in proportion to the bytes a launch must move, so the roofline object reports this ratio times
 # the average algorithmic bytes per launch.  Set to None when the kernel changes after the capture.
-ATTEND_TRAFFIC_RATIO = 1546.7 / 1676.0
+ATTEND_TRAFFIC_RATIO = 1548.8 / 1676.0
 UNIT = "scale-steps/s"
 
 
