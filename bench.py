@@ -34,6 +34,7 @@ METRIC = "scale_steps_per_sec"
 # the average algorithmic bytes per launch.  Set to None when the kernel changes after the capture.
 ATTEND_TRAFFIC_RATIO = 1548.8 / 1676.0
 UNIT = "scale-steps/s"
+E2E_HOST_LAYERS = 4
 
 
 def parse_args():
@@ -279,7 +280,7 @@ def run_scalekv(args):
         asi, roles = pipeline.calibrate_roles(wl, wl.n_drafters, device=local_rank)
         if args.overall_pct > 0:
             r1000 = max(1, round(args.overall_pct * 1000 / 3.25))          # refiner share in 1/100000 of T_c
-            budgets = pipeline.budget_table(wl, roles, drafter_pct=(10 * r1000, 100000), refiner_pct=(r1000, 100000))
+            budgets = pipeline.budget_table(wl, roles, drafter_frac=10 * r1000 / 100000, refiner_frac=r1000 / 100000)
         else:
             budgets = pipeline.budget_table(wl, roles)
         planted = synth.drafter_layers(wl)
@@ -291,7 +292,7 @@ def run_scalekv(args):
         role_note = (f"{wl.n_drafters} drafters per scale from scalekv_layer_stats; {hits}/{len(planted) * len(ks)} planted "
                      f"drafters recovered at the {len(ks)} scales whose history exceeds 4 K'")
     else:
-        b = pipeline.pct_budget(10, 100, sum(wl.n_tokens[:-1]))
+        b = binding.scalekv_budget_tokens(0.10, wl.sides)
         budgets = [[b] * wl.n_scales for _ in range(wl.n_layers)]
         role_note = "uniform 10%"
     calib_s = time.perf_counter() - t0
@@ -410,7 +411,7 @@ def run_scalekv(args):
     peak_tf = peaks["bf16_sustained"] if wl.dtype == "bf16" else None
     kernels = {}
     for name, key in (("append", "append_bytes"), ("score", "score_bytes"), ("select", "select_bytes"),
-                      ("compact", "compact_bytes")):
+                      ("compact", "compact_bytes"), ("compress", "compress_bytes")):
         kms, kn = prof_alone[name]
         if kn == 0:
             continue
@@ -431,7 +432,7 @@ def run_scalekv(args):
                 "avg_launch_ms": att_ms / max(att_n, 1),
                 "flop_per_launch_avg": work["attend_flop"] / max(work["attend_launches"], 1),
                 "ms_per_pass_with_events": ms_events / args.steps}
-    hbm_bytes = work["compact_bytes"] + work["select_bytes"] + work["score_bytes"]
+    hbm_bytes = work["compress_bytes"]
     ser_ms = (work["attend_flop"] / (peaks["bf16_sustained"] * 1e12) + hbm_bytes / (peaks["hbm_gbs"] * 1e9)) * 1e3
     pass_ms = ms / args.steps
     roofline["pass_roofline_ms_serial"] = ser_ms
@@ -442,9 +443,13 @@ def run_scalekv(args):
     if not args.no_e2e:
         n_max = max(wl.n_tokens)
         dt = synth.torch_dtype(wl.dtype)
+        # pinned host copies of the inputs of E2E_HOST_LAYERS layers (a full set would pin 33 GB); layer l reads set
+        # l mod E2E_HOST_LAYERS, so consecutive steps copy from different host pages
         host = {}
-        for k in range(wl.n_scales):
-            host[k] = tuple(t.cpu().pin_memory() for t in inputs.data[(0, k)])
+        n_host = min(E2E_HOST_LAYERS, wl.n_layers)
+        for r in range(n_host):
+            for k in range(wl.n_scales):
+                host[(r, k)] = tuple(t.cpu().pin_memory() for t in inputs.data[(r, k)])
         Oh = [torch.empty(wl.batch, wl.n_heads, n_max, wl.head_dim, dtype=dt).pin_memory() for _ in range(2)]
         staging = torch.empty(8 * wl.batch * wl.n_heads * n_max * wl.head_dim, dtype=dt, device="cuda")
         torch.cuda.synchronize()
@@ -453,9 +458,9 @@ def run_scalekv(args):
             kv.scalekv_reset()
             for k in range(wl.n_scales):
                 nk = wl.n_tokens[k]
-                Qh, Kh, Vh = host[k]
                 last = k + 1 == wl.n_scales
                 for l in range(wl.n_layers):
+                    Qh, Kh, Vh = host[(l % n_host, k)]
                     kv.scalekv_step_host(l, k, Qh, Kh, Vh, Oh[(l + k) & 1], staging, window_pos=None if last else windows[k])
             kv.scalekv_sync()                  # every output has reached the host
         e2e_steps = max(1, min(args.steps, 3))
@@ -472,8 +477,8 @@ def run_scalekv(args):
         e2e = {"value": wl.n_scales * e2e_steps * world / e2e_s, "unit": UNIT, "h2d_bytes_per_step": 3 * tok_bytes,
                "d2h_bytes_per_step": tok_bytes, "steps": e2e_steps,
                "note": "scalekv_step_host per layer and scale: pinned host Q/K/V -> device, append + attend + compress, O -> "
-                       "pinned host; the copies of neighbouring steps overlap the kernels; one sync per pass; layer 0's "
-                       "host tensors are reused for every layer"}
+                       "pinned host; the copies of neighbouring steps overlap the kernels; one sync per pass; layer l reads "
+                       f"the pinned host tensors of layer l mod {n_host}"}
         del staging
 
     cpu = None
@@ -492,7 +497,7 @@ def run_scalekv(args):
                        "window": wl.window, "parallelism": f"replica x{world} (batch-sharded, no collective)",
                        "l2_policy": f"inputs larger than L2: {inputs.bytes() / 1e9:.1f} GB of Q/K/V per pass",
                        "side_stream": not args.no_side_stream, "cuda_graph": graph_note, "calibration_s": round(calib_s, 1),
-                       "attend_kernel": "tcgen05" if os.environ.get("SCALEKV_ATTEND", "") != "simt" else "simt"},
+                       "attend_kernel": "tcgen05" if (wl.dtype == "bf16" and wl.head_dim == 128) else "fp32 FMA"},
             "roofline": roofline, "kernels": kernels, "per_scale": per_scale, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches,
             "clocks": clocks, "work_per_pass": {k: v for k, v in work.items() if k != "per_scale_flop"},
         }

@@ -122,7 +122,15 @@ scalekv_status scalekv_destroy(scalekv_ctx *ctx);
  * on the critical path); any other next call for this layer (compress, layer_stats, export, the
  * next append) copies first with a kernel of its own.  K and V must therefore stay unmodified
  * until stream_main has passed the layer's next call.  For f32 x 64 the copy is enqueued here.
- * Ordered on stream_main after this layer's previous compress. */
+ * Ordered on stream_main after this layer's previous compress.
+ * Layers of equal parity (0, 2, 4, .. / 1, 3, 5, ..) share one transient page set, which holds the part of a
+ * current map that exceeds the layer's persistent capacity, and one buffer of recorded window logits.  An append
+ * therefore returns SCALEKV_ERR_BAD_STATE, and touches nothing, while another layer of the same parity still
+ * holds an appended map that reaches into the transient pages and has not been compressed; otherwise it waits
+ * (on stream_main) for that layer's last compress.  The one exception is a map of the LAST scale that has been
+ * attended: no later step reads it, so its transient rows are given up, and that layer then refuses compress and
+ * layer_stats (BAD_STATE) and exports only the entries before that map until scalekv_reset.  The model's own order -
+ * append, attend, compress of layer l before layer l + 1 - never meets this rule. */
 scalekv_status scalekv_append(scalekv_ctx *ctx, int32_t layer, int32_t scale, scalekv_tensor K, scalekv_tensor V);
 
 /* Eq. 5: O[b][h][i] = sum_j softmax_j(scale * <Q[b][h][i], K_j>) V_j over all L entries of the
@@ -155,7 +163,8 @@ scalekv_status scalekv_compress(scalekv_ctx *ctx, int32_t layer, scalekv_tensor 
  *                window; attention sinks + recent tokens): there is no observation window (Qw, w,
  *                window_pos are ignored), the n_sink lowest original positions always stay and the most
  *                recent other entries fill the budget; here k^l = budgets[layer][scale] counts the WHOLE
- *                cache after the call, sinks included.
+ *                cache after the call, sinks included.  The layer's pages were sized from the table, so
+ *                min(n_sink, tokens so far) beyond the persistent capacity returns SCALEKV_ERR_CAPACITY.
  *   pool_kernel  SCORE only.  Odd width (< 64) of a 1-D average pooling of the importance along the slot
  *                axis before the selection ("average pooling", Sec. 3.3, read as smoothing along keys: zeros
  *                beyond both ends, always divided by the width; the neighbours are the entries next to it in
@@ -173,6 +182,10 @@ scalekv_status scalekv_compress(scalekv_ctx *ctx, int32_t layer, scalekv_tensor 
  *                different numbers of entries.  Each value must lie in [0, budgets[layer][scale]] (the
  *                pages were sized for the table's value); any value >= 0 when the table says KEEP_ALL.
  *                With head_shared the heads must agree.  At most 128 heads.
+ *   separate_kernels  0: importance, selection and pruning of a slice run in ONE launch (one CTA per slice, the
+ *                slice's keys and keep list in shared memory) whenever a slice of the configured schedule fits;
+ *                1: as three launches (importance; selection; pruning spread over 8 CTAs per slice), which is what
+ *                slices too long for one CTA's shared memory and head_shared get in any case.  Same results.
  * opts == NULL is scalekv_compress. */
 #define SCALEKV_SELECT_SCORE 0
 #define SCALEKV_SELECT_RECENT 1
@@ -182,6 +195,7 @@ typedef struct {
   int32_t n_sink;        /* RECENT only */
   int32_t head_shared;   /* SCORE only */
   const int32_t *head_budgets;
+  int32_t separate_kernels;   /* see below */
 } scalekv_select_opts;
 scalekv_status scalekv_compress_ex(scalekv_ctx *ctx, int32_t layer, scalekv_tensor Qw, int32_t w, const int32_t *window_pos,
                                    int32_t qw_is_full_map, const scalekv_select_opts *opts);
@@ -245,6 +259,13 @@ scalekv_status scalekv_assign_roles(const double *asi, int32_t L, int32_t K, int
 scalekv_status scalekv_make_budgets(const uint8_t *is_drafter, int32_t L, int32_t K, double b_uniform, double b_r0,
                                     double delta, int32_t *budgets_out);
 
+/* Sec. 4.1 / Sec. 4.3: a budget quoted as a fraction of "the original KV cache size" is that fraction of
+ * T_c = N_{K-1}, the tokens that ever need caching (the last map is never read by a later step - Table 1's
+ * full-cache sizes divide by exactly that count), rounded half up: *tokens = floor(fraction * T_c + 1/2).
+ * 13-scale schedule: 0.30 -> 1928, 0.03 -> 193, 0.10 -> 643.  Host only. */
+scalekv_status scalekv_budget_tokens(double fraction, const int32_t *scale_h, const int32_t *scale_w, int32_t n_scales,
+                                     int32_t *tokens);
+
 /* ---- introspection ------------------------------------------------------------------------ */
 
 /* Current number of entries of every slice of a layer -> len_host HOST [B][H].  Synchronous. */
@@ -264,6 +285,16 @@ scalekv_status scalekv_export_scores(scalekv_ctx *ctx, int32_t b, int32_t h, flo
 /* Waits for both streams; returns the sticky device status (OK, TIMEOUT or DEVICE_CHECK). */
 scalekv_status scalekv_sync(scalekv_ctx *ctx);
 
+/* Self-test of the failure path every device-side wait of the library shares (no counterpart in the paper).
+ * A one-CTA kernel waits, through the same bounded-wait routine the attention kernel uses, on a barrier
+ * that nothing ever arrives at, with a limit of limit_ms (1 .. 1000) instead of the library's 2 s.  The wait
+ * gives up after the limit, raises the sticky device status and the kernel RETURNS (it never spins without
+ * bound, traps or faults).  *gave_up (HOST) = 1 when the wait reported the time-out, *seen_by_peer (HOST) = 1
+ * when a second warp of the CTA saw the CTA-wide abort flag that the give-up sets.  Synchronous on
+ * stream_main.  Afterwards scalekv_sync returns SCALEKV_ERR_TIMEOUT and every later attention CTA returns at
+ * once (the status is sticky for the context's life): use a context of its own. */
+scalekv_status scalekv_selftest_wait(scalekv_ctx *ctx, int32_t limit_ms, int32_t *gave_up, int32_t *seen_by_peer);
+
 /* Number of kernels this context has launched since scalekv_init (HOST out). */
 scalekv_status scalekv_launch_count(scalekv_ctx *ctx, int64_t *count);
 
@@ -271,7 +302,8 @@ scalekv_status scalekv_launch_count(scalekv_ctx *ctx, int64_t *count);
  * it runs on (durations of kernels on the two streams may overlap and then include contention).
  * on = 2: compress runs on stream_main as well, so that no two kernels overlap and each duration
  * is the kernel's own.  on = 0: off.  scalekv_profile_read waits for both streams and returns, for
- * class `which` (0 append, 1 attend, 2 score, 3 select, 4 compact, 5 other), the
+ * class `which` (0 append, 1 attend, 2 score, 3 select, 4 compact, 5 other, 6 compress = importance, selection
+ * and pruning in one launch), the
  * summed milliseconds and the number of launches since profiling was last enabled. */
 scalekv_status scalekv_profile_enable(scalekv_ctx *ctx, int32_t on);
 scalekv_status scalekv_profile_read(scalekv_ctx *ctx, int32_t which, double *ms_total, int64_t *launches);

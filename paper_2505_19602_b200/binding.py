@@ -21,7 +21,7 @@ KEEP_ALL = -1
 MAX_WINDOW = 64
 BF16, F32 = 0, 1
 STATUS_NAMES = ["OK", "INVALID_ARG", "BAD_STATE", "CAPACITY", "UNSUPPORTED", "CUDA", "TIMEOUT", "DEVICE_CHECK"]
-KERNEL_CLASSES = ["append", "attend", "score", "select", "compact", "other"]
+KERNEL_CLASSES = ["append", "attend", "score", "select", "compact", "other", "compress"]
 
 
 class ScaleKVError(RuntimeError):
@@ -45,7 +45,7 @@ class scalekv_config(C.Structure):
 
 class scalekv_select_opts(C.Structure):
     _fields_ = [("policy", C.c_int32), ("pool_kernel", C.c_int32), ("n_sink", C.c_int32), ("head_shared", C.c_int32),
-                ("head_budgets", C.POINTER(C.c_int32))]
+                ("head_budgets", C.POINTER(C.c_int32)), ("separate_kernels", C.c_int32)]
 
 
 class scalekv_tensor(C.Structure):
@@ -106,6 +106,8 @@ def load_library():
         "scalekv_export_scores": [ctx_p, i32, i32, P(C.c_float), i32, P(i32)],
         "scalekv_sync": [ctx_p],
         "scalekv_join": [ctx_p],
+        "scalekv_budget_tokens": [f64, P(i32), P(i32), i32, P(i32)],
+        "scalekv_selftest_wait": [ctx_p, i32, P(i32), P(i32)],
         "scalekv_launch_count": [ctx_p, P(i64)],
         "scalekv_profile_enable": [ctx_p, i32],
         "scalekv_profile_read": [ctx_p, i32, P(f64), P(i64)],
@@ -177,6 +179,17 @@ def scalekv_make_budgets(is_drafter, b_uniform, b_r0, delta):
     if st:
         raise ScaleKVError(st)
     return out
+
+
+def scalekv_budget_tokens(fraction, sides_h, sides_w=None):
+    """Tokens that a budget quoted as a fraction of the cached tokens T_c = N_{K-1} stands for (rounded half up)."""
+    lib = load_library()
+    sides_w = sides_h if sides_w is None else sides_w
+    out = C.c_int32(0)
+    st = lib.scalekv_budget_tokens(float(fraction), _i32_array(sides_h), _i32_array(sides_w), len(sides_h), C.byref(out))
+    if st:
+        raise ScaleKVError(st, "scalekv_budget_tokens")
+    return out.value
 
 
 def scalekv_select_static(scores: torch.Tensor, k: int, idx_out: torch.Tensor = None, stream=None):
@@ -282,10 +295,11 @@ class ScaleKV:
             self._check(self.lib.scalekv_compress(self.ctx, layer, tensor_arg(Qw), len(window_pos), wp, int(qw_is_full_map)))
 
     def scalekv_compress_ex(self, layer, Qw=None, window_pos=None, qw_is_full_map=False, policy="score", pool_kernel=1,
-                            n_sink=0, head_shared=False, head_budgets=None):
+                            n_sink=0, head_shared=False, head_budgets=None, separate_kernels=False):
         """scalekv_compress with a selection variant: policy "score" (optionally pooled) or "recent"."""
         hb = _i32_array(head_budgets) if head_budgets is not None else None
-        opts = scalekv_select_opts({"score": 0, "recent": 1}[policy], pool_kernel, n_sink, int(head_shared), hb)
+        opts = scalekv_select_opts({"score": 0, "recent": 1}[policy], pool_kernel, n_sink, int(head_shared), hb,
+                                   int(separate_kernels))
         q = tensor_arg(Qw) if Qw is not None else scalekv_tensor(None, 0, 0, 0)
         if window_pos is None:
             wp, w = None, 0
@@ -371,6 +385,12 @@ class ScaleKV:
 
     def scalekv_join(self):
         self._check(self.lib.scalekv_join(self.ctx))
+
+    def scalekv_selftest_wait(self, limit_ms=50):
+        """(gave_up, seen_by_peer) of the bounded-wait self-test; leaves the context's device status at TIMEOUT."""
+        a, b = C.c_int32(0), C.c_int32(0)
+        self._check(self.lib.scalekv_selftest_wait(self.ctx, int(limit_ms), C.byref(a), C.byref(b)))
+        return a.value, b.value
 
     def scalekv_launch_count(self):
         n = C.c_int64(0)

@@ -2,7 +2,7 @@
 // O = softmax(scale * Q K^T) V with online softmax.  One CTA owns up to two 128-query tiles (A, B)
 // of one slice and streams the slice's K/V pages once for both.
 //
-// Roles inside a CTA of 128 + 128 * kParts threads:
+// Roles inside a CTA of 384 threads:
 //   warp 0 (one thread) : TMA producer.  The query tiles once; then per 128-key tile the K and V rows into
 //                         128B-swizzled shared memory: history tiles page by page through the slice's
 //                         page table, tiles of a not yet appended current map from the caller's tensors.
@@ -11,21 +11,23 @@
 //                         j is  S_A(j), PV_B(j-1), S_B(j), PV_A(j): while one tile's softmax runs, the
 //                         tensor pipe works for the other tile.  With one query tile the two S buffers
 //                         alternate and S(j+1) is issued ahead of PV(j).
-//   warps 4 ..          : softmax, kParts warps per TMEM lane quarter (kParts = 2: warps 4-11).  Warp w takes
-//                         columns kCols * ((w - 4) / 4) .. + kCols - 1 of every S tile; the warps w, w + 4, ..
-//                         share the 32 query rows (TMEM lanes) of quarter w % 4, and all of them work on tile
-//                         A's S, then on tile B's.  A thread sweeps its row part once (tcgen05.ld):
-//                         p = exp2(s * c - m) against the running reference m with packed f32x2 arithmetic
-//                         (a share of the exponentials on the FMA pipe), the partial row sum, and P as bf16
-//                         pairs written back into the first columns of its own part of the S buffer
-//                         (tcgen05.st), from where the PV product takes its A operand.  The warps of a
-//                         quarter meet on an mbarrier per tile: only when a part's sum shows that an
-//                         exponent left the lazy band (2^8) do they recompute the row against a new
-//                         reference and rescale O.  Threads that own a row of the observation window also
+//   warps 4-7, 8-11     : softmax, one warpgroup per query tile (warps 4-7 tile A, warps 8-11 tile B), one
+//                         thread per query row (TMEM lane), so that no row state is shared between threads and
+//                         the two tiles' chains  S -> softmax -> PV  run concurrently, each hiding the other's
+//                         hand-over latencies.  A thread sweeps its row of an S tile once, in four chunks of 32
+//                         columns (tcgen05.ld, the next chunk in flight): p = exp2(s * c - m) against a lazy
+//                         reference m with packed f32x2 arithmetic (a share of the exponentials on the FMA
+//                         pipe), the chunk's sum, and P as bf16 pairs written over the first 64 columns of the
+//                         row's S buffer (tcgen05.st; a chunk's P only covers columns already read), from
+//                         where the PV product takes its A operand.  Only when a chunk's sum shows that an
+//                         exponent left the lazy band (2^8) does the warp raise the reference: the chunk is
+//                         recomputed, the P chunks already stored for this tile, the running sum and the O
+//                         accumulator are scaled down.  Threads that own a row of the observation window also
 //                         store that row's raw products (16-byte stores, key tile j in columns 128 j ..) for
-//                         the compress that follows.  At the end the same warps normalise O, stage each tile
-//                         in the query tile's shared memory and one thread sends it out with TMA stores.
-//                         (Four warps per quarter, 16 softmax warps, measured the same as two.)
+//                         the compress that follows.  At the end each warpgroup normalises its O tile, stages
+//                         it in the query tile's shared memory and one thread sends it out with TMA stores.
+//                         With a single query tile (n_k <= 128, or the last odd tile of a map) warps 4-7 serve
+//                         both S buffers and warps 8-11 idle.
 //   warps 2-3           : append.  When the current map has not been copied into the store yet, its K/V
 //                         tiles come from the caller's tensors, and the CTA whose turn it is writes each
 //                         tile's rows from shared memory to the slice's pages (and their original
@@ -44,22 +46,19 @@
 namespace scalekv {
 namespace tc {
 
-constexpr int kParts = 2;                        // softmax warps per TMEM lane quarter: each takes 128 / kParts columns of an S tile
-constexpr int kCols = 128 / kParts;              // S columns per softmax thread and tile
-constexpr int kChunks = kCols / 32;              // tcgen05.ld x32 loads per thread and tile
-constexpr int kThreads = 128 + 128 * kParts;     // warps: TMA, MMA, 2 x append, 4 * kParts x softmax
+constexpr int kChunks = 4;                       // tcgen05.ld x32 loads per softmax thread (= query row) and S tile
+constexpr int kThreads = 128 + 2 * 128;          // warps: TMA, MMA, 2 x append, one softmax warpgroup per query tile
 constexpr int kStages = 5;                       // one ring for the K and V tiles: K_0, V_0, K_1, V_1, ...
 constexpr uint32_t kTileBytes = 128 * 128 * 2;   // one 128 x 128 bf16 operand tile
 constexpr uint32_t kHalfBytes = kTileBytes / 2;  // 64 head-dim columns = one 128-byte swizzle span
 constexpr uint32_t kOffQ = 0;                    // two query tiles (the dynamic shared memory must start 1024-byte aligned)
 constexpr uint32_t kOffRing = kOffQ + 2 * kTileBytes;
 constexpr uint32_t kOffBar = kOffRing + kStages * kTileBytes;
-constexpr uint32_t kOffX = kOffBar + 256;        // exchange area of the softmax warps of a quarter: flags [2][4][kParts], values [2][4][kParts][32]
-constexpr uint32_t kSmemBytes = kOffX + 128 + 2 * 4 * kParts * 32 * 4;
+constexpr uint32_t kSmemBytes = kOffBar + 256;
 static_assert(kSmemBytes <= 232448, "more shared memory than a CTA can have");
 // barrier slots (8 bytes each): one full/empty pair per ring stage, one S/P/PV barrier per S buffer or query tile
 enum { bQFull = 0, bFull = 1, bEmpty = bFull + kStages, bSFull = bEmpty + kStages, bPFull = bSFull + 2, bPvDone = bPFull + 2,
-       bPair = bPvDone + 2, bFinal = bPair + 4, bOut = bFinal + 2, bCount = bOut + 2 };
+       bFinal = bPvDone + 2, bOut = bFinal + 2, bCount = bOut + 2 };
 constexpr uint32_t kOffTmemSlot = 208;            // inside the barrier area, behind the barriers
 static_assert(bCount * 8 <= kOffTmemSlot, "barriers overlap the TMEM slot");
 constexpr uint32_t kTmemCols = 512;
@@ -96,13 +95,14 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait: false when the CTA is aborting or the time limit ran out (status raised).
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status) {
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status,
+                                            unsigned long long limit_ns = kWaitLimitNs) {
   const unsigned long long t0 = globaltimer();
   while (true) {
     for (int i = 0; i < 64; ++i)
       if (mbar_try(bar, parity)) return true;
     if (*abort_flag || *reinterpret_cast<volatile int *>(status) != 0) return false;
-    if (globaltimer() - t0 > kWaitLimitNs) {
+    if (globaltimer() - t0 > limit_ns) {
       *abort_flag = 1;
       atomicExch(status, kDevTimeout);
       return false;
@@ -112,6 +112,31 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volat
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status) {
   if (mbar_try(bar, parity)) return true;
   return mbar_wait_slow(bar, parity, abort_flag, status);
+}
+// Self-test of the bounded wait (scalekv_selftest_wait): one warp waits, with the given limit, on a barrier
+// that nobody ever arrives at.  The wait must give up, raise the sticky status and return; a second warp that
+// polls the CTA's abort flag (also bounded) shows that the other roles of a CTA see the give-up.
+// out[0] = 1 when the wait returned false, out[1] = 1 when the second warp saw the abort flag.
+__global__ void wait_probe_kernel(int *status, unsigned long long limit_ns, int *out) {
+  __shared__ __align__(8) unsigned long long probe_bar;
+  __shared__ int abort_word;
+  const uint32_t bar = smem_u32(&probe_bar);
+  if (threadIdx.x == 0) {
+    abort_word = 0;
+    mbar_init(bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  volatile int *abort_flag = &abort_word;
+  if (threadIdx.x == 0) {
+    const bool ok = mbar_try(bar, 0) || mbar_wait_slow(bar, 0, abort_flag, status, limit_ns);
+    out[0] = ok ? 0 : 1;
+  } else if (threadIdx.x == 32) {
+    const unsigned long long t0 = globaltimer();
+    int seen = 0;
+    while (!seen && globaltimer() - t0 < 4 * limit_ns + 1000000ull) seen = *abort_flag;
+    out[1] = seen;
+  }
 }
 // Same, with a warp-uniform result (the callers go on to warp-collective tcgen05 instructions).
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status) {
@@ -173,9 +198,9 @@ __device__ __forceinline__ void tc_mma_ss_x8(uint32_t d_tmem, uint32_t a_lo, uin
       "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc)
       : "memory");
 }
-// TS: A = P in TMEM (16 keys = 8 columns per step; every softmax thread's keys sit at the start of its
-// own kCols columns of the S buffer), B = V in shared memory as the MN-major operand (16 keys = 2048 B per step).
-__device__ __forceinline__ constexpr uint32_t p_col(int kk) { return (uint32_t)(((kk * 16) / kCols) * kCols + ((kk * 16) % kCols) / 2); }
+// TS: A = P in TMEM (16 keys = 8 columns per step; a row's 128 bf16 values of P fill the first 64 columns of
+// its S buffer), B = V in shared memory as the MN-major operand (16 keys = 2048 B per step).
+__device__ __forceinline__ constexpr uint32_t p_col(int kk) { return (uint32_t)(kk * 8); }
 __device__ __forceinline__ void tc_mma_ts_x8(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t hi, uint32_t idesc,
                                              uint32_t accumulate_first) {
   asm volatile(
@@ -229,6 +254,15 @@ __device__ __forceinline__ void tc_st32(uint32_t taddr, const float *v) {
       : "memory");
 }
 // 16 consecutive 32-bit columns (32 bf16 values of P) of this thread's TMEM lane
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t *r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+        "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
 __device__ __forceinline__ void tc_st16(uint32_t taddr, const uint32_t *v) {
   asm volatile(
       "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
@@ -309,68 +343,66 @@ __host__ __device__ constexpr uint32_t instr_desc(bool b_mn_major) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
 }
 
-// Rare path of the softmax, taken together by the kParts warps that share a quarter's rows when the
-// fast sweep of one of their row parts overflowed the lazy band (the first tile takes its first
-// reference from its first columns and comes here as well if that was too low).  The S row part is still intact at s_addr: a first sweep finds its maximum,
-// the parts exchange theirs through shared memory (mine -> x_quarter[part], with one rendezvous on
-// pair_bar), the reference moves up to the row maximum if that is larger, the part's P is recomputed
-// against it and written over the part's first columns (a chunk's columns are only overwritten
-// after it was read), and this warp's kCols columns of the O accumulator at o_addr are multiplied by
-// 2^(old reference - new reference) once the previous PV product of the tile has landed.
-// `valid` = number of columns of this part that hold keys (may be <= 0).  Returns the part's row sum
-// and the new reference; sum < 0 when a wait gave up.
-struct Redo { float sum, m; };
-__device__ __noinline__ Redo redo_part(uint32_t s_addr, uint32_t o_addr, int valid, float c, float m_used, bool with_o,
-                                       uint32_t pv_bar, uint32_t pv_parity, uint32_t pair_bar, uint32_t pair_parity,
-                                       volatile float *x_quarter, int part, int lane, volatile int *abort_flag, int *status) {
+// Rare path of the softmax, taken by a whole warp when the sum of one of its rows' chunks shows that an
+// exponent left the lazy band.  The chunk's 32 raw products are still intact in the row's S buffer (chunk cc
+// sits in columns [32 cc, 32 cc + 32) of s_addr, the P chunks stored so far only cover columns below 16 cc) and
+// are read again; `valid` of them are real keys.  Per lane the reference moves up to the chunk's maximum if
+// that is larger (a lane that needs nothing gets the factor 1): the chunk's P is recomputed against the new
+// reference and stored, and everything accumulated under the old one is multiplied by f = 2^(old - new): the
+// running row sum, the P chunks 0 .. cc-1 already stored for this tile (16 columns each), and - once the
+// previous PV product of the tile has landed - the row's 128 columns of the O accumulator at o_addr.
+// Everything goes in and out by value so that the caller's state stays in registers.
+struct Raised { float m, l, sum; int o_landed, ok; };
+__device__ __noinline__ Raised raise_reference(int valid, float c, float m, float l_run, uint32_t s_addr, int cc, uint32_t o_addr,
+                                               int with_o, int o_landed, uint32_t pv_bar, uint32_t pv_parity,
+                                               volatile int *abort_flag, int *status) {
+  float x[32];
+  tc_ld32(s_addr + cc * 32, x);
+  tc_wait_ld();
   float mt = -INFINITY;
-#pragma unroll 1
-  for (int cc = 0; cc < kChunks; ++cc) {
-    float x[32];
-    tc_ld32(s_addr + cc * 32, x);
-    tc_wait_ld();
 #pragma unroll
-    for (int i = 0; i < 32; ++i)
-      if (cc * 32 + i < valid) mt = fmaxf(mt, x[i]);
-  }
-  x_quarter[part * 32 + lane] = mt;
-  mbar_arrive(pair_bar);
-  if (!mbar_wait_warp(pair_bar, pair_parity, abort_flag, status)) return {-1.f, m_used};
-#pragma unroll
-  for (int q = 0; q < kParts; ++q) mt = fmaxf(mt, x_quarter[q * 32 + lane]);
-  const float m_new = fmaxf(m_used, mt * c);
-  const float sc = ex2(m_used - m_new);
+  for (int i = 0; i < 32; ++i)
+    if (i < valid) mt = fmaxf(mt, x[i]);
+  const float m_new = fmaxf(m, mt * c);
+  const float f = ex2(m - m_new);
   float sum = 0.f;
+  uint32_t pk[16];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    const float p0 = (2 * i < valid) ? ex2(fmaf(x[2 * i], c, -m_new)) : 0.f;
+    const float p1 = (2 * i + 1 < valid) ? ex2(fmaf(x[2 * i + 1], c, -m_new)) : 0.f;
+    sum += p0 + p1;
+    pk[i] = pack_bf16(p0, p1);
+  }
+  tc_st16(s_addr + cc * 16, pk);
 #pragma unroll 1
-  for (int cc = 0; cc < kChunks; ++cc) {
-    float x[32];
-    uint32_t pk[16];
-    tc_ld32(s_addr + cc * 32, x);
+  for (int e = 0; e < cc; ++e) {
+    uint32_t r[16];
+    tc_ld16(s_addr + e * 16, r);
     tc_wait_ld();
 #pragma unroll
-    for (int i = 0; i < 16; ++i) {
-      const float p0 = (cc * 32 + 2 * i < valid) ? ex2(fmaf(x[2 * i], c, -m_new)) : 0.f;
-      const float p1 = (cc * 32 + 2 * i + 1 < valid) ? ex2(fmaf(x[2 * i + 1], c, -m_new)) : 0.f;
-      sum += p0 + p1;
-      pk[i] = pack_bf16(p0, p1);
-    }
-    tc_st16(s_addr + cc * 16, pk);
+    for (int i = 0; i < 16; ++i)
+      r[i] = pack_bf16(__uint_as_float(r[i] << 16) * f, __uint_as_float(r[i] & 0xffff0000u) * f);
+    tc_st16(s_addr + e * 16, r);
   }
   if (with_o) {
-    if (!mbar_wait_warp(pv_bar, pv_parity, abort_flag, status)) return {-1.f, m_new};
-    tc_fence_after();
+    if (!o_landed) {
+      if (!mbar_wait_warp(pv_bar, pv_parity, abort_flag, status)) return {m_new, l_run * f, sum, 0, 0};
+      tc_fence_after();
+      o_landed = 1;
+    }
 #pragma unroll 1
-    for (int cc = 0; cc < kChunks; ++cc) {
+    for (int e = 0; e < 4; ++e) {
       float o[32];
-      tc_ld32(o_addr + cc * 32, o);
+      tc_ld32(o_addr + e * 32, o);
       tc_wait_ld();
 #pragma unroll
-      for (int i = 0; i < 32; ++i) o[i] *= sc;
-      tc_st32(o_addr + cc * 32, o);
+      for (int i = 0; i < 32; ++i) o[i] *= f;
+      tc_st32(o_addr + e * 32, o);
     }
   }
   tc_wait_st();
-  return {sum, m_new};
+  return {m_new, l_run * f, sum, o_landed, 1};
 }
 
 struct Params {
@@ -423,14 +455,17 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     return rest < 128 ? rest : 128;
   };
   int *status = lv.status;
-  if (*reinterpret_cast<volatile int *>(status) != 0) return;   // an earlier CTA gave up: do not pile on
-  if (base & 1023u) {                                            // swizzled tiles need the alignment: report, do not fault
-    if (tid == 0) atomicExch(status, kDevCheck);
-    return;
-  }
-  if (L > (lv.pages_per_slice << lv.page_shift)) {               // the slice would outgrow its page table: report, do not fault
-    if (tid == 0) atomicExch(status, kDevCheck);
-    return;
+  {
+    // One thread decides for the whole CTA whether it runs at all (the status word may change between two
+    // threads' reads, and a CTA of which only a part left would go on with barriers and TMEM nobody set up):
+    // an earlier CTA gave up - do not pile on; swizzled tiles need the alignment, and a slice must not outgrow
+    // its page table - report, do not fault.
+    int leave = 0;
+    if (tid == 0) {
+      if (*reinterpret_cast<volatile int *>(status) != 0) leave = 1;
+      else if ((base & 1023u) || L > (lv.pages_per_slice << lv.page_shift)) { atomicExch(status, kDevCheck); leave = 1; }
+    }
+    if (__syncthreads_or(leave)) return;
   }
 
   if (tid == 0) {
@@ -442,12 +477,11 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     }
     for (int s = 0; s < 2; ++s) {
       mbar_init(bar(bSFull + s), 1);
-      mbar_init(bar(bPFull + s), 128 * kParts);
+      mbar_init(bar(bPFull + s), 4);      // one arrival per warp of the softmax warpgroup that serves the buffer
       mbar_init(bar(bPvDone + s), 1);
     }
-    for (int s = 0; s < 4; ++s) mbar_init(bar(bPair + s), 32 * kParts);
     for (int s = 0; s < 2; ++s) mbar_init(bar(bFinal + s), 1);
-    for (int s = 0; s < 2; ++s) mbar_init(bar(bOut + s), 128 * kParts);
+    for (int s = 0; s < 2; ++s) mbar_init(bar(bOut + s), 4);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -602,204 +636,162 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   }
   } else {
     // ------------------------------------------------------------------ softmax + epilogue
-    const int part = (warp - 4) >> 2;            // which kCols columns of every S tile
+    const int qt = (warp - 4) >> 2;              // the query tile this warpgroup serves
     const int quarter = warp & 3;                // the TMEM lane quarter this warp may access
     const int row = quarter * 32 + lane;
     const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
     const float c = prm.scale_log2e;
     const uint64_t c2 = pack2(c, c);
-    volatile int *xflag = reinterpret_cast<volatile int *>(base_ptr + kOffX);                            // [2][4][kParts]
-    // values [2][4][kParts][32]: x_quarter points at [0][quarter]; the second block is only used by the epilogue
-    volatile float *x_quarter = reinterpret_cast<volatile float *>(base_ptr + kOffX + 128) + quarter * kParts * 32;
-    const uint32_t pair_bar = bar(bPair + quarter);
-    uint32_t pair_uses = 0;                      // rendezvous so far of this quarter's warps (same in all of them)
-    // rendezvous of the kParts warps of this quarter; false when a wait gave up
-    auto meet = [&]() -> bool {
-      mbar_arrive(pair_bar);
-      const bool r = mbar_wait_warp(pair_bar, pair_uses & 1u, abort_flag, status);
-      ++pair_uses;
-      return r;
-    };
-    const int ntile = single ? 1 : 2;
-    float m_used[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f};
-    // window rows of this thread (rank in the window, or -1) and whether its warp has any
-    int wrank[2] = {-1, -1};
-    bool wwarp[2] = {false, false};
-    if (prm.win_logits != nullptr) {
-#pragma unroll
-      for (int qt = 0; qt < 2; ++qt) {
-        const int qi = q_first + qt * 128 + row;
-        for (int e = 0; e < prm.w; ++e)
-          if (prm.win_pos[e] == qi) wrank[qt] = e;
-        wwarp[qt] = __any_sync(0xffffffffu, wrank[qt] >= 0);
-      }
+    const bool active = qt == 0 || !single;      // with one query tile the second warpgroup has nothing to do
+    float m = -INFINITY, l = 0.f;
+    // window row of this thread (rank in the window, or -1) and whether its warp has any
+    int wrank = -1;
+    bool wwarp = false;
+    if (prm.win_logits != nullptr && active) {
+      const int qi = q_first + qt * 128 + row;
+      for (int e = 0; e < prm.w; ++e)
+        if (prm.win_pos[e] == qi) wrank = e;
+      wwarp = __any_sync(0xffffffffu, wrank >= 0);
     }
+    const uint32_t o_addr = lane_addr + kColO + qt * 128;
     bool ok = true;
-    for (int j = 0; j < T && ok; ++j) {
+    for (int j = 0; j < T && ok && active; ++j) {
+      const int buf = single ? (j & 1) : qt;
+      const uint32_t par = single ? ((j >> 1) & 1) : (j & 1);
+      ok = mbar_wait_warp(bar(bSFull + buf), par, abort_flag, status);
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t s_addr = lane_addr + kColS + buf * 128;
+      const int valid = tile_valid(j);           // < 128 only in a ragged tile
+      int o_landed = 0;                          // the previous PV product of this tile has been waited for
+      float v[2][32];
+      tc_ld32(s_addr, v[0]);
 #pragma unroll
-      for (int qt = 0; qt < 2; ++qt) {
-        if (qt >= ntile || !ok) break;
-        const int buf = single ? (j & 1) : qt;
-        const uint32_t par = single ? ((j >> 1) & 1) : (j & 1);
-        ok = mbar_wait_warp(bar(bSFull + buf), par, abort_flag, status);
-        if (!ok) break;
-        tc_fence_after();
-        const uint32_t s_addr = lane_addr + kColS + buf * 128 + part * kCols;
-        const int valid = tile_valid(j) - part * kCols;   // < kCols only in a ragged tile; may be <= 0
-        float v[kChunks > 1 ? 2 : 1][32];
-        tc_ld32(s_addr, v[0]);
-        if (j == 0) {
-          // first tile: no reference yet.  The largest of the first 32 columns of every part serves (the
-          // parts exchange theirs): the lazy band absorbs a row maximum up to 2^8 above it, and a row that
-          // exceeds the band takes the rare path below like in any other tile.  Column 0 of the first tile
-          // always holds a key, so the reference is finite; the chunk stays in registers for the sweep.
-          tc_wait_ld();
+      for (int cc = 0; cc < kChunks; ++cc) {
+        tc_wait_ld();
+        if (cc + 1 < kChunks) tc_ld32(s_addr + (cc + 1) * 32, v[(cc + 1) & 1]);
+        float *x = v[cc & 1];
+        if (wwarp) {
+          if (wrank >= 0) {
+            // The row's raw products go out as they are (the score kernel applies the softmax scale), 32
+            // columns as eight 16-byte stores, at column 128 j + ...: key tile j owns columns [128 j, 128 j + 128)
+            // of a logit row, so the current map starts at the next multiple of 128 behind the history and
+            // every store is aligned.  Columns of a ragged tile beyond its keys hold finite values nobody reads.
+            const int col0 = j * 128 + cc * 32;
+            float4 *dst = reinterpret_cast<float4 *>(prm.win_logits + ((size_t)slice * prm.w + wrank) * prm.ld_l + col0);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) dst[i] = make_float4(x[4 * i], x[4 * i + 1], x[4 * i + 2], x[4 * i + 3]);
+          }
+          __syncwarp();   // the tcgen05 instructions that follow want the warp converged
+        }
+        if (j == 0 && cc == 0) {
+          // no reference yet: the largest of the row's first 32 products serves (column 0 of the first tile
+          // always holds a key, so it is finite); a later chunk that exceeds the band raises it like any other
           float mt = -INFINITY;
 #pragma unroll
           for (int i = 0; i < 32; i += 2) {
-            const float e0 = (i < valid) ? v[0][i] : -INFINITY;
-            const float e1 = (i + 1 < valid) ? v[0][i + 1] : -INFINITY;
+            const float e0 = (i < valid) ? x[i] : -INFINITY;
+            const float e1 = (i + 1 < valid) ? x[i + 1] : -INFINITY;
             mt = max3(mt, e0, e1);
           }
-          x_quarter[part * 32 + lane] = mt;
-          ok = meet();
-          if (!ok) break;
-#pragma unroll
-          for (int q = 0; q < kParts; ++q) mt = fmaxf(mt, x_quarter[q * 32 + lane]);
-          m_used[qt] = mt * c;
+          m = mt * c;
         }
-        // one sweep: x = s * c - m, p = exp2(x), partial row sum; the bf16 pairs of p stay in registers
-        // until all parts know that no exponent left the lazy band.  (kCols values of at most 2^8 sum to
-        // at most 2^8 kCols; a larger, infinite or NaN sum means that some x exceeded 8.)
-        const uint64_t negm2 = pack2(-m_used[qt], -m_used[qt]);
+        // x = s * c - m, p = exp2(x), the chunk's sum.  32 values of at most 2^8 sum to at most 2^13; a larger,
+        // infinite or NaN sum means that some x exceeded 8.
+        const uint64_t negm2 = pack2(-m, -m);
         uint64_t sum2a = pack2(0.f, 0.f), sum2b = sum2a;
-        uint32_t pk[kCols / 2];
+        uint32_t pk[16];
+        const int vc = valid - cc * 32;          // real keys in this chunk (>= 32: all)
 #pragma unroll
-        for (int cc = 0; cc < kChunks; ++cc) {
-          tc_wait_ld();
-          if (cc + 1 < kChunks) tc_ld32(s_addr + (cc + 1) * 32, v[(cc + 1) & 1]);
-          float *x = v[cc & 1];
-          if (wwarp[qt]) {
-            if (wrank[qt] >= 0) {
-              // The row's raw products go out as they are (the score kernel applies the softmax scale), 32
-              // columns as eight 16-byte stores, at column 128 j + ...: key tile j owns columns [128 j, 128 j + 128)
-              // of a logit row, so the current map starts at the next multiple of 128 behind the history and
-              // every store is aligned.  Columns of a ragged tile beyond its keys hold finite values nobody reads.
-              const int col0 = j * 128 + part * kCols + cc * 32;
-              float4 *dst = reinterpret_cast<float4 *>(prm.win_logits + ((size_t)slice * prm.w + wrank[qt]) * prm.ld_l + col0);
-#pragma unroll
-              for (int i = 0; i < 8; ++i) dst[i] = make_float4(x[4 * i], x[4 * i + 1], x[4 * i + 2], x[4 * i + 3]);
-            }
-            __syncwarp();   // the tcgen05 instructions that follow want the warp converged
+        for (int i = 0; i < 16; i += 4) {
+          float a0, a1, a2, a3, a4, a5, a6, a7;
+          unpack2(fma2(pack2(x[2 * i + 0], x[2 * i + 1]), c2, negm2), a0, a1);
+          unpack2(fma2(pack2(x[2 * i + 2], x[2 * i + 3]), c2, negm2), a2, a3);
+          unpack2(fma2(pack2(x[2 * i + 4], x[2 * i + 5]), c2, negm2), a4, a5);
+          unpack2(fma2(pack2(x[2 * i + 6], x[2 * i + 7]), c2, negm2), a6, a7);
+          if (vc < 32) {
+            if (2 * i + 0 >= vc) a0 = -INFINITY;
+            if (2 * i + 1 >= vc) a1 = -INFINITY;
+            if (2 * i + 2 >= vc) a2 = -INFINITY;
+            if (2 * i + 3 >= vc) a3 = -INFINITY;
+            if (2 * i + 4 >= vc) a4 = -INFINITY;
+            if (2 * i + 5 >= vc) a5 = -INFINITY;
+            if (2 * i + 6 >= vc) a6 = -INFINITY;
+            if (2 * i + 7 >= vc) a7 = -INFINITY;
           }
-          if (valid < kCols) {
-#pragma unroll
-            for (int i = 0; i < 32; ++i)
-              if (cc * 32 + i >= valid) x[i] = -INFINITY;
-          }
-#pragma unroll
-          for (int i = 0; i < 16; i += 4) {
-            float a0, a1, a2, a3, a4, a5, a6, a7;
-            unpack2(fma2(pack2(x[2 * i + 0], x[2 * i + 1]), c2, negm2), a0, a1);
-            unpack2(fma2(pack2(x[2 * i + 2], x[2 * i + 3]), c2, negm2), a2, a3);
-            unpack2(fma2(pack2(x[2 * i + 4], x[2 * i + 5]), c2, negm2), a4, a5);
-            unpack2(fma2(pack2(x[2 * i + 6], x[2 * i + 7]), c2, negm2), a6, a7);
-            float p0, p1, p2, p3, p4, p5, p6, p7;
-            if (kPolyPairs > 0) exp2_poly_pair(a0, a1, p0, p1); else { p0 = ex2(a0); p1 = ex2(a1); }
-            if (kPolyPairs > 1) exp2_poly_pair(a2, a3, p2, p3); else { p2 = ex2(a2); p3 = ex2(a3); }
-            if (kPolyPairs > 2) exp2_poly_pair(a4, a5, p4, p5); else { p4 = ex2(a4); p5 = ex2(a5); }
-            if (kPolyPairs > 3) exp2_poly_pair(a6, a7, p6, p7); else { p6 = ex2(a6); p7 = ex2(a7); }
-            sum2a = add2(sum2a, pack2(p0, p1));
-            sum2b = add2(sum2b, pack2(p2, p3));
-            sum2a = add2(sum2a, pack2(p4, p5));
-            sum2b = add2(sum2b, pack2(p6, p7));
-            pk[cc * 16 + i + 0] = pack_bf16(p0, p1);
-            pk[cc * 16 + i + 1] = pack_bf16(p2, p3);
-            pk[cc * 16 + i + 2] = pack_bf16(p4, p5);
-            pk[cc * 16 + i + 3] = pack_bf16(p6, p7);
-          }
+          float p0, p1, p2, p3, p4, p5, p6, p7;
+          if (kPolyPairs > 0) exp2_poly_pair(a0, a1, p0, p1); else { p0 = ex2(a0); p1 = ex2(a1); }
+          if (kPolyPairs > 1) exp2_poly_pair(a2, a3, p2, p3); else { p2 = ex2(a2); p3 = ex2(a3); }
+          if (kPolyPairs > 2) exp2_poly_pair(a4, a5, p4, p5); else { p4 = ex2(a4); p5 = ex2(a5); }
+          if (kPolyPairs > 3) exp2_poly_pair(a6, a7, p6, p7); else { p6 = ex2(a6); p7 = ex2(a7); }
+          sum2a = add2(sum2a, pack2(p0, p1));
+          sum2b = add2(sum2b, pack2(p2, p3));
+          sum2a = add2(sum2a, pack2(p4, p5));
+          sum2b = add2(sum2b, pack2(p6, p7));
+          pk[i + 0] = pack_bf16(p0, p1);
+          pk[i + 1] = pack_bf16(p2, p3);
+          pk[i + 2] = pack_bf16(p4, p5);
+          pk[i + 3] = pack_bf16(p6, p7);
         }
         float s0, s1, s2, s3;
         unpack2(sum2a, s0, s1);
         unpack2(sum2b, s2, s3);
-        const float lt = (s0 + s1) + (s2 + s3);
-        // the warps of the quarter tell each other whether one of their rows needs the rare path
-        int mine = __any_sync(0xffffffffu, !(lt <= 256.f * (float)kCols)) ? 1 : 0;
-        const int slot = (int)(pair_uses & 1u);
-        if (lane == 0) xflag[(slot * 4 + quarter) * kParts + part] = mine;
-        ok = meet();
-        if (!ok) break;
-#pragma unroll
-        for (int q = 0; q < kParts; ++q) mine |= xflag[(slot * 4 + quarter) * kParts + q];
-        if (mine) {
-          const Redo r = redo_part(s_addr, lane_addr + kColO + qt * 128 + part * kCols, valid, c, m_used[qt], j > 0,
-                                   bar(bPvDone + qt), (j - 1) & 1, pair_bar, pair_uses & 1u, x_quarter, part, lane, abort_flag,
-                                   status);
-          ++pair_uses;
-          ok = __all_sync(0xffffffffu, r.sum >= 0.f);
+        float lt = (s0 + s1) + (s2 + s3);
+        if (__any_sync(0xffffffffu, !(lt <= 8192.f))) {
+          const Raised r = raise_reference(vc, c, m, l, s_addr, cc, o_addr, j > 0 ? 1 : 0, o_landed, bar(bPvDone + qt),
+                                           (j - 1) & 1, abort_flag, status);
+          ok = __all_sync(0xffffffffu, r.ok != 0);
           if (!ok) break;
-          l[qt] = l[qt] * ex2(m_used[qt] - r.m) + r.sum;
-          m_used[qt] = r.m;
+          m = r.m; l = r.l + r.sum; o_landed = r.o_landed;
         } else {
-#pragma unroll
-          for (int cc = 0; cc < kChunks; ++cc) tc_st16(s_addr + cc * 16, pk + cc * 16);
-          l[qt] += lt;
+          tc_st16(s_addr + cc * 16, pk);
+          l += lt;
         }
-        tc_wait_st();
-        tc_fence_before();
-        mbar_arrive(bar(bPFull + buf));
       }
+      if (!ok) break;
+      tc_wait_st();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(bPFull + buf));
     }
-    // the row sums are the sums of the parts' partial sums: one exchange for both tiles (the rendezvous
-    // before it orders the other warps' last read of the exchange area before its reuse)
-    if (ok) ok = meet();
-    if (ok) {
-#pragma unroll
-      for (int qt = 0; qt < 2; ++qt) x_quarter[(qt * 4 * kParts + part) * 32 + lane] = l[qt];
-      ok = meet();
-    }
-#pragma unroll
-    for (int qt = 0; qt < 2; ++qt) {
-      if (qt >= ntile || !ok) break;
-      float lsum = 0.f;
-#pragma unroll
-      for (int q = 0; q < kParts; ++q) lsum += x_quarter[(qt * 4 * kParts + q) * 32 + lane];
+    if (ok && active) {
       // a barrier that completes exactly once, after the last PV product: the per-tile PV barrier will
       // not do, a parity wait cannot tell phases two apart and this warp may be that far behind it
       ok = mbar_wait_warp(bar(bFinal + qt), 0, abort_flag, status);
-      if (!ok) break;
+    }
+    if (ok && active) {
       tc_fence_after();
-      const float inv = 1.f / lsum;
+      const float inv = 1.f / l;
       const int qi = q_first + qt * 128 + row;
-      float o[kChunks][32];
-#pragma unroll
-      for (int cc = 0; cc < kChunks; ++cc) tc_ld32(lane_addr + kColO + qt * 128 + part * kCols + cc * 32, o[cc]);
-      tc_wait_ld();
       // The normalised rows go to the query tile's shared memory (no product reads it any more) in the layout
       // of a TMA box - two halves of 64 columns, rows of 128 bytes, 128-byte swizzle - and one thread sends the
       // tile out with two bulk tensor stores: a row written by its own thread straight to global memory costs a
       // 128-byte line per lane and store instruction.  The tensor map clips the rows beyond n_k.
-      static_assert(kCols == 64, "one softmax part = one 64-column half of the output tile");
-      const uint32_t stage = base + kOffQ + qt * kTileBytes + part * kHalfBytes + row * 128;
+      const uint32_t stage = base + kOffQ + qt * kTileBytes + row * 128;
+      float o[2][32];
+      tc_ld32(o_addr, o[0]);
 #pragma unroll
       for (int cc = 0; cc < kChunks; ++cc) {
+        tc_wait_ld();
+        if (cc + 1 < kChunks) tc_ld32(o_addr + (cc + 1) * 32, o[(cc + 1) & 1]);
+        const float *oc = o[cc & 1];
 #pragma unroll
         for (int v4 = 0; v4 < 4; ++v4) {
-          const uint32_t wx = pack_bf16(o[cc][8 * v4 + 0] * inv, o[cc][8 * v4 + 1] * inv);
-          const uint32_t wy = pack_bf16(o[cc][8 * v4 + 2] * inv, o[cc][8 * v4 + 3] * inv);
-          const uint32_t wz = pack_bf16(o[cc][8 * v4 + 4] * inv, o[cc][8 * v4 + 5] * inv);
-          const uint32_t ww = pack_bf16(o[cc][8 * v4 + 6] * inv, o[cc][8 * v4 + 7] * inv);
-          const uint32_t addr = stage + ((uint32_t)((cc * 4 + v4) ^ (row & 7)) << 4);
+          const uint32_t wx = pack_bf16(oc[8 * v4 + 0] * inv, oc[8 * v4 + 1] * inv);
+          const uint32_t wy = pack_bf16(oc[8 * v4 + 2] * inv, oc[8 * v4 + 3] * inv);
+          const uint32_t wz = pack_bf16(oc[8 * v4 + 4] * inv, oc[8 * v4 + 5] * inv);
+          const uint32_t ww = pack_bf16(oc[8 * v4 + 6] * inv, oc[8 * v4 + 7] * inv);
+          const uint32_t addr = stage + (uint32_t)(cc >> 1) * kHalfBytes + ((uint32_t)(((cc & 1) * 4 + v4) ^ (row & 7)) << 4);
           asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(wx), "r"(wy), "r"(wz), "r"(ww) : "memory");
         }
       }
       fence_proxy_async();
-      mbar_arrive(bar(bOut + qt));
-      if (warp == 4) {
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(bOut + qt));
+      if (quarter == 0) {
         // one warp waits until all rows of the tile are staged; one of its lanes issues the stores
         ok = mbar_wait_warp(bar(bOut + qt), 0, abort_flag, status);
-        if (!ok) break;
-        if (elect_one()) {
+        if (ok && elect_one()) {
           const uint32_t src = base + kOffQ + qt * kTileBytes;
           tma_store_4d(&tmO, src, 0, q_first + qt * 128, h, b);
           tma_store_4d(&tmO, src + kHalfBytes, 64, q_first + qt * 128, h, b);
@@ -807,11 +799,10 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         }
         __syncwarp();
       }
-      if (prm.lse != nullptr && part == 0 && qi < n_k)
-        prm.lse[(size_t)slice * n_k + qi] = (m_used[qt] + log2f(lsum)) * 0.6931471805599453f;
-      if (wrank[qt] >= 0 && part == 0) prm.win_lse[(size_t)slice * prm.w + wrank[qt]] = m_used[qt] + log2f(lsum);
+      if (prm.lse != nullptr && qi < n_k) prm.lse[(size_t)slice * n_k + qi] = (m + log2f(l)) * 0.6931471805599453f;
+      if (wrank >= 0) prm.win_lse[(size_t)slice * prm.w + wrank] = m + log2f(l);
     }
-    if (warp == 4) tma_store_wait_all();      // (a lane that issued nothing has nothing to wait for)
+    if (quarter == 0) tma_store_wait_all();   // (a lane that issued nothing has nothing to wait for)
     tc_fence_before();
   }
   __syncthreads();
@@ -836,8 +827,6 @@ struct AttendTc {
   bool init(int dtype, int head_dim, void *k_pool, void *v_pool, long long n_pages, int page_tokens, std::string &err) {
     on = false;
     if (dtype != 0 || head_dim != 128) return true;   // f32 x 64 is served by the FMA kernel
-    const char *env = std::getenv("SCALEKV_ATTEND");
-    if (env && std::string(env) == "simt") return true;
     void *fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn) {

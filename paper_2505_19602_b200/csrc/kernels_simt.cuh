@@ -501,54 +501,39 @@ __global__ void head_budget_kernel(HeadBudgets hb, int n_heads, int n_slices, in
   const int s = blockIdx.x * blockDim.x + threadIdx.x;
   if (s < n_slices) slice_budget[s] = hb.v[s % n_heads];
 }
-// slice_budget: per-slice budgets (nullptr: every slice takes `budget`).
-__global__ void __launch_bounds__(1024) select_kernel(LayerView lv, WindowArg wa, int budget, const int *slice_budget, const uint32_t *keys,
-                                                      const float *scores, int pool, int ld_s, int *keep_list,
-                                                      int *kept_count) {
-  extern __shared__ uint32_t key[];            // [L]
-  __shared__ int hist[256];
-  __shared__ int warp_sums[33];
-  __shared__ uint32_t sh_prefix;
-  __shared__ int sh_remaining;
-  const int tid = threadIdx.x, lane = tid & 31;
-  const int slice = blockIdx.x;
-  const int dev_status = *reinterpret_cast<volatile int *>(lv.status);   // both loads in flight before the test
-  const int L = lv.hist_len[slice] + wa.n_k;
-  if (dev_status != 0) return;                 // an earlier kernel reported a failed check: leave the store alone
-  int *out = keep_list + (size_t)slice * ld_s;
+// Shared state of one selection (static shared memory of the calling kernel).
+struct SelectShared {
+  int hist[256];
+  int warp_sums[33];
+  uint32_t prefix;
+  int remaining;
+};
 
+// The selection proper, run by a whole CTA of 1024 threads: key[0 .. L) (shared or global memory) -> out[] = the
+// ascending slots of the survivors (the `budget` largest keys, equal keys by lowest slot, plus every sentinel
+// entry).  Returns the number of survivors; *kprime_plus_win receives the count the rule demands.
+__device__ __forceinline__ int select_and_emit(const uint32_t *key, int L, int budget, int *out, SelectShared &sh,
+                                                int *kprime_plus_win) {
+  const int tid = threadIdx.x, lane = tid & 31;
   int n_win_local = 0;
-  for (int i = tid; i < L; i += 1024) {
-    uint32_t k = __ldg(keys + (size_t)slice * ld_s + i);
-    if (pool > 1 && k != kWindowKey) {
-      // the importance averaged over `pool` neighbouring entries (zeros beyond both ends), summed in slot order
-      const float *sc = scores + (size_t)slice * ld_s;
-      const int r = pool >> 1;
-      float acc = 0.f;
-      for (int d = -r; d <= r; ++d)
-        if (i + d >= 0 && i + d < L) acc += __ldg(sc + i + d);
-      k = __float_as_uint(acc / (float)pool) & 0x7FFFFFFFu;
-    }
-    key[i] = k;
-    n_win_local += (k == kWindowKey) ? 1 : 0;
-  }
+  for (int i = tid; i < L; i += 1024) n_win_local += (key[i] == kWindowKey) ? 1 : 0;
   int n_win;
-  block_exclusive_scan(n_win_local, warp_sums, &n_win);
+  block_exclusive_scan(n_win_local, sh.warp_sums, &n_win);
   const int cand = L - n_win;
-  if (slice_budget != nullptr) budget = slice_budget[slice];
   const int kprime = (budget < 0 || budget > cand) ? cand : budget;
+  *kprime_plus_win = kprime + n_win;
 
   // radix select of the kprime-th largest key
   uint32_t threshold = 0;
   int n_ties_taken = 0;       // how many entries equal to the threshold are kept
   if (kprime > 0 && kprime < cand) {
-    if (tid == 0) { sh_prefix = 0; sh_remaining = kprime; }
+    if (tid == 0) { sh.prefix = 0; sh.remaining = kprime; }
     for (int pass = 0; pass < 4; ++pass) {
       const int shift = 24 - 8 * pass;
       const uint32_t mask_hi = pass == 0 ? 0u : (0xFFFFFFFFu << (shift + 8));
-      if (tid < 256) hist[tid] = 0;
+      if (tid < 256) sh.hist[tid] = 0;
       __syncthreads();
-      const uint32_t prefix = sh_prefix;
+      const uint32_t prefix = sh.prefix;
       for (int i0 = 0; i0 < L; i0 += 1024) {
         const int i = i0 + tid;
         const uint32_t k = i < L ? key[i] : kWindowKey;
@@ -556,20 +541,20 @@ __global__ void __launch_bounds__(1024) select_kernel(LayerView lv, WindowArg wa
         const uint32_t digit = in ? ((k >> shift) & 0xFFu) : 256u;
         // one shared-memory atomic per distinct digit in the warp
         const uint32_t peers = __match_any_sync(0xffffffffu, digit);
-        if (in && lane == (__ffs(peers) - 1)) atomicAdd(&hist[digit], __popc(peers));
+        if (in && lane == (__ffs(peers) - 1)) atomicAdd(&sh.hist[digit], __popc(peers));
       }
       __syncthreads();
       if (tid < 32) {
         // digits 255 .. 0 in descending order, 8 per lane; find where the running count reaches `rem`
         int c[8], tot = 0;
 #pragma unroll
-        for (int e = 0; e < 8; ++e) { c[e] = hist[255 - (lane * 8 + e)]; tot += c[e]; }
+        for (int e = 0; e < 8; ++e) { c[e] = sh.hist[255 - (lane * 8 + e)]; tot += c[e]; }
         int incl = tot;
         for (int o = 1; o < 32; o <<= 1) {
           const int t = __shfl_up_sync(0xffffffffu, incl, o);
           if (lane >= o) incl += t;
         }
-        const int rem = sh_remaining;
+        const int rem = sh.remaining;
         const int before = incl - tot;
         __syncwarp();
         if (before < rem && incl >= rem) {
@@ -577,17 +562,17 @@ __global__ void __launch_bounds__(1024) select_kernel(LayerView lv, WindowArg wa
 #pragma unroll
           for (int e = 0; e < 8; ++e) {
             if (r > 0) {
-              if (c[e] >= r) { dsel = 255 - (lane * 8 + e); sh_remaining = r; r = 0; }
+              if (c[e] >= r) { dsel = 255 - (lane * 8 + e); sh.remaining = r; r = 0; }
               else r -= c[e];
             }
           }
-          sh_prefix = prefix | ((uint32_t)dsel << shift);
+          sh.prefix = prefix | ((uint32_t)dsel << shift);
         }
       }
       __syncthreads();
     }
-    threshold = sh_prefix;
-    n_ties_taken = sh_remaining;
+    threshold = sh.prefix;
+    n_ties_taken = sh.remaining;
   }
   const bool keep_all = (kprime >= cand);
   const bool keep_none = (kprime == 0);
@@ -601,7 +586,7 @@ __global__ void __launch_bounds__(1024) select_kernel(LayerView lv, WindowArg wa
     n_tie += (k != kWindowKey && !keep_all && !keep_none && k == threshold) ? 1 : 0;
   }
   int tie_total, keep_total;
-  int tie_rank = block_exclusive_scan(n_tie, warp_sums, &tie_total);
+  int tie_rank = block_exclusive_scan(n_tie, sh.warp_sums, &tie_total);
   int n_keep = 0;
   {
     int tr = tie_rank;
@@ -618,7 +603,7 @@ __global__ void __launch_bounds__(1024) select_kernel(LayerView lv, WindowArg wa
       n_keep += keep ? 1 : 0;
     }
   }
-  int oidx = block_exclusive_scan(n_keep, warp_sums, &keep_total);
+  int oidx = block_exclusive_scan(n_keep, sh.warp_sums, &keep_total);
   for (int i = i_lo; i < i_hi; ++i) {
     const uint32_t k = key[i];
     bool keep = (k == kWindowKey);
@@ -631,10 +616,49 @@ __global__ void __launch_bounds__(1024) select_kernel(LayerView lv, WindowArg wa
     }
     if (keep) out[oidx++] = i;
   }
+  return keep_total;
+}
+
+// The importance averaged over `pool` neighbouring entries (zeros beyond both ends), summed in slot order.
+__device__ __forceinline__ uint32_t pooled_key(const float *sc, int i, int L, int pool) {
+  const int r = pool >> 1;
+  float acc = 0.f;
+  for (int d = -r; d <= r; ++d)
+    if (i + d >= 0 && i + d < L) acc += sc[i + d];
+  return __float_as_uint(acc / (float)pool) & 0x7FFFFFFFu;
+}
+
+// slice_budget: per-slice budgets (nullptr: every slice takes `budget`).
+// in_smem != 0: the slice's keys are staged in dynamic shared memory (4 * ld_s bytes); 0: a slice too long for
+// that is selected from the global key array as it stands (with pool > 1 the pooled keys are first written back
+// there), every pass streaming the keys through L2.
+__global__ void __launch_bounds__(1024) select_kernel(LayerView lv, WindowArg wa, int budget, const int *slice_budget, uint32_t *keys,
+                                                      const float *scores, int pool, int ld_s, int in_smem, int *keep_list,
+                                                      int *kept_count) {
+  extern __shared__ uint32_t key_sm[];         // [L] when in_smem
+  __shared__ SelectShared sh;
+  const int tid = threadIdx.x;
+  const int slice = blockIdx.x;
+  const int dev_status = *reinterpret_cast<volatile int *>(lv.status);   // both loads in flight before the test
+  const int L = lv.hist_len[slice] + wa.n_k;
+  if (dev_status != 0) return;                 // an earlier kernel reported a failed check: leave the store alone
+  int *out = keep_list + (size_t)slice * ld_s;
+  uint32_t *gkey = keys + (size_t)slice * ld_s;
+  const float *sc = scores + (size_t)slice * ld_s;
+  for (int i = tid; i < L; i += 1024) {
+    uint32_t k = gkey[i];
+    if (pool > 1 && k != kWindowKey) k = pooled_key(sc, i, L, pool);
+    if (in_smem) key_sm[i] = k;
+    else if (pool > 1) gkey[i] = k;
+  }
+  __syncthreads();
+  if (slice_budget != nullptr) budget = slice_budget[slice];
+  int want;
+  const int keep_total = select_and_emit(in_smem ? key_sm : gkey, L, budget, out, sh, &want);
   if (tid == 0) {
     kept_count[slice] = keep_total;
     // the count rule of the selection: k' candidates and every sentinel entry survive
-    if (keep_total != kprime + n_win) atomicExch(lv.status, kDevCheck);
+    if (keep_total != want) atomicExch(lv.status, kDevCheck);
   }
 }
 
@@ -646,12 +670,12 @@ __global__ void __launch_bounds__(1024) select_kernel(LayerView lv, WindowArg wa
 // depend on no further global look-up.  keep is ascending, so keep[j] >= j: within a chunk every
 // source is read before any destination is written, and the sources of later chunks lie beyond
 // every earlier destination.  256 threads, chunks of 2048 / ppq rows (ppq = pieces per row
-// quarter), 8 pieces in flight per thread.  Dynamic shared memory: 4 * (ld_s + pages_per_slice) B.
+// quarter), 8 pieces in flight per thread.  Dynamic shared memory: 4 * (pages_per_slice [+ ld_s]) B.
 // ------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) compact_kernel(LayerView lv, const int *keep_list, int ld_s, const int *kept_count) {
+__global__ void __launch_bounds__(256) compact_kernel(LayerView lv, const int *keep_list, int ld_s, int list_in_smem,
+                                                      const int *kept_count) {
   extern __shared__ int csm[];
-  int *list = csm;                 // [kept]
-  int *pt = csm + ld_s;            // [pages_per_slice]
+  int *pt = csm;                   // [pages_per_slice]
   const int slice = blockIdx.x;
   const int which = blockIdx.y;
   const int quarter = blockIdx.z;
@@ -659,7 +683,13 @@ __global__ void __launch_bounds__(256) compact_kernel(LayerView lv, const int *k
   const int dev_status = *reinterpret_cast<volatile int *>(lv.status);   // both loads in flight before the test
   const int kept = kept_count[slice];
   if (dev_status != 0) return;                 // the selection did not run: nothing to move
-  for (int i = threadIdx.x; i < kept; i += 256) list[i] = __ldg(keep_list + (size_t)slice * ld_s + i);
+  // the keep list is staged in shared memory when it fits ([kept] behind the page table), else read where it is
+  const int *list = keep_list + (size_t)slice * ld_s;
+  if (list_in_smem) {
+    int *ls = csm + lv.pages_per_slice;
+    for (int i = threadIdx.x; i < kept; i += 256) ls[i] = __ldg(list + i);
+    list = ls;
+  }
   for (int i = threadIdx.x; i < lv.pages_per_slice; i += 256) pt[i] = __ldg(lv.page_table + (size_t)slice * lv.pages_per_slice + i);
   __syncthreads();
   auto row_of = [&](int slot) { return ((size_t)pt[slot >> lv.page_shift] << lv.page_shift) + (size_t)(slot & lv.page_mask); };
@@ -700,6 +730,135 @@ __global__ void __launch_bounds__(256) compact_kernel(LayerView lv, const int *k
   }
   // no CTA of this kernel reads the length (the keep list's length is kept_count)
   if (do_pos_cta && threadIdx.x == 0) lv.hist_len[slice] = kept;
+}
+
+// ------------------------------------------------------------------------------------------
+// compress in one launch (Sec. 3.3, "KV Cache Selection"): importance, selection and pruning of one slice by one
+// CTA of 1024 threads, the phases separated by block barriers - what score_kernel, select_kernel and
+// compact_kernel do in three launches, for every slice whose keys and keep list fit in shared memory.
+//   phase 1  policy 0: s_i = (1/w) sum_j 2^(y_ji * logit_scale - lse_j) from the window rows' logits (see
+//            score_kernel) -> scores (global, kept for inspection and for the pooling) and radix keys (shared);
+//            policy 1: keys from the original positions (see recent_keys_kernel).
+//   phase 2  select_and_emit: radix select in shared memory, ascending keep list in shared memory.
+//   phase 3  slot j <- old slot keep[j] for K, V and pos, in chunks: every thread loads its 8 16-byte pieces of
+//            the chunk, block barrier, stores them (keep[j] >= j, see compact_kernel); the untouched prefix is skipped.
+// Dynamic shared memory: 4 * (2 * ld_s + pages_per_slice) bytes.  grid = n_slices.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(1024) compress_fused_kernel(LayerView lv, WindowArg wa, int policy, int n_sink,
+                                                              const float *logits, const float *lse, int ld_l, float logit_scale,
+                                                              int tile_padded, int budget, const int *slice_budget, int pool,
+                                                              float *scores, int ld_s, int *kept_count) {
+  extern __shared__ uint32_t fsm[];
+  uint32_t *key = fsm;                                   // [ld_s]
+  int *list = reinterpret_cast<int *>(fsm + ld_s);       // [ld_s]
+  int *pt = list + ld_s;                                 // [pages_per_slice]
+  __shared__ SelectShared sh;
+  __shared__ float lse_row[kMaxWindow];
+  const int tid = threadIdx.x;
+  const int slice = blockIdx.x;
+  const int dev_status = *reinterpret_cast<volatile int *>(lv.status);
+  const int hist = lv.hist_len[slice];
+  if (dev_status != 0) return;                 // an earlier kernel reported a failed check: leave the store alone
+  const int L = hist + wa.n_k;
+  const int w = wa.w;
+  for (int i = tid; i < lv.pages_per_slice; i += 1024) pt[i] = __ldg(lv.page_table + (size_t)slice * lv.pages_per_slice + i);
+  if (policy == 0 && tid < w) lse_row[tid] = lse[(size_t)slice * w + tid];
+  __syncthreads();
+  auto row_of = [&](int slot) { return ((size_t)pt[slot >> lv.page_shift] << lv.page_shift) + (size_t)(slot & lv.page_mask); };
+
+  // ---- phase 1: keys
+  float *sc_out = scores + (size_t)slice * ld_s;
+  if (policy == 0) {
+    const int pad = tile_padded ? ((((hist + 127) >> 7) << 7) - hist) : 0;     // the current map starts at a multiple of 128 columns
+    const float inv_w = 1.f / (float)w;
+    for (int i = tid; i < L; i += 1024) {
+      const float *y = logits + (size_t)slice * w * ld_l + (i >= hist ? i + pad : i);
+      float sc = 0.f;
+      int j = 0;
+      for (; j + 8 <= w; j += 8) {
+        float t[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) t[e] = __ldg(y + (size_t)(j + e) * ld_l);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) sc += exp2f(fmaf(t[e], logit_scale, -lse_row[j + e]));
+      }
+      for (; j < w; ++j) sc += exp2f(fmaf(__ldg(y + (size_t)j * ld_l), logit_scale, -lse_row[j]));
+      sc *= inv_w;
+      sc_out[i] = sc;
+      const bool win = is_window_pos(wa, lv.pos_pool[row_of(i)]);
+      key[i] = win ? kWindowKey : (__float_as_uint(sc) & 0x7FFFFFFFu);
+    }
+    if (pool > 1) {
+      __syncthreads();                         // this CTA's scores are visible to all of its threads
+      for (int i = tid; i < L; i += 1024)
+        if (key[i] != kWindowKey) list[i] = (int)pooled_key(sc_out, i, L, pool);
+      __syncthreads();
+      for (int i = tid; i < L; i += 1024)
+        if (key[i] != kWindowKey) key[i] = (uint32_t)list[i];
+    }
+  } else {
+    for (int i = tid; i < L; i += 1024) {
+      const int pos = lv.pos_pool[row_of(i)];
+      key[i] = pos < n_sink ? kWindowKey : (uint32_t)pos + 1u;
+    }
+  }
+  __syncthreads();
+
+  // ---- phase 2: selection
+  if (slice_budget != nullptr) budget = slice_budget[slice];
+  int want;
+  const int kept = select_and_emit(key, L, budget, list, sh, &want);
+  if (kept != want) {                          // the count rule of the selection (block-uniform)
+    if (tid == 0) atomicExch(lv.status, kDevCheck);
+    return;
+  }
+  __syncthreads();
+
+  // ---- phase 3: in-place gather of K, V and pos
+  const int ppr = lv.row_bytes >> 4;           // 16-byte pieces per row
+  const int per_row = 2 * ppr;                 // K pieces, then V pieces
+  const int r_step = 1024 / per_row;           // rows per sweep of the CTA
+  const int C = 8 * r_step;                    // rows per chunk
+  int lo = 0, hi = kept;                       // first j with keep[j] != j
+  while (lo < hi) {
+    const int mid = (lo + hi) >> 1;
+    if (list[mid] == mid) lo = mid + 1; else hi = mid;
+  }
+  const int r_in = tid / per_row, c = tid % per_row;
+  char *pool_ptr = c < ppr ? lv.k_pool : lv.v_pool;
+  const int piece = c < ppr ? c : c - ppr;
+  const bool pos_thread = c == 0;
+  if (r_in < r_step) {
+    for (int c0 = lo; c0 < kept; c0 += C) {
+      uint4 buf[8];
+      int pv[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int j = c0 + r_in + u * r_step;
+        if (j < kept) {
+          const size_t row = row_of(list[j]);
+          buf[u] = reinterpret_cast<const uint4 *>(pool_ptr + row * lv.row_bytes)[piece];
+          if (pos_thread) pv[u] = lv.pos_pool[row];
+        }
+      }
+      __syncthreads();
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int j = c0 + r_in + u * r_step;
+        if (j < kept) {
+          const size_t row = row_of(j);
+          reinterpret_cast<uint4 *>(pool_ptr + row * lv.row_bytes)[piece] = buf[u];
+          if (pos_thread) lv.pos_pool[row] = pv[u];
+        }
+      }
+    }
+  } else {
+    for (int c0 = lo; c0 < kept; c0 += C) __syncthreads();     // keeps the barrier count of the working threads
+  }
+  if (tid == 0) {
+    lv.hist_len[slice] = kept;
+    kept_count[slice] = kept;
+  }
 }
 
 // ------------------------------------------------------------------------------------------

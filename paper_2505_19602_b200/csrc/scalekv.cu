@@ -20,8 +20,8 @@ using namespace scalekv;
 
 namespace {
 
-constexpr int kNumClasses = 6;
-enum KernelClass { kAppend = 0, kAttend = 1, kScore = 2, kSelect = 3, kCompact = 4, kOther = 5 };
+constexpr int kNumClasses = 7;
+enum KernelClass { kAppend = 0, kAttend = 1, kScore = 2, kSelect = 3, kCompact = 4, kOther = 5, kCompress = 6 };
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -190,6 +190,14 @@ struct scalekv_ctx {
   std::vector<scalekv_tensor> pend_k, pend_v;   // the caller's tensors of a pending map that is not in the store yet
   std::vector<cudaEvent_t> ev_attend, ev_compress;
   std::vector<char> ev_compress_live;
+  std::vector<char> ev_compress_joined;   // stream_main has already waited for that compress (scalekv_join)
+  std::vector<char> map_lost;      // the layer's last map was attended and its transient rows then given to another layer
+  bool fused_ok = false;           // a slice's keys and keep list fit one CTA's shared memory: compress is one launch
+  bool select_smem_ok = false;     // the separate select kernel can stage a slice's keys in shared memory
+  bool compact_smem_ok = false;    // the separate compact kernel can stage a slice's keep list in shared memory
+  size_t fused_smem = 0;
+  bool side_dirty = false;         // stream_side has work that stream_main has not joined yet
+  int set_owner[2] = {-1, -1};     // layer that last appended into the transient page set / logit buffer of each parity
   int64_t launches = 0;
   int scores_len = 0;              // length of the score vectors left by the last evicting compress
   bool profile = false;            // launches are bracketed by events
@@ -248,7 +256,7 @@ bool tensor_ok(const scalekv_tensor &t, int esize) {
 }
 
 const char *const kClassNames[kNumClasses] = {"scalekv.append", "scalekv.attend", "scalekv.score", "scalekv.select",
-                                               "scalekv.compact", "scalekv.other"};
+                                               "scalekv.compact", "scalekv.other", "scalekv.compress"};
 
 struct Scope {  // brackets one launch with an NVTX range and, when profiling, with events; counts launches
   scalekv_ctx *c; cudaStream_t s; int cls; cudaEvent_t a = nullptr, b = nullptr;
@@ -256,17 +264,22 @@ struct Scope {  // brackets one launch with an NVTX range and, when profiling, w
     nvtxRangePushA(kClassNames[cls]);
     if (c->profile) {
       a = take(); b = take();
-      cudaEventRecord(a, s);
+      if (a && b) cudaEventRecord(a, s);
     }
   }
   cudaEvent_t take() {
     if (!c->event_pool.empty()) { cudaEvent_t e = c->event_pool.back(); c->event_pool.pop_back(); return e; }
-    cudaEvent_t e; cudaEventCreate(&e); return e;
+    cudaEvent_t e = nullptr;
+    if (cudaEventCreate(&e) != cudaSuccess) { cudaGetLastError(); return nullptr; }   // this launch goes untimed
+    return e;
   }
   ~Scope() {
     nvtxRangePop();
     c->launches++;
-    if (c->profile) { cudaEventRecord(b, s); c->timed.push_back({a, b, cls}); }
+    if (c->profile) {
+      if (a && b) { cudaEventRecord(b, s); c->timed.push_back({a, b, cls}); }
+      else { if (a) c->event_pool.push_back(a); if (b) c->event_pool.push_back(b); }
+    }
   }
 };
 
@@ -279,8 +292,12 @@ void drain_profile(scalekv_ctx *c) {
   c->timed.clear();
 }
 
-template <typename F> void set_smem(F *f, size_t bytes) {
-  cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+// Raises a kernel's dynamic shared-memory limit; false when the device cannot give that much.
+template <typename F> bool set_smem(F *f, size_t bytes) {
+  if (bytes > (size_t)0x7fffffff) return false;
+  if (cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) == cudaSuccess) return true;
+  cudaGetLastError();
+  return false;
 }
 
 scalekv_status check_launch(scalekv_ctx *ctx, const char *what) {
@@ -418,22 +435,38 @@ scalekv_status scalekv_init(const scalekv_config *cfg, scalekv_ctx **out) {
   ctx->pend_k.resize(p.n_layers); ctx->pend_v.resize(p.n_layers);
   ctx->ev_attend.resize(p.n_layers); ctx->ev_compress.resize(p.n_layers);
   ctx->ev_compress_live.assign(p.n_layers, 0);
+  ctx->ev_compress_joined.assign(p.n_layers, 0);
+  ctx->map_lost.assign(p.n_layers, 0);
   for (int l = 0; l < p.n_layers; ++l) {
     if (cudaEventCreateWithFlags(&ctx->ev_attend[l], cudaEventDisableTiming) != cudaSuccess) return bail(SCALEKV_ERR_CUDA);
     if (cudaEventCreateWithFlags(&ctx->ev_compress[l], cudaEventDisableTiming) != cudaSuccess) return bail(SCALEKV_ERR_CUDA);
   }
-  if (cfg->dtype == SCALEKV_BF16) {
-    set_smem(attend_simt_kernel<__nv_bfloat16, 128>, (64 * 132 * 2 + 64 * 65 + 192) * 4);
-    set_smem(score_logits_kernel<__nv_bfloat16, 128>, 2 * 64 * 132 * 4);
-    set_smem(layer_stats_kernel<__nv_bfloat16, 128>, (size_t)(128 + p.ld_s) * 4);
-  } else {
-    set_smem(attend_simt_kernel<float, 64>, (64 * 68 * 2 + 64 * 65 + 192) * 4);
-    set_smem(score_logits_kernel<float, 64>, 2 * 64 * 68 * 4);
-    set_smem(layer_stats_kernel<float, 64>, (size_t)(64 + p.ld_s) * 4);
+  {
+    // every kernel that sizes its shared memory from the schedule is checked now, so that a configuration the
+    // kernels cannot take is refused here and not at its first launch
+    bool ok = true;
+    if (cfg->dtype == SCALEKV_BF16) {
+      ok = ok && set_smem(attend_simt_kernel<__nv_bfloat16, 128>, (64 * 132 * 2 + 64 * 65 + 192) * 4);
+      ok = ok && set_smem(score_logits_kernel<__nv_bfloat16, 128>, 2 * 64 * 132 * 4);
+      ok = ok && set_smem(layer_stats_kernel<__nv_bfloat16, 128>, (size_t)(128 + p.ld_s) * 4);
+    } else {
+      ok = ok && set_smem(layer_stats_kernel<float, 64>, (size_t)(64 + p.ld_s) * 4);
+      ok = ok && set_smem(attend_simt_kernel<float, 64>, (64 * 68 * 2 + 64 * 65 + 192) * 4);
+      ok = ok && set_smem(score_logits_kernel<float, 64>, 2 * 64 * 68 * 4);
+    }
+    // select and compact stage a slice in shared memory when it fits and work from global memory when it does not
+    int max_pages = 0;
+    for (const LayerPlan &lp : p.layers) max_pages = std::max(max_pages, lp.total_pages);
+    ctx->select_smem_ok = set_smem(select_kernel, (size_t)p.ld_s * 4);
+    ctx->compact_smem_ok = set_smem(compact_kernel, (size_t)(p.ld_s + max_pages) * 4);
+    if (!ctx->compact_smem_ok) ok = ok && set_smem(compact_kernel, (size_t)max_pages * 4);
+    ctx->fused_smem = (size_t)(2 * p.ld_s + max_pages) * 4;
+    ctx->fused_ok = set_smem(compress_fused_kernel, ctx->fused_smem);
+    if (!ok) {
+      fprintf(stderr, "scalekv_init: a slice of up to %d entries needs more shared memory than a CTA of this device has\n", p.ld_s);
+      return bail(SCALEKV_ERR_UNSUPPORTED);
+    }
   }
-  set_smem(select_kernel, (size_t)p.ld_s * 4);
-  set_smem(compact_kernel, (size_t)(p.ld_s + (p.ld_s + p.P - 1) / p.P + 1) * 4);
-  cudaGetLastError();
   std::string tc_err;
   if (!ctx->tc.init(cfg->dtype, p.d, ctx->pool + p.off_k, ctx->pool + p.off_v, p.n_pages, p.P, tc_err)) {
     scalekv_status s = fail(ctx, SCALEKV_ERR_CUDA, "tensor-core attend set-up failed: %s", tc_err.c_str());
@@ -469,6 +502,9 @@ scalekv_status scalekv_reset(scalekv_ctx *ctx) {
   std::fill(ctx->in_store.begin(), ctx->in_store.end(), 1);
   std::fill(ctx->logits_of.begin(), ctx->logits_of.end(), -1);
   std::fill(ctx->ev_compress_live.begin(), ctx->ev_compress_live.end(), 0);
+  ctx->set_owner[0] = ctx->set_owner[1] = -1;
+  ctx->side_dirty = ctx->s_side != ctx->s_main;   // the side stream was sent behind the reset: a capture has to join it again
+  std::fill(ctx->map_lost.begin(), ctx->map_lost.end(), 0);
   return SCALEKV_OK;
 }
 
@@ -500,17 +536,29 @@ scalekv_status scalekv_append(scalekv_ctx *ctx, int32_t layer, int32_t scale, sc
   if (scale != ctx->next_scale[layer])
     return fail(ctx, SCALEKV_ERR_BAD_STATE, "layer %d expects scale %d, got %d", layer, ctx->next_scale[layer], scale);
   if (!tensor_ok(K, p.esize) || !tensor_ok(V, p.esize)) return fail(ctx, SCALEKV_ERR_INVALID_ARG, "K/V null or rows not 16-byte aligned");
-  // the previous compress of this layer, and the compress of the layer that last used the same
-  // transient page set, must have finished
-  if (ctx->s_side != ctx->s_main) {
-    if (ctx->ev_compress_live[layer]) CU(cudaStreamWaitEvent(ctx->s_main, ctx->ev_compress[layer], 0));
-    const int other = layer >= 2 ? layer - 2 : -1;
-    if (other >= 0 && ctx->ev_compress_live[other]) CU(cudaStreamWaitEvent(ctx->s_main, ctx->ev_compress[other], 0));
-    if (layer < 2 && scale > 0) {
-      // transient set reuse across scales: the last layer of this parity at the previous scale
-      for (int o = p.n_layers - 1; o >= 0; --o)
-        if ((o & 1) == (layer & 1)) { if (ctx->ev_compress_live[o]) CU(cudaStreamWaitEvent(ctx->s_main, ctx->ev_compress[o], 0)); break; }
+  // The transient page set and the logit buffer of this layer's parity are shared with every other layer of
+  // that parity.  Their last user (the owner) must be through with them: a pending map of the owner whose
+  // rows reach into the transient pages would be overwritten, so that order of calls is refused; otherwise
+  // stream_main waits for the owner's last compress (and for this layer's own).
+  const int par = layer & 1;
+  const int owner = ctx->set_owner[par];
+  if (owner >= 0 && owner != layer && ctx->pending[owner] != 0) {
+    const LayerPlan &op = p.layers[owner];
+    if (ctx->hist[owner] + ctx->pending[owner] > op.persist_pages * p.P) {
+      // the one map that nothing needs after its attend is the last scale's (no later step reads it): its
+      // transient rows may go, and the layer then accepts nothing but a reset
+      if (ctx->next_scale[owner] == p.K && ctx->attended[owner]) ctx->map_lost[owner] = 1;
+      else
+        return fail(ctx, SCALEKV_ERR_BAD_STATE,
+                    "layer %d: layer %d still holds an uncompressed map in the transient pages both layers share; compress it first",
+                    layer, owner);
     }
+    ctx->logits_of[owner] = -1;      // its recorded window logits are about to be overwritten: score from K instead
+  }
+  if (ctx->s_side != ctx->s_main) {
+    if (ctx->ev_compress_live[layer] && !ctx->ev_compress_joined[layer]) CU(cudaStreamWaitEvent(ctx->s_main, ctx->ev_compress[layer], 0));
+    if (owner >= 0 && owner != layer && ctx->ev_compress_live[owner] && !ctx->ev_compress_joined[owner])
+      CU(cudaStreamWaitEvent(ctx->s_main, ctx->ev_compress[owner], 0));
   }
   scalekv_status st = materialize(ctx, layer);
   if (st != SCALEKV_OK) return st;
@@ -533,6 +581,7 @@ scalekv_status scalekv_append(scalekv_ctx *ctx, int32_t layer, int32_t scale, sc
   ctx->pending[layer] = nk;
   ctx->attended[layer] = 0;
   ctx->next_scale[layer] = scale + 1;
+  ctx->set_owner[par] = layer;
   return check_launch(ctx, "append");
 }
 
@@ -591,6 +640,7 @@ scalekv_status scalekv_compress_ex(scalekv_ctx *ctx, int32_t layer, scalekv_tens
   const Plan &p = ctx->plan;
   if (layer < 0 || layer >= p.n_layers) return fail(ctx, SCALEKV_ERR_INVALID_ARG, "layer %d out of range", layer);
   if (ctx->pending[layer] == 0) return fail(ctx, SCALEKV_ERR_BAD_STATE, "layer %d: compress needs a preceding append", layer);
+  if (ctx->map_lost[layer]) return fail(ctx, SCALEKV_ERR_BAD_STATE, "layer %d: the rows of its last map were handed to another layer after its attend", layer);
   const int policy = opts ? opts->policy : SCALEKV_SELECT_SCORE;
   const int pool = (opts && opts->pool_kernel > 1) ? opts->pool_kernel : 1;
   const int n_sink = opts ? opts->n_sink : 0;
@@ -612,6 +662,14 @@ scalekv_status scalekv_compress_ex(scalekv_ctx *ctx, int32_t layer, scalekv_tens
     wa.w = 0; wa.all = 0; wa.n_prev = p.N[k]; wa.n_k = p.n[k];
     for (int j = 0; j < kMaxWindow; ++j) wa.pos[j] = 0x7fffffff;
     always_kept = std::min(n_sink, p.N[k + 1]);          // positions 0 .. n_sink-1 are never evicted once appended
+    {
+      // the pages were sized for the table's value: sinks beyond it would be left in pages shared with other layers
+      const int tab = p.budgets[(size_t)layer * p.K + k];
+      const LayerPlan &lp = p.layers[layer];
+      if (tab != SCALEKV_KEEP_ALL && lp.persist_pages < lp.total_pages && std::max(tab, always_kept) > lp.persist_pages * p.P)
+        return fail(ctx, SCALEKV_ERR_CAPACITY, "layer %d: %d sinks exceed the persistent capacity %d planned from the budget table",
+                    layer, always_kept, lp.persist_pages * p.P);
+    }
   } else {
     if (!tensor_ok(Qw, p.esize)) return fail(ctx, SCALEKV_ERR_INVALID_ARG, "Qw null or rows not 16-byte aligned");
     st = fill_window(ctx, layer, w, window_pos, wa);
@@ -660,13 +718,23 @@ scalekv_status scalekv_compress_ex(scalekv_ctx *ctx, int32_t layer, scalekv_tens
     int *keep = reinterpret_cast<int *>(ctx->ws + p.off_keep);
     int *kept = reinterpret_cast<int *>(ctx->ws + p.off_kept);
     uint32_t *keys = reinterpret_cast<uint32_t *>(ctx->ws + p.off_keys);
-    if (recent) {
+    const bool fused = ctx->fused_ok && !head_shared && !(opts && opts->separate_kernels);
+    if (recent && !fused) {
       Scope sc(ctx, s, kScore);
       recent_keys_kernel<<<dim3((L + 255) / 256, p.n_slices), 256, 0, s>>>(lv, wa.n_k, n_sink, keys, p.ld_s);
     }
     // the logits of exactly this window may already be there, recorded by attend
     bool recorded = recent || (ctx->logits_of[layer] == k && (int)p.windows[k].size() == wa.w);
     for (int j = 0; !recent && recorded && j < wa.w; ++j) recorded = p.windows[k][j] == wa.pos[j];
+    if (!recorded) {
+      // this writes the logit buffer of the layer's parity: if another layer of that parity has appended since, what
+      // its attend recorded there is lost (its compress scores from K too), and its attend must be through first
+      const int ow = ctx->set_owner[layer & 1];
+      if (ow >= 0 && ow != layer) {
+        ctx->logits_of[ow] = -1;
+        if (s != ctx->s_main && ctx->attended[ow]) CU(cudaStreamWaitEvent(s, ctx->ev_attend[ow], 0));
+      }
+    }
     if (!recorded) {
       Scope sc(ctx, s, kScore);
       dim3 grid((L + 63) / 64, p.n_slices);
@@ -683,30 +751,40 @@ scalekv_status scalekv_compress_ex(scalekv_ctx *ctx, int32_t layer, scalekv_tens
       Scope sc(ctx, s, kScore);
       row_lse_kernel<<<p.n_slices, 1024, 0, s>>>(lv, wa, logits, p.ld_l, wlse);
     }
-    if (!recent) {
-      Scope sc(ctx, s, kScore);
-      // logits recorded by attend are raw products in the tile-aligned layout; the logits kernel writes base-2 logits by slot
-      score_kernel<<<dim3((L + 255) / 256, p.n_slices), 256, 0, s>>>(lv, wa, logits, wlse, p.ld_l, recorded ? ctx->scale * 1.4426950408889634f : 1.f,
-                                                                     (recorded && ctx->logits_padded[layer]) ? 1 : 0, scores, keys, p.ld_s);
-    }
-    if (head_shared) {
-      Scope sc(ctx, s, kScore);
-      head_mean_kernel<<<dim3((L + 255) / 256, p.n_slices / p.H), 256, 0, s>>>(lv, wa, scores, keys, p.ld_s);
-    }
+    // logits recorded by attend are raw products in the tile-aligned layout; the logits kernel writes base-2 logits by slot
+    const float logit_scale = recorded ? ctx->scale * 1.4426950408889634f : 1.f;
+    const int tile_padded = (recorded && ctx->logits_padded[layer]) ? 1 : 0;
     int *slice_budget = nullptr;
     if (hb_on) {
       slice_budget = reinterpret_cast<int *>(ctx->ws + p.off_hbud);
       Scope sc(ctx, s, kSelect);
       head_budget_kernel<<<(p.n_slices + 255) / 256, 256, 0, s>>>(hb, p.H, p.n_slices, slice_budget);
     }
-    {
-      Scope sc(ctx, s, kSelect);
-      select_kernel<<<p.n_slices, 1024, (size_t)p.ld_s * 4, s>>>(lv, wa, budget, slice_budget, keys, recent ? nullptr : scores, pool, p.ld_s,
-                                                                 keep, kept);
-    }
-    {
-      Scope sc(ctx, s, kCompact);
-      compact_kernel<<<dim3(p.n_slices, 2, 4), 256, (size_t)(p.ld_s + lv.pages_per_slice) * 4, s>>>(lv, keep, p.ld_s, kept);
+    if (fused) {
+      // importance, selection and pruning of a slice by one CTA, in one launch
+      Scope sc(ctx, s, kCompress);
+      compress_fused_kernel<<<p.n_slices, 1024, ctx->fused_smem, s>>>(lv, wa, recent ? 1 : 0, n_sink, logits, wlse, p.ld_l, logit_scale,
+                                                                     tile_padded, budget, slice_budget, pool, scores, p.ld_s, kept);
+    } else {
+      if (!recent) {
+        Scope sc(ctx, s, kScore);
+        score_kernel<<<dim3((L + 255) / 256, p.n_slices), 256, 0, s>>>(lv, wa, logits, wlse, p.ld_l, logit_scale, tile_padded, scores,
+                                                                       keys, p.ld_s);
+      }
+      if (head_shared) {
+        Scope sc(ctx, s, kScore);
+        head_mean_kernel<<<dim3((L + 255) / 256, p.n_slices / p.H), 256, 0, s>>>(lv, wa, scores, keys, p.ld_s);
+      }
+      {
+        Scope sc(ctx, s, kSelect);
+        select_kernel<<<p.n_slices, 1024, ctx->select_smem_ok ? (size_t)p.ld_s * 4 : 0, s>>>(
+            lv, wa, budget, slice_budget, keys, recent ? nullptr : scores, pool, p.ld_s, ctx->select_smem_ok ? 1 : 0, keep, kept);
+      }
+      {
+        Scope sc(ctx, s, kCompact);
+        const size_t sm = (size_t)(lv.pages_per_slice + (ctx->compact_smem_ok ? p.ld_s : 0)) * 4;
+        compact_kernel<<<dim3(p.n_slices, 2, 4), 256, sm, s>>>(lv, keep, p.ld_s, ctx->compact_smem_ok ? 1 : 0, kept);
+      }
     }
     ctx->scores_len = recent ? 0 : L;
     ctx->hist[layer] = budget + always_kept;
@@ -717,7 +795,9 @@ scalekv_status scalekv_compress_ex(scalekv_ctx *ctx, int32_t layer, scalekv_tens
   }
   if (s != ctx->s_main) {
     CU(cudaEventRecord(ctx->ev_compress[layer], s));
+    ctx->side_dirty = true;
     ctx->ev_compress_live[layer] = 1;
+    ctx->ev_compress_joined[layer] = 0;
   }
   return SCALEKV_OK;
 }
@@ -804,6 +884,7 @@ scalekv_status scalekv_layer_stats_ex(scalekv_ctx *ctx, int32_t layer, scalekv_t
   const Plan &p = ctx->plan;
   if (layer < 0 || layer >= p.n_layers) return fail(ctx, SCALEKV_ERR_INVALID_ARG, "layer %d out of range", layer);
   if (ctx->pending[layer] == 0) return fail(ctx, SCALEKV_ERR_BAD_STATE, "layer %d: layer_stats needs a preceding append", layer);
+  if (ctx->map_lost[layer]) return fail(ctx, SCALEKV_ERR_BAD_STATE, "layer %d: the rows of its last map were handed to another layer after its attend", layer);
   if (topk_prime < 0 || topk_prime > 64 || query_stride < 1) return fail(ctx, SCALEKV_ERR_INVALID_ARG, "topk_prime in [0,64], stride >= 1");
   if (!tensor_ok(Q, p.esize)) return fail(ctx, SCALEKV_ERR_INVALID_ARG, "Q null or rows not 16-byte aligned");
   scalekv_status st0 = materialize(ctx, layer);
@@ -902,11 +983,50 @@ scalekv_status scalekv_make_budgets(const uint8_t *is_drafter, int32_t L, int32_
   return SCALEKV_OK;
 }
 
+scalekv_status scalekv_budget_tokens(double fraction, const int32_t *scale_h, const int32_t *scale_w, int32_t n_scales,
+                                     int32_t *tokens) {
+  if (!scale_h || !scale_w || !tokens || n_scales < 1 || !(fraction >= 0.0)) return SCALEKV_ERR_INVALID_ARG;
+  long long t_c = 0;
+  for (int k = 0; k + 1 < n_scales; ++k) {
+    if (scale_h[k] < 1 || scale_w[k] < 1) return SCALEKV_ERR_INVALID_ARG;
+    t_c += (long long)scale_h[k] * scale_w[k];
+  }
+  const double v = std::floor(fraction * (double)t_c + 0.5 + 1e-9);   // a decimal fraction that lands on .5 rounds up
+  if (v > 2147483647.0) return SCALEKV_ERR_INVALID_ARG;
+  *tokens = (int32_t)v;
+  return SCALEKV_OK;
+}
+
+scalekv_status scalekv_selftest_wait(scalekv_ctx *ctx, int32_t limit_ms, int32_t *gave_up, int32_t *seen_by_peer) {
+  if (!ctx || !gave_up || !seen_by_peer) return SCALEKV_ERR_INVALID_ARG;
+  if (limit_ms < 1 || limit_ms > 1000) return fail(ctx, SCALEKV_ERR_INVALID_ARG, "limit_ms must lie in [1, 1000]");
+  const Plan &p = ctx->plan;
+  int *out = reinterpret_cast<int *>(ctx->ws + p.off_acc);
+  CU(cudaMemsetAsync(out, 0, 8, ctx->s_main));
+  {
+    Scope sc(ctx, ctx->s_main, kOther);
+    tc::wait_probe_kernel<<<1, 64, 0, ctx->s_main>>>(reinterpret_cast<int *>(ctx->pool + p.off_status),
+                                                     (unsigned long long)limit_ms * 1000000ull, out);
+  }
+  scalekv_status st = check_launch(ctx, "wait probe");
+  if (st != SCALEKV_OK) return st;
+  int host[2] = {0, 0};
+  CU(cudaMemcpyAsync(host, out, 8, cudaMemcpyDeviceToHost, ctx->s_main));
+  CU(cudaStreamSynchronize(ctx->s_main));
+  *gave_up = host[0];
+  *seen_by_peer = host[1];
+  return SCALEKV_OK;
+}
+
 scalekv_status scalekv_join(scalekv_ctx *ctx) {
   if (!ctx) return SCALEKV_ERR_INVALID_ARG;
-  if (ctx->s_side != ctx->s_main) {
+  if (ctx->s_side != ctx->s_main && ctx->side_dirty) {   // (nothing enqueued there since the last join: nothing to wait for)
     CU(cudaEventRecord(ctx->ev_join, ctx->s_side));
     CU(cudaStreamWaitEvent(ctx->s_main, ctx->ev_join, 0));
+    // stream_main is now behind every compress enqueued so far: later appends need not wait for them again
+    // (which also lets the next scale-step be captured into a graph of its own)
+    std::fill(ctx->ev_compress_joined.begin(), ctx->ev_compress_joined.end(), 1);
+    ctx->side_dirty = false;
   }
   return SCALEKV_OK;
 }
@@ -948,7 +1068,7 @@ scalekv_status scalekv_export_slice(scalekv_ctx *ctx, int32_t layer, int32_t b, 
   const int slice = b * p.H + h;
   int hist = 0;
   CU(cudaMemcpy(&hist, ctx->pool + p.off_len + ((size_t)layer * p.n_slices + slice) * 4, 4, cudaMemcpyDeviceToHost));
-  const int L = hist + ctx->pending[layer];
+  const int L = hist + (ctx->map_lost[layer] ? 0 : ctx->pending[layer]);   // a given-up last map is not exported
   *len = L;
   if (L > cap) return fail(ctx, SCALEKV_ERR_CAPACITY, "slice holds %d entries, cap is %d", L, cap);
   const LayerPlan &lp = p.layers[layer];

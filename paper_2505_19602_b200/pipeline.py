@@ -16,15 +16,10 @@ def windows_for(sides, n_patches=16):
     return [binding.scalekv_window_centroids(a, a, n_patches) for a in sides]
 
 
-def pct_budget(fraction_num, fraction_den, t_c):
-    """round-half-up of (num/den) * T_c in integers."""
-    return (2 * fraction_num * t_c + fraction_den) // (2 * fraction_den)
-
-
-def budget_table(wl: synth.Workload, roles, drafter_pct=(30, 100), refiner_pct=(3, 100)):
-    """budgets[l][k]: drafter or refiner budget by role (percentages of T_c = N_{K-1})."""
-    t_c = sum(wl.n_tokens[:-1])
-    bd, br = pct_budget(*drafter_pct, t_c), pct_budget(*refiner_pct, t_c)
+def budget_table(wl: synth.Workload, roles, drafter_frac=0.30, refiner_frac=0.03):
+    """budgets[l][k]: drafter or refiner budget by role (fractions of T_c = N_{K-1}, scalekv_budget_tokens)."""
+    bd = binding.scalekv_budget_tokens(drafter_frac, wl.sides)
+    br = binding.scalekv_budget_tokens(refiner_frac, wl.sides)
     return [[bd if roles[l][k] else br for k in range(wl.n_scales)] for l in range(wl.n_layers)]
 
 
@@ -128,6 +123,8 @@ def pass_work(wl: synth.Workload, budgets, windows):
     score_bytes       the score kernel: w x L logits and L positions in, L scores and L keys out (plus K read
                       by the stand-alone logits kernel when attend did not record the logits).
     select_bytes      the select kernel: L keys in, the keep list out.
+    compress_bytes    the one-launch compress (score + select + compact of a slice by one CTA): the w x L logits and
+                      L positions in, L scores out, the survivors' rows moved; keys and keep list stay on chip.
     compact_bytes     K and V rows (and positions) of the survivors, read and written (upper bound: which
                       rows already sit in place is unknown on the host).
     """
@@ -137,7 +134,7 @@ def pass_work(wl: synth.Workload, budgets, windows):
     slices = wl.batch * wl.n_heads
     fused = wl.dtype == "bf16" and d == 128
     out = {"attend_flop": 0, "attend_min_bytes": 0, "score_bytes": 0, "compact_bytes": 0, "append_bytes": 0,
-           "select_bytes": 0, "attend_launches": 0}
+           "select_bytes": 0, "attend_launches": 0, "compress_bytes": 0, "compress_launches": 0}
     per_scale_flop = [0] * wl.n_scales
     for l in range(wl.n_layers):
         hist = 0
@@ -163,6 +160,9 @@ def pass_work(wl: synth.Workload, budgets, windows):
                 out["score_bytes"] += (4 * w * L + 4 * L + 4 * L + 4 * L) * slices
                 out["select_bytes"] += (4 * L + 4 * (b + w)) * slices
                 out["compact_bytes"] += (b + w) * (2 * 2 * d * esz + 8) * slices
+                # the one-launch compress: logits and positions in, scores out, the survivors' rows moved
+                out["compress_bytes"] += ((4 * w * L + 4 * L + 4 * L) + (b + w) * (2 * 2 * d * esz + 8)) * slices
+                out["compress_launches"] += 1
                 hist = b + w
             else:
                 hist = L

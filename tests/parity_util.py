@@ -32,9 +32,11 @@ class ParityRun:
         self.caches = {s: orc.SliceCache(self.n, kv.head_dim) for s in slices}
         self.resyncs = 0
         self.max_err = 0.0
-        self.max_tol = 0.0
         self.max_lse_err = 0.0
         self.evictions = 0
+        self.separate_kernels = False  # compress as three launches (the path long slices take) instead of one
+        self.compared = 0             # slice-steps whose attention output was compared
+        self.rel_bound_used = 0       # ... of which the relative branch of the bf16 bound (|O| > 2.56) decided
 
     def run(self):
         kv = self.kv
@@ -51,7 +53,9 @@ class ParityRun:
                 O = kv.scalekv_attend(l, Qd, lse=lse)
                 do_compress = (k + 1 < len(self.n)) or self.compress_last
                 if do_compress:
-                    if wpos is None:
+                    if self.separate_kernels:
+                        kv.scalekv_compress_ex(l, Qd, wpos, qw_is_full_map=True, separate_kernels=True)
+                    elif wpos is None:
                         kv.scalekv_compress(l, Qd, None)
                     else:
                         # alternate between the two ways of passing the window rows
@@ -70,7 +74,119 @@ class ParityRun:
                                         to64(Oh[b, h]), to64(lseh[b, h]), wpos, do_compress)
         return self
 
-    def _compare_slice(self, key, k, Q, K, V, O_gpu, lse_gpu, wpos, do_compress):
+    def summary(self):
+        return (f"{self.compared} slice-steps compared, max |O - oracle| = {self.max_err:.3e}, relative bound decided "
+                f"{self.rel_bound_used} of them, {self.evictions} evicting compressions, {self.resyncs} tie-band re-syncs")
+
+    # ---- the execution mode the benchmark times -------------------------------------------------------------
+    def run_pipelined(self, mode="eager", device_inputs=False):
+        """One scalekv_step per layer and scale - compress of layer l on the side stream under attend of layer
+        l + 1, transient page sets and logit buffers handed from layer l to layer l + 2 - with NO host
+        synchronisation between the layers of a scale-step.  The host syncs once per scale-step (the kept set a
+        compress leaves stays readable until the layer's next compress), exports every followed slice and lets
+        the oracle compare and, inside the tie band, re-sync.
+        mode "eager": the calls as they are.  mode "graph": the calls of every scale-step are captured on
+        stream_main into a CUDA graph (compress forks to the side stream inside the capture) and the graph is
+        replayed."""
+        kv = self.kv
+        n_layers = kv.n_layers
+        if mode == "graph":
+            kv.scalekv_reset()          # a capture must not start inside another stream's pending work
+            kv.scalekv_sync()
+        for k, nk in enumerate(self.n):
+            wpos = self.window_fn(k)
+            do_compress = (k + 1 < len(self.n)) or self.compress_last
+            host, dev, O, lse = {}, {}, {}, {}
+            for l in range(n_layers):
+                Q, K, V = self.inputs_fn(l, k)
+                dev[l] = (Q.cuda(), K.cuda(), V.cuda())
+                host[l] = (Q, K, V)
+                O[l] = torch.zeros_like(dev[l][0])
+                lse[l] = torch.zeros(kv.batch, kv.n_heads, nk, dtype=torch.float32, device="cuda")
+            torch.cuda.synchronize()
+            wp = kv.window_array(wpos) if (do_compress and wpos is not None) else None
+
+            def steps():
+                for l in range(n_layers):
+                    Qd, Kd, Vd = dev[l]
+                    kv.scalekv_step(l, k, Qd, Kd, Vd, O[l], window_pos=wp, whole_map=do_compress and wp is None, lse=lse[l])
+
+            if mode == "graph":
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=kv.stream_main):
+                    steps()
+                    kv.scalekv_join()
+                with torch.cuda.stream(kv.stream_main):
+                    g.replay()
+            else:
+                steps()
+            kv.scalekv_sync()
+            for l in sorted({s[0] for s in self.slices}):
+                Q, K, V = host[l]
+                Oh, lseh = O[l].cpu(), lse[l].cpu()
+                for (sl, b, h) in [s for s in self.slices if s[0] == l]:
+                    Qs, Ks, Vs = (t[b, h].cpu() for t in (Q, K, V))
+                    self._compare_slice((sl, b, h), k, to64(Qs), to64(Ks), to64(Vs), to64(Oh[b, h]), to64(lseh[b, h]), wpos,
+                                        do_compress, scores_fresh=(l == n_layers - 1))
+        return self
+
+    def run_graph_pass(self):
+        """The whole pass - reset, then every scale and layer - captured into ONE CUDA graph and replayed twice,
+        which is what the benchmark's timed region does.  Nothing can be exported between the scales of a replay,
+        so the oracle walks the pass with its own selections (no re-sync possible: use inputs for which
+        run_pipelined reports zero re-syncs) and compares every layer's output of every scale, and at the end the
+        positions and K/V rows every followed slice holds."""
+        kv = self.kv
+        n_layers, K_s = kv.n_layers, len(self.n)
+        host, dev, O, lse = {}, {}, {}, {}
+        for k, nk in enumerate(self.n):
+            for l in range(n_layers):
+                Q, K, V = self.inputs_fn(l, k)
+                host[(l, k)] = (Q, K, V)
+                dev[(l, k)] = (Q.cuda(), K.cuda(), V.cuda())
+                O[(l, k)] = torch.zeros_like(dev[(l, k)][0])
+                lse[(l, k)] = torch.zeros(kv.batch, kv.n_heads, nk, dtype=torch.float32, device="cuda")
+        wps = []
+        for k in range(K_s):
+            wpos = self.window_fn(k)
+            do_compress = (k + 1 < K_s) or self.compress_last
+            wps.append((kv.window_array(wpos) if (do_compress and wpos is not None) else None, do_compress, wpos))
+        kv.scalekv_sync()
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=kv.stream_main):
+            kv.scalekv_reset()
+            for k in range(K_s):
+                wp, do_compress, _ = wps[k]
+                for l in range(n_layers):
+                    Qd, Kd, Vd = dev[(l, k)]
+                    kv.scalekv_step(l, k, Qd, Kd, Vd, O[(l, k)], window_pos=wp, whole_map=do_compress and wp is None,
+                                    lse=lse[(l, k)])
+            kv.scalekv_join()
+        for rep in range(2):
+            for t in O.values():
+                t.zero_()
+            torch.cuda.synchronize()
+            with torch.cuda.stream(kv.stream_main):
+                g.replay()
+            kv.scalekv_sync()
+        for k in range(K_s):
+            _, do_compress, wpos = wps[k]
+            for (l, b, h) in self.slices:
+                Q, K, V = (t[b, h].cpu() for t in host[(l, k)])
+                self._compare_slice((l, b, h), k, to64(Q), to64(K), to64(V), to64(O[(l, k)][b, h].cpu()),
+                                    to64(lse[(l, k)][b, h].cpu()), wpos, do_compress, exported=False)
+        for (l, b, h) in self.slices:
+            cache = self.caches[(l, b, h)]
+            pos, Kg, Vg = kv.scalekv_export_slice(l, b, h, with_kv=True)
+            # a layer whose last map reached into pages that a later layer took over exports the entries before that map
+            m = len(pos)
+            assert m == len(cache) or (not self.compress_last and m == len(cache) - self.n[-1])
+            assert np.array_equal(pos.numpy().astype(np.int64), cache.pos[:m]), f"slice {(l, b, h)}: positions after the replayed pass"
+            assert np.array_equal(to64(Kg), cache.K[:m]) and np.array_equal(to64(Vg), cache.V[:m]), f"slice {(l, b, h)}: rows after the replayed pass"
+        return self
+
+    def _compare_slice(self, key, k, Q, K, V, O_gpu, lse_gpu, wpos, do_compress, scores_fresh=True, exported=True):
         l, b, h = key
         kv = self.kv
         cache = self.caches[key]
@@ -85,8 +201,10 @@ class ParityRun:
         self.max_err = max(self.max_err, err)
         # bf16: two roundings to 8 significant bits (P, then O), each at most 2^-9 relative: beyond |O| = 2.56 the
         # bound that follows from the arithmetic, 2^-7 max|O|, is larger than the 2e-2 quoted for unit-scale outputs
-        tol = max(TOL[self.dtype], REL[self.dtype] * float(np.max(np.abs(O))))
-        self.max_tol = max(self.max_tol, tol)
+        rel = REL[self.dtype] * float(np.max(np.abs(O)))
+        tol = max(TOL[self.dtype], rel)
+        self.compared += 1
+        self.rel_bound_used += int(rel > TOL[self.dtype])
         assert err <= tol, f"slice {key} scale {k}: attention max-abs error {err} (bound {tol})"
         if self.check_lse:
             le = float(np.max(np.abs(lse - lse_gpu)))
@@ -102,6 +220,12 @@ class ParityRun:
         s = cache.scores(Q[w_list])
         keep = orc.select(s, cache.pos, cache.N[k], w_list, budget)
         want_pos = cache.pos[keep]
+        if not exported:
+            # nothing to read back at this point of a replayed pass: the oracle goes on with its own selection
+            cand = L - len(w_list)
+            self.evictions += int(budget != orc.KEEP_ALL and budget < cand)
+            cache.adopt_positions(want_pos)
+            return
         got_pos, Kg, Vg = kv.scalekv_export_slice(l, b, h, with_kv=True)
         got_pos = got_pos.numpy().astype(np.int64)
         cand = L - len(w_list)
@@ -129,10 +253,6 @@ class ParityRun:
         assert np.array_equal(to64(Kg), cache.K), f"slice {key} scale {k}: compacted K rows differ"
         assert np.array_equal(to64(Vg), cache.V), f"slice {key} scale {k}: compacted V rows differ"
         if kprime < cand:
-            sg = kv.scalekv_export_scores(b, h).numpy().astype(np.float64) if self._scores_fresh(l) else None
+            sg = kv.scalekv_export_scores(b, h).numpy().astype(np.float64) if scores_fresh else None
             if sg is not None and len(sg) == L:
                 assert np.all(np.abs(sg - s) <= 2e-4 * s + 1e-9), "importance scores differ"
-
-    def _scores_fresh(self, l):
-        # the score scratch belongs to the most recent evicting compress; valid when the run syncs per layer
-        return True

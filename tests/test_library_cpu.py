@@ -92,3 +92,14 @@ def test_product_path_refuses_to_run_without_gpu():
         pytest.skip("GPU present")
     with pytest.raises(RuntimeError):
         binding.ScaleKV(1, 1, 4, 64, "f32", (1, 2), (1, 2), [[-1, -1]])
+
+
+def test_budget_tokens_matches_oracle(lib):
+    """The fraction -> tokens rule behind the ABI against the oracle's exact-rational version, on the fractions the
+    workloads use (30 %, 3 %, 10 %, the 4 / 10 / 20 % sweep's drafter and refiner shares) and on .5 cases."""
+    for sides in (SIDES_13, SIDES_16, (1, 2, 4, 8)):
+        n = orc.scale_token_counts(sides)
+        for f in (0.30, 0.03, 0.10, 0.04, 0.20, 0.0123, 0.123, 0.01231, 0.03077, 0.3077, 0.06154, 0.6154, 1.0, 0.0, 0.5):
+            assert binding.scalekv_budget_tokens(f, sides) == orc.budget_tokens(f, n), (sides, f)
+    assert binding.scalekv_budget_tokens(0.30, SIDES_13) == 1928        # 1927.5 rounds up
+    assert binding.scalekv_budget_tokens(0.5, (1, 1, 1)) == 1 and binding.scalekv_budget_tokens(0.25, (1, 1, 1)) == 1

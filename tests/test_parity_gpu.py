@@ -262,20 +262,115 @@ def test_full_size_single_layer_sampled_slices():
     kv.close()
 
 
-def test_full_size_pass_sampled_slices():
-    """configs[2] at full size (32 layers, drafter / refiner budgets of 30 % / 3 %, planted roles): all
-    layers run on the GPU, the oracle follows one slice in each of two drafter and two refiner layers."""
+def sampled_slices(wl, planted, count):
+    """`count` slices spread over drafter and refiner layers (first, last and layers in between), first / last
+    batch element and head, and seeded ones in between."""
+    refiners = [l for l in range(wl.n_layers) if l not in planted]
+    layers = [planted[0], refiners[0], planted[-1], refiners[-1], 0, 1, wl.n_layers - 2, wl.n_layers - 1]
+    rng = np.random.default_rng(wl.seed)
+    out, corners = [], [(0, 0), (wl.batch - 1, wl.n_heads - 1), (0, wl.n_heads - 1), (wl.batch - 1, 0)]
+    i = 0
+    while len(out) < count:
+        l = layers[i % len(layers)] if i < 2 * len(layers) else int(rng.integers(wl.n_layers))
+        b, h = corners[i % 4] if i < 8 else (int(rng.integers(wl.batch)), int(rng.integers(wl.n_heads)))
+        if (l, b, h) not in out:
+            out.append((l, b, h))
+        i += 1
+    return out
+
+
+def test_full_size_pass_pipelined_16_slices():
+    """configs[2] at full size (32 layers, B 8, H 16, 13 scales, drafter / refiner budgets of 30 % / 3 %, planted
+    roles) in the execution mode the benchmark times: one scalekv_step per layer and scale, compress on the side
+    stream, no host synchronisation inside a scale-step.  The oracle follows 16 slices (drafter and refiner
+    layers, first and last batch element and head) through the whole pass, log-sum-exp included."""
     wl = synth.WORKLOADS["pass2b"]
     n = wl.n_tokens
     planted = synth.drafter_layers(wl)
     bd, br = orc.budget_tokens(0.30, n), orc.budget_tokens(0.03, n)
     budgets = [[bd if l in planted else br] * wl.n_scales for l in range(wl.n_layers)]
     kv = binding.ScaleKV(wl.n_layers, wl.batch, wl.n_heads, 128, "bf16", wl.sides, wl.sides, budgets, max_window=16)
-    refiners = [l for l in range(wl.n_layers) if l not in planted]
-    slices = [(planted[0], 0, 0), (planted[-1], 7, 15), (refiners[0], 2, 5), (refiners[-1], 5, 9)]
+    slices = sampled_slices(wl, planted, 16)
+    assert {s[0] for s in slices} & set(planted) and {s[0] for s in slices} - set(planted)
     run = ParityRun(kv, "bf16", wl.sides, budgets, lambda l, k: synth.scale_inputs(wl, l, k, device="cuda"),
-                    lambda k: orc.window_centroids(wl.sides[k], wl.sides[k], 16), slices, check_lse=False).run()
+                    lambda k: orc.window_centroids(wl.sides[k], wl.sides[k], 16), slices, check_lse=True).run_pipelined("eager")
+    print("config 3, pipelined:", run.summary())
+    assert run.evictions > 0 and run.compared == 16 * wl.n_scales
+    kv.close()
+
+
+def test_8b_class_full_40_layers_pipelined_8_slices():
+    """configs[3] with all 40 layers and 32 heads (the page plan the benchmark runs) at the 10 / 30 drafter /
+    refiner split, pipelined like the benchmark; the oracle follows 8 slices, attention on 1 024 evenly spaced
+    rows of the large maps."""
+    wl = synth.WORKLOADS["pass8b"]
+    n = wl.n_tokens
+    planted = synth.drafter_layers(wl)
+    bd, br = orc.budget_tokens(0.30, n), orc.budget_tokens(0.03, n)
+    budgets = [[bd if l in planted else br] * wl.n_scales for l in range(wl.n_layers)]
+    kv = binding.ScaleKV(wl.n_layers, wl.batch, wl.n_heads, 128, "bf16", wl.sides, wl.sides, budgets, max_window=16)
+    slices = sampled_slices(wl, planted, 8)
+    run = ParityRun(kv, "bf16", wl.sides, budgets, lambda l, k: synth.scale_inputs(wl, l, k, device="cuda"),
+                    lambda k: orc.window_centroids(wl.sides[k], wl.sides[k], 16), slices, check_lse=True,
+                    max_rows=1024).run_pipelined("eager")
+    print("config 4, pipelined:", run.summary())
     assert run.evictions > 0
+    kv.close()
+
+
+def test_hires_full_32_layers_pipelined_8_slices():
+    """configs[4] with all 32 layers (16 scales up to 128 x 128) at the 10 % point of the sweep, pipelined like
+    the benchmark; the oracle follows 8 slices, attention on 512 evenly spaced rows of the large maps."""
+    wl = synth.WORKLOADS["hires"]
+    n = wl.n_tokens
+    refiner_pct = 0.10 / 3.25
+    bd, br = orc.budget_tokens(round(10 * refiner_pct, 6), n), orc.budget_tokens(round(refiner_pct, 6), n)
+    planted = synth.drafter_layers(wl)
+    budgets = [[bd if l in planted else br] * wl.n_scales for l in range(wl.n_layers)]
+    kv = binding.ScaleKV(wl.n_layers, wl.batch, wl.n_heads, 128, "bf16", wl.sides, wl.sides, budgets, max_window=16)
+    slices = sampled_slices(wl, planted, 8)
+    run = ParityRun(kv, "bf16", wl.sides, budgets, lambda l, k: synth.scale_inputs(wl, l, k, device="cuda"),
+                    lambda k: orc.window_centroids(wl.sides[k], wl.sides[k], 16), slices, check_lse=True,
+                    max_rows=512).run_pipelined("eager")
+    print("config 5, pipelined:", run.summary())
+    assert run.evictions > 0
+    kv.close()
+
+
+def _ragged_five_layer_case():
+    """Five layers with budgets from 0 to KEEP_ALL-like, odd map sizes, small pages: persistent and transient pages,
+    evicting and non-evicting compressions, drafter- and refiner-like inputs all occur."""
+    sides = (1, 2, 3, 5, 9, 14, 19, 23)
+    budgets = [[150] * len(sides), [21] * len(sides), [60] * len(sides), [0] * len(sides), [400] * len(sides)]
+    wl = synth.Workload("p", 5, 2, 2, 128, "bf16", sides, seed=37, n_drafters=2)
+    return sides, budgets, wl
+
+
+@pytest.mark.parametrize("mode", ["eager", "graph"])
+@pytest.mark.parametrize("page_tokens", [0, 32])
+def test_pipelined_scale_steps_match_oracle(mode, page_tokens):
+    """The benchmark's execution mode against the oracle on a small ragged case, every slice followed: compress
+    of layer l runs on the side stream under attend of layer l + 1, layers l and l + 2 share a transient page
+    set and a logit buffer, and the host only synchronises between scale-steps - eager, and with every
+    scale-step replayed from a CUDA graph."""
+    sides, budgets, wl = _ragged_five_layer_case()
+    kv = binding.ScaleKV(5, 2, 2, 128, "bf16", sides, sides, budgets, max_window=16, page_tokens=page_tokens)
+    run = ParityRun(kv, "bf16", sides, budgets, lambda l, k: synth.scale_inputs(wl, l, k),
+                    lambda k: orc.window_centroids(sides[k], sides[k], 16), all_slices(5, 2, 2)).run_pipelined(mode)
+    print("pipelined", mode, run.summary())
+    assert run.evictions >= 40 and run.resyncs == 0
+    kv.close()
+
+
+def test_whole_pass_graph_replay_matches_oracle():
+    """What the benchmark's timed region does - one CUDA graph of the whole pass, replayed - against the oracle:
+    every layer's output of every scale and the store every slice is left with."""
+    sides, budgets, wl = _ragged_five_layer_case()
+    kv = binding.ScaleKV(5, 2, 2, 128, "bf16", sides, sides, budgets, max_window=16)
+    run = ParityRun(kv, "bf16", sides, budgets, lambda l, k: synth.scale_inputs(wl, l, k),
+                    lambda k: orc.window_centroids(sides[k], sides[k], 16), all_slices(5, 2, 2)).run_graph_pass()
+    print("whole-pass graph:", run.summary())
+    assert run.evictions >= 40 and run.compared == 20 * len(sides)
     kv.close()
 
 
@@ -736,7 +831,6 @@ def run_random_configuration(seed, max_side=20):
     slices = [(l, b, h) for l in range(n_layers) for b in range(B) for h in range(H)]
     run = ParityRun(kv, dtype, sides_h, budgets, inputs, lambda k: orc.window_centroids(sides_h[k], sides_w[k], patches),
                     slices, compress_last=bool(rng.random() < 0.5), sides_w=sides_w).run()
-    assert run.max_err <= run.max_tol
     kv.close()
     return run
 
@@ -847,5 +941,147 @@ def test_dominant_keys_anywhere_in_the_first_tiles(amp):
 
     run = ParityRun(kv, "bf16", sides, budgets, inputs, lambda k: orc.window_centroids(sides[k], sides[k], 16),
                     [(0, 0, 0), (0, 0, 1)], check_lse=True).run()
-    assert run.max_err <= run.max_tol
+    kv.close()
+
+
+def test_exact_ties_on_the_tensor_core_path():
+    """bf16 x 128 with Q = 0: the window logits come out of the tensor core and the recorded-logits score
+    kernel, every importance is bit-equal, so the kept candidates must be exactly the lowest positions (the
+    oracle's rule), with no tie-band allowance used."""
+    sides = (2, 5, 9, 14, 18)
+    n = orc.scale_token_counts(sides)
+    budgets = [[7] * len(sides), [130] * len(sides)]
+    g = torch.Generator().manual_seed(91)
+
+    def inputs(l, k):
+        Kt = torch.randn(1, 2, n[k], 128, generator=g).to(torch.bfloat16)
+        V = torch.randn(1, 2, n[k], 128, generator=g).to(torch.bfloat16)
+        return torch.zeros(1, 2, n[k], 128, dtype=torch.bfloat16), Kt, V
+
+    for mode in ("synced", "pipelined"):
+        kv = binding.ScaleKV(2, 1, 2, 128, "bf16", sides, sides, budgets, max_window=16)
+        run = ParityRun(kv, "bf16", sides, budgets, inputs, lambda k: orc.window_centroids(sides[k], sides[k], 16),
+                        all_slices(2, 1, 2), compress_last=True)
+        run = run.run() if mode == "synced" else run.run_pipelined("eager")
+        assert run.evictions >= 6 and run.resyncs == 0
+        # layer 0 after the last compress: the 7 lowest positions that never were window entries, and the window
+        pos = kv.scalekv_export_slice(0, 0, 1).tolist()
+        assert len(pos) == 7 + 16 and pos[:4] == [0, 1, 2, 3]
+        kv.close()
+
+
+def test_bounded_wait_gives_up_and_reports_timeout():
+    """The failure path of every device-side wait: a wait on a barrier that nothing arrives at runs out after its
+    limit (50 ms here instead of 2 s), the kernel returns, the CTA's other warps see the abort flag, and
+    scalekv_sync reports SCALEKV_ERR_TIMEOUT.  The context stays usable for host calls and the device for
+    other contexts."""
+    import time
+
+    sides = (1, 2, 4)
+    kv = binding.ScaleKV(1, 1, 2, 128, "bf16", sides, sides, [[4] * 3], max_window=16)
+    kv.scalekv_sync()                                   # status clean
+    t0 = time.perf_counter()
+    gave_up, seen = kv.scalekv_selftest_wait(50)
+    dt = time.perf_counter() - t0
+    assert gave_up == 1 and seen == 1
+    assert 0.04 <= dt < 1.5, dt                         # it waited for the limit, and not much longer
+    with pytest.raises(binding.ScaleKVError) as e:
+        kv.scalekv_sync()
+    assert e.value.status == 6                          # TIMEOUT, sticky
+    # an attend launched now returns at once (its CTAs see the status) instead of computing on a failed context
+    x = torch.randn(1, 2, 1, 128, device="cuda").to(torch.bfloat16)
+    O = torch.full_like(x, 7.0)
+    torch.cuda.synchronize()
+    kv.scalekv_append(0, 0, x, x)
+    kv.scalekv_attend(0, x, O)
+    with pytest.raises(binding.ScaleKVError) as e:
+        kv.scalekv_sync()
+    assert e.value.status == 6
+    assert torch.all(O == 7.0)
+    kv.close()
+    # a fresh context on the same device works
+    kv = binding.ScaleKV(1, 1, 2, 128, "bf16", sides, sides, [[4] * 3], max_window=16)
+    kv.scalekv_append(0, 0, x, x)
+    kv.scalekv_attend(0, x, O)
+    kv.scalekv_sync()
+    assert torch.allclose(O.float(), x.float(), atol=1e-2)     # one key: O = V
+    kv.close()
+
+
+def test_append_refuses_to_overwrite_a_layer_that_shares_its_transient_pages():
+    """Layers of equal parity share a transient page set and a logit buffer.  An order of calls that would
+    overwrite another layer's uncompressed map (append / attend of layers 0, 1, 2 before any compress; or layer 0
+    then layer 4) is refused with BAD_STATE and nothing is touched; after the compress it goes through, and the
+    kept rows are the oracle's."""
+    sides = (4, 12, 20)
+    n = orc.scale_token_counts(sides)
+    budgets = [[10] * 3] * 5                            # small persistent capacity: maps reach the transient pages
+    kv = binding.ScaleKV(5, 1, 2, 128, "bf16", sides, sides, budgets, max_window=16)
+    g = torch.Generator().manual_seed(3)
+    data = {(l, k): tuple(torch.randn(1, 2, n[k], 128, generator=g).to(torch.bfloat16) for _ in range(3))
+            for l in range(5) for k in range(3)}
+    dev = {key: tuple(t.cuda() for t in v) for key, v in data.items()}
+    torch.cuda.synchronize()
+    wpos = [orc.window_centroids(a, a, 16) for a in sides]
+    for l in range(5):                                  # scale 0: the whole map is the window, nothing evicted
+        Q, K, V = dev[(l, 0)]
+        kv.scalekv_step(l, 0, Q, K, V, torch.empty_like(Q), window_pos=wpos[0])
+    for l in (0, 1):
+        Q, K, V = dev[(l, 1)]
+        kv.scalekv_append(l, 1, K, V)
+        kv.scalekv_attend(l, Q)
+    for other in (2, 4):
+        with pytest.raises(binding.ScaleKVError) as e:
+            kv.scalekv_append(other, 1, dev[(other, 1)][1], dev[(other, 1)][2])
+        assert e.value.status == 2 and "layer 0" in str(e.value)
+    kv.scalekv_compress(0, dev[(0, 1)][0], wpos[1], qw_is_full_map=True)
+    Q, K, V = dev[(2, 1)]
+    kv.scalekv_append(2, 1, K, V)                       # layer 0 is through: accepted
+    kv.scalekv_attend(2, Q)
+    kv.scalekv_compress(1, dev[(1, 1)][0], wpos[1], qw_is_full_map=True)
+    kv.scalekv_compress(2, Q, wpos[1], qw_is_full_map=True)
+    kv.scalekv_sync()
+    for l in (0, 1, 2):
+        for h in range(2):
+            c = orc.SliceCache(n, 128)
+            for k in range(2):
+                Qh, Kh, Vh = (t[0, h].double().numpy() for t in data[(l, k)])
+                c.append(Kh, Vh)
+                c.compress(Qh[wpos[k]], wpos[k], 10)
+            pos, Kg, Vg = kv.scalekv_export_slice(l, 0, h, with_kv=True)
+            assert np.array_equal(pos.numpy(), c.pos)
+            assert np.array_equal(Kg.double().numpy(), c.K) and np.array_equal(Vg.double().numpy(), c.V)
+    kv.close()
+
+
+def test_sinks_beyond_the_planned_capacity_are_refused():
+    sides = (4, 12, 20)
+    kv = binding.ScaleKV(1, 1, 2, 128, "bf16", sides, sides, [[10] * 3], max_window=16)
+    x = {k: torch.randn(1, 2, a * a, 128, device="cuda").to(torch.bfloat16) for k, a in enumerate(sides)}
+    torch.cuda.synchronize()
+    kv.scalekv_append(0, 0, x[0], x[0])
+    kv.scalekv_attend(0, x[0])
+    kv.scalekv_compress_ex(0, policy="recent", n_sink=4)
+    kv.scalekv_append(0, 1, x[1], x[1])
+    kv.scalekv_attend(0, x[1])
+    with pytest.raises(binding.ScaleKVError) as e:
+        kv.scalekv_compress_ex(0, policy="recent", n_sink=150)      # 150 sinks, pages planned for 10 + 16 entries
+    assert e.value.status == 3
+    kv.scalekv_compress_ex(0, policy="recent", n_sink=4)
+    kv.scalekv_sync()
+    assert kv.scalekv_lengths(0) == [[10, 10]]
+    kv.close()
+
+
+def test_compress_as_three_launches_matches_oracle():
+    """The one-launch compress is what every other test runs; here the same ragged case goes through the three
+    separate kernels (importance; selection; pruning over 8 CTAs per slice), the path that slices too long for
+    one CTA's shared memory take."""
+    sides, budgets, wl = _ragged_five_layer_case()
+    kv = binding.ScaleKV(5, 2, 2, 128, "bf16", sides, sides, budgets, max_window=16)
+    run = ParityRun(kv, "bf16", sides, budgets, lambda l, k: synth.scale_inputs(wl, l, k),
+                    lambda k: orc.window_centroids(sides[k], sides[k], 16), all_slices(5, 2, 2), compress_last=True)
+    run.separate_kernels = True
+    run.run()
+    assert run.evictions >= 40 and run.resyncs == 0
     kv.close()

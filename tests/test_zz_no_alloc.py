@@ -8,6 +8,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import scalekv_oracle as orc
 from paper_2505_19602_b200 import binding
 
 pytestmark = pytest.mark.gpu
@@ -91,3 +92,20 @@ def test_static_select_ties_and_limits():
     torch.cuda.synchronize()
     want = torch.sort(torch.topk(full, 3, dim=1).indices, dim=1).values
     assert torch.equal(out.cpu().long(), want.cpu())
+
+
+def test_static_select_matches_the_oracle_selection():
+    """The same rows through the CPU oracle's selection rule (largest scores, equal scores by lowest index):
+    random rows, rows with many repeated values, and a row whose values are all equal."""
+    g = torch.Generator().manual_seed(7)
+    rows = torch.rand(6, 777, generator=g)
+    rows[1] = torch.round(rows[1] * 8) / 8              # heavy ties
+    rows[2] = 0.125
+    rows[3, 100:300] = rows[3, 5]
+    dev = rows.cuda()
+    for k in (1, 13, 400, 777):
+        for rep in range(2):
+            out = binding.scalekv_select_static(dev, k).cpu().numpy()
+            for r in range(rows.shape[0]):
+                want = orc.select(rows[r].double().numpy(), np.arange(777), 777, [], k)
+                assert np.array_equal(out[r], want), (k, r, rep)
