@@ -49,6 +49,12 @@ def parse_args():
     ap.add_argument("--overall-pct", type=float, default=0.0,
                     help="overall budget in per cent of the cached tokens (the 4 / 10 / 20 sweep of the 16-scale workload): "
                          "refiner budget = overall / 3.25, drafter budget = 10 x refiner; default: 30 %% / 3 %%")
+    ap.add_argument("--delta", type=float, default=None,
+                    help="budget table from Eq. 4 with the paper's constants (650 tokens per head and layer on average, "
+                         "B_r(0) = 600) and this refiner decay rate (Sec. 4.3 sweeps 0 .. 70) instead of 30 %% / 3 %%")
+    ap.add_argument("--policy", default="scalekv", choices=["scalekv", "sliding", "sinks", "snapkv", "pyramid"],
+                    help="keep-rule timed on the same store at equal total budget: the paper's (default) or one of the "
+                         "comparison policies of Sec. 4.1 (see include/scalekv.h, scalekv_policy_budgets)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-side-stream", action="store_true")
@@ -283,6 +289,8 @@ def run_scalekv(args):
             budgets = pipeline.budget_table(wl, roles, drafter_frac=10 * r1000 / 100000, refiner_frac=r1000 / 100000)
         else:
             budgets = pipeline.budget_table(wl, roles)
+        if args.delta is not None:
+            budgets = [[int(x) for x in row] for row in binding.scalekv_make_budgets(roles, 650, 600, args.delta)]
         planted = synth.drafter_layers(wl)
         # Eq. 2 cannot tell the roles apart while the history is shorter than K' (then the top-K' mass is all of the
         # history mass and ASI = c (1 - c) is symmetric): count the recovery over the scales with a longer history
@@ -291,20 +299,41 @@ def run_scalekv(args):
         hits = sum(int(roles[l][k]) for k in ks for l in planted)
         role_note = (f"{wl.n_drafters} drafters per scale from scalekv_layer_stats; {hits}/{len(planted) * len(ks)} planted "
                      f"drafters recovered at the {len(ks)} scales whose history exceeds 4 K'")
+        if args.delta is not None:
+            role_note += f"; Eq. 4 table: 650 average, B_r(0) = 600, delta = {args.delta:g}"
+
     else:
         b = binding.scalekv_budget_tokens(0.10, wl.sides)
         budgets = [[b] * wl.n_scales for _ in range(wl.n_layers)]
         role_note = "uniform 10%"
     calib_s = time.perf_counter() - t0
+    # the comparison policies run at the total budget of the table above: its mean over layers, window included
+    select, window_kind = None, "centroids"
+    if args.policy != "scalekv":
+        args.no_e2e = args.no_cpu_baseline = True      # those legs run the paper's rule; an A/B line is kernel timing only
+        w_obs = min(wl.window, binding.MAX_WINDOW)
+        k_ref = wl.n_scales - 2
+        mean_cache = sum(min(budgets[l][k_ref], 10 ** 9) + w_obs for l in range(wl.n_layers)) / wl.n_layers
+        if args.policy in ("sliding", "sinks"):
+            table = binding.scalekv_policy_budgets("uniform", wl.n_layers, wl.n_scales, mean_cache)
+            select = {"policy": "recent", "n_sink": 4 if args.policy == "sinks" else 0}
+        else:
+            table = binding.scalekv_policy_budgets("uniform" if args.policy == "snapkv" else "pyramid", wl.n_layers, wl.n_scales,
+                                                   mean_cache - w_obs, 20.0)
+            select = {"policy": "score", "pool_kernel": 7}
+            window_kind = "last"
+            windows = [binding.scalekv_window_last(a, a, w_obs) for a in wl.sides]
+        budgets = [[int(x) for x in row] for row in table]
+        role_note = f"policy {args.policy} at {mean_cache:.1f} cached tokens per head and layer on average"
 
     def make_kv():
         return binding.ScaleKV(wl.n_layers, wl.batch, wl.n_heads, wl.head_dim, wl.dtype, wl.sides, wl.sides, budgets,
                                max_window=min(wl.window, binding.MAX_WINDOW), device=local_rank,
-                               side_stream=not args.no_side_stream)
+                               side_stream=not args.no_side_stream, window_kind=window_kind)
 
     kv = make_kv()
     inputs = pipeline.PassInputs(wl, device=local_rank)
-    work = pipeline.pass_work(wl, budgets, windows)
+    work = pipeline.pass_work(wl, budgets, windows, recent=select is not None and select["policy"] == "recent")
     torch.cuda.synchronize()
 
     def barrier():
@@ -325,7 +354,7 @@ def run_scalekv(args):
                 if graph is not None:
                     graph.replay()
             if graph is None:
-                pipeline.run_pass(kv, inputs, windows)
+                pipeline.run_pass(kv, inputs, windows, select=select)
         kv.scalekv_join()
         with torch.cuda.stream(kv.stream_main):
             marks[n_pass].record()
@@ -334,7 +363,7 @@ def run_scalekv(args):
         return marks[0].elapsed_time(marks[n_pass])
 
     for _ in range(args.warmup):
-        pipeline.run_pass(kv, inputs, windows)
+        pipeline.run_pass(kv, inputs, windows, select=select)
     kv.scalekv_sync()
     # A pass is the same sequence of launches every time (the schedule, the budgets and the buffers are
     # fixed), so it is captured once into a CUDA graph - stream_main plus the side stream that compress
@@ -347,7 +376,7 @@ def run_scalekv(args):
             torch.cuda.synchronize()
             # thread_local: other threads (a process group's watchdog under torchrun) may call CUDA meanwhile
             with torch.cuda.graph(graph, stream=kv.stream_main, capture_error_mode="thread_local"):
-                pipeline.run_pass(kv, inputs, windows)
+                pipeline.run_pass(kv, inputs, windows, select=select)
                 kv.scalekv_join()
             with torch.cuda.stream(kv.stream_main):
                 graph.replay()                         # one untimed replay
@@ -358,7 +387,7 @@ def run_scalekv(args):
             torch.cuda.synchronize()
             kv.close()
             kv = make_kv()
-            pipeline.run_pass(kv, inputs, windows)
+            pipeline.run_pass(kv, inputs, windows, select=select)
             kv.scalekv_sync()
             launches0 = kv.scalekv_launch_count()
     launches_per_pass = kv.scalekv_launch_count() - launches0
@@ -387,7 +416,7 @@ def run_scalekv(args):
     per_pass = []
     for _ in range(args.steps):
         marks = []
-        pipeline.run_pass(kv, inputs, windows, marks=marks)
+        pipeline.run_pass(kv, inputs, windows, marks=marks, select=select)
         kv.scalekv_sync()
         per_pass.append([marks[i].elapsed_time(marks[i + 1]) for i in range(len(marks) - 1)])
     cols = list(zip(*per_pass))
@@ -403,7 +432,7 @@ def run_scalekv(args):
     # the same passes once more with compress serialised onto stream_main: every kernel timed alone
     kv.scalekv_profile_enable(2)
     for _ in range(args.steps):
-        pipeline.run_pass(kv, inputs, windows)
+        pipeline.run_pass(kv, inputs, windows, select=select)
     prof_alone = kv.scalekv_profile_read()
     kv.scalekv_profile_enable(0)
     att_ms, att_n = prof_timed["attend"]
@@ -494,6 +523,7 @@ def run_scalekv(args):
             "config": {"workload": wl.name, "layers": wl.n_layers, "batch": wl.batch, "heads": wl.n_heads,
                        "head_dim": wl.head_dim, "scales": wl.n_scales, "tokens": sum(wl.n_tokens),
                        "budget": role_note + (f"; overall {args.overall_pct} %" if args.overall_pct > 0 else ""),
+                       "policy": args.policy,
                        "window": wl.window, "parallelism": f"replica x{world} (batch-sharded, no collective)",
                        "l2_policy": f"inputs larger than L2: {inputs.bytes() / 1e9:.1f} GB of Q/K/V per pass",
                        "side_stream": not args.no_side_stream, "cuda_graph": graph_note, "calibration_s": round(calib_s, 1),

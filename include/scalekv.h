@@ -77,7 +77,12 @@ typedef struct {
                                  /* map (scalekv_window_centroids) while it computes them anyway, and a */
                                  /* scalekv_compress called with exactly that window scores the cache   */
                                  /* from them instead of reading K again.  Any other window still works.*/
+  int32_t window_kind;           /* which rows window_patches = N stands for: SCALEKV_WINDOW_CENTROIDS (0, the   */
+                                 /* paper's patch centroids) or SCALEKV_WINDOW_LAST (the last N rows of the map */
+                                 /* in raster order, scalekv_window_last - the SnapKV-like comparison rule)     */
 } scalekv_config;
+#define SCALEKV_WINDOW_CENTROIDS 0
+#define SCALEKV_WINDOW_LAST 1
 
 /* A [batch][n_heads][tokens][head_dim] tensor view: device pointer + ELEMENT strides; the
  * innermost (head_dim) axis is contiguous and every row must start on a 16-byte boundary. */
@@ -258,6 +263,25 @@ scalekv_status scalekv_assign_roles(const double *asi, int32_t L, int32_t K, int
  * everywhere; values rounded half up.  budgets_out HOST [L][K].  Host only. */
 scalekv_status scalekv_make_budgets(const uint8_t *is_drafter, int32_t L, int32_t K, double b_uniform, double b_r0,
                                     double delta, int32_t *budgets_out);
+
+/* Sec. 4.1 "Compression Baselines": the comparison policies as configurations of this store (their image
+ * quality is outside this library; they run on the same cache for A/B timing):
+ *   sliding window        SCALEKV_SELECT_RECENT, n_sink = 0, a uniform table
+ *   sinks + recent tokens SCALEKV_SELECT_RECENT, n_sink > 0, a uniform table
+ *   SnapKV-like           SCALEKV_SELECT_SCORE observed by the LAST rows of the map (scalekv_window_last,
+ *                         window_kind = SCALEKV_WINDOW_LAST), importance pooled along the keys (pool_kernel, e.g.
+ *                         7), a uniform table
+ *   pyramid budgets       the SnapKV-like rule with a table that falls linearly with the layer index.
+ * scalekv_window_last: the last min(n_obs, h * w) raster indices of an h x w map, ascending -> pos (HOST, room
+ * for n_obs entries), *count their number.
+ * scalekv_policy_budgets: budgets_out HOST [L][K], every scale alike.  SCALEKV_BUDGETS_UNIFORM: b_mean rounded
+ * half up everywhere.  SCALEKV_BUDGETS_PYRAMID: layer l gets b_max - (b_max - b_min) l / (L - 1) rounded half
+ * up, with b_min = b_mean / beta (beta >= 1) and b_max = 2 b_mean - b_min, so the mean over layers is b_mean;
+ * a single layer gets b_mean.  Host only. */
+#define SCALEKV_BUDGETS_UNIFORM 0
+#define SCALEKV_BUDGETS_PYRAMID 1
+scalekv_status scalekv_window_last(int32_t h, int32_t w, int32_t n_obs, int32_t *pos, int32_t *count);
+scalekv_status scalekv_policy_budgets(int32_t shape, int32_t L, int32_t K, double b_mean, double beta, int32_t *budgets_out);
 
 /* Sec. 4.1 / Sec. 4.3: a budget quoted as a fraction of "the original KV cache size" is that fraction of
  * T_c = N_{K-1}, the tokens that ever need caching (the last map is never read by a later step - Table 1's

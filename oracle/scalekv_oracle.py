@@ -24,7 +24,8 @@ accounting helpers by the values printed in Table 1, Table 3 and Sec. 4.3; layer
 its invariants and the uniform-attention closed form; make_budgets by Eq. 4 itself.
 window_centroids (patch geometry) and assign_roles tie order are readings with no printed
 value to check against: parity unpinned for those two choices (their invariants are
-tested).
+tested).  window_last and policy_budgets (the comparison policies as configurations of this
+store) are pinned by their closed forms: the arithmetic series' sum, monotonicity, endpoints.
 """
 from __future__ import annotations
 
@@ -402,3 +403,42 @@ def make_budgets(is_drafter, b_uniform, b_r0, delta):
         out[is_drafter[:, k], k] = int(math.floor(bd + 0.5))
         out[~is_drafter[:, k], k] = int(math.floor(br + 0.5))
     return out
+
+
+# --------------------------------------------------------------------------------------
+# The comparison policies of Sec. 4.1 ("Compression Baselines") stated as configurations of the same
+# store: which rows observe, how the importance is smoothed, how the budget is spread over layers.
+# Their image quality is not in scope; these are keep-rules that run on the same cache for timing.
+# --------------------------------------------------------------------------------------
+def window_last(h, w, n_obs=16):
+    """Observation window of the SnapKV-like rule: the last n_obs tokens of the h x w map in raster
+    order (that method observes with the end of its input); a map with at most n_obs tokens is its
+    own window.  Ascending raster indices."""
+    n = int(h) * int(w)
+    m = min(int(n_obs), n)
+    return list(range(n - m, n))
+
+
+def policy_budgets(policy, n_layers, n_scales, b_mean, beta=20.0):
+    """Budget table [L][K] of a comparison policy with the same mean per layer as `b_mean`.
+
+    "uniform": every layer and scale gets b_mean (sliding window, sinks + recent, SnapKV-like).
+    "pyramid": budgets fall linearly with the layer index from b_max at the first layer to
+    b_min = b_mean / beta at the last one, b_max = 2 b_mean - b_min, so that the mean over layers is
+    b_mean (the pyramid-shaped allocation of PyramidKV); the same row for every scale; one layer
+    gets b_mean.  Values are rounded half up.
+    Returns int64 [L][K]."""
+    L, K = int(n_layers), int(n_scales)
+    out = np.zeros((L, K), dtype=np.int64)
+    if policy == "uniform" or L == 1:
+        out[:, :] = int(math.floor(float(b_mean) + 0.5))
+        return out
+    if policy != "pyramid":
+        raise ValueError(policy)
+    b_min = float(b_mean) / float(beta)
+    b_max = 2.0 * float(b_mean) - b_min
+    for l in range(L):
+        b = b_max - (b_max - b_min) * l / (L - 1)
+        out[l, :] = int(math.floor(b + 0.5))
+    return out
+

@@ -40,6 +40,7 @@ class scalekv_config(C.Structure):
         ("pool", C.c_void_p), ("pool_bytes", C.c_size_t),
         ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
         ("stream_main", C.c_void_p), ("stream_side", C.c_void_p), ("device", C.c_int32), ("window_patches", C.c_int32),
+        ("window_kind", C.c_int32),
     ]
 
 
@@ -107,6 +108,8 @@ def load_library():
         "scalekv_sync": [ctx_p],
         "scalekv_join": [ctx_p],
         "scalekv_budget_tokens": [f64, P(i32), P(i32), i32, P(i32)],
+        "scalekv_window_last": [i32, i32, i32, P(i32), P(i32)],
+        "scalekv_policy_budgets": [i32, i32, i32, f64, f64, P(i32)],
         "scalekv_selftest_wait": [ctx_p, i32, P(i32), P(i32)],
         "scalekv_launch_count": [ctx_p, P(i64)],
         "scalekv_profile_enable": [ctx_p, i32],
@@ -181,6 +184,29 @@ def scalekv_make_budgets(is_drafter, b_uniform, b_r0, delta):
     return out
 
 
+def scalekv_window_last(h, w, n_obs=16):
+    lib = load_library()
+    pos = (C.c_int32 * max(n_obs, 1))()
+    cnt = C.c_int32(0)
+    st = lib.scalekv_window_last(h, w, n_obs, pos, C.byref(cnt))
+    if st:
+        raise ScaleKVError(st)
+    return [pos[i] for i in range(cnt.value)]
+
+
+def scalekv_policy_budgets(shape, n_layers, n_scales, b_mean, beta=20.0):
+    """Budget table [L][K] of a comparison policy: shape "uniform" or "pyramid" (see include/scalekv.h)."""
+    import numpy as np
+
+    lib = load_library()
+    out = np.zeros((n_layers, n_scales), dtype=np.int32)
+    st = lib.scalekv_policy_budgets({"uniform": 0, "pyramid": 1}[shape], n_layers, n_scales, float(b_mean), float(beta),
+                                    out.ctypes.data_as(C.POINTER(C.c_int32)))
+    if st:
+        raise ScaleKVError(st)
+    return out
+
+
 def scalekv_budget_tokens(fraction, sides_h, sides_w=None):
     """Tokens that a budget quoted as a fraction of the cached tokens T_c = N_{K-1} stands for (rounded half up)."""
     lib = load_library()
@@ -214,7 +240,7 @@ class ScaleKV:
     """Owns the device pool / workspace (torch tensors) and one library context."""
 
     def __init__(self, n_layers, batch, n_heads, head_dim, dtype, sides_h, sides_w, budgets, max_window=16,
-                 softmax_scale=0.0, page_tokens=0, device=0, side_stream=True, window_patches=16):
+                 softmax_scale=0.0, page_tokens=0, device=0, side_stream=True, window_patches=16, window_kind="centroids"):
         if not torch.cuda.is_available():
             raise RuntimeError("ScaleKV needs a CUDA device (sm_100a); there is no CPU path")
         self.lib = load_library()
@@ -234,6 +260,7 @@ class ScaleKV:
         cfg.scale_h, cfg.scale_w, cfg.budgets = self._h, self._w, self._b
         cfg.max_window, cfg.softmax_scale, cfg.page_tokens, cfg.device = max_window, softmax_scale, page_tokens, device
         cfg.window_patches = window_patches if window_patches <= max_window else 0
+        cfg.window_kind = {"centroids": 0, "last": 1}[window_kind]
         pb, wb = C.c_size_t(0), C.c_size_t(0)
         st = self.lib.scalekv_query_sizes(C.byref(cfg), C.byref(pb), C.byref(wb))
         if st:

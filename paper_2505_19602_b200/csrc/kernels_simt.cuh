@@ -862,93 +862,157 @@ __global__ void __launch_bounds__(1024) compress_fused_kernel(LayerView lv, Wind
 }
 
 // ------------------------------------------------------------------------------------------
-// layer statistics (Eq. 2): one block per (sampled query row, slice).  The softmax row is held
-// in shared memory; c = mass on the current map, t = sum of the K' largest history weights.
-// grid (n_rows, n_slices), 256 threads, dynamic smem = (L + D) floats.
+// layer statistics (Eq. 2): for sampled query rows i of the current map, alpha_i = softmax row over all L
+// entries, c_i = mass on the current map, t_i = sum of the K' largest alpha_ij over the history.
+// A CTA of 256 threads owns 64 sampled rows of one slice and streams the slice's keys in tiles of 64, so a
+// key tile is read once for 64 rows.  Per tile: logits by fp32 FMA (thread (ty, tx) owns rows ty + 16 i,
+// columns tx + 16 j), staged in shared memory; then four threads per row, 16 columns each, fold the tile into
+// the row's running maximum, normaliser and current-map mass (online softmax statistics) and into their own
+// descending list of the K' largest history logits seen in their columns (the K' largest weights are the K'
+// largest logits).  Nothing of length L is kept.  At the end one thread per row merges the four lists (K'
+// steps of a four-way merge) and the block adds its rows' c_i and t_i to the accumulators.
+// grid (ceil(n_rows / 64), n_slices); dynamic shared memory: layer_stats_smem_bytes<D>(K').
 // ------------------------------------------------------------------------------------------
+template <int D> __host__ __device__ constexpr size_t layer_stats_smem_bytes(int topk) {
+  return (size_t)(2 * 64 * (D + 4) + 64 * 65 + 64 + 256 * (topk > 0 ? topk : 1)) * 4;
+}
+
 template <typename T, int D>
-__global__ void __launch_bounds__(256) layer_stats_kernel(LayerView lv, TensorView Q, int n_k, int n_prev, int stride,
+__global__ void __launch_bounds__(256) layer_stats_kernel(LayerView lv, TensorView Q, int n_k, int n_prev, int stride, int n_rows,
                                                           int topk_prime, float scale, double *acc) {
-  extern __shared__ float smem[];
-  __shared__ float red[8];
-  __shared__ float best_v[8];
-  __shared__ int best_i[8];
-  float *qs = smem;          // [D]
-  float *p = smem + D;       // [L]
-  constexpr int VN = Vec16<T>::N;
+  constexpr int LD = D + 4, LDS = 65;
   constexpr int CH = D * (int)sizeof(T) / 16;
+  constexpr int VN = Vec16<T>::N;
+  extern __shared__ float smem[];
+  float *Qs = smem;                    // [64][LD]
+  float *Ks = Qs + 64 * LD;            // [64][LD]
+  float *Ss = Ks + 64 * LD;            // [64][LDS] scaled logits of the tile
+  int *is_cur = reinterpret_cast<int *>(Ss + 64 * LDS);   // [64] the tile's entries that belong to the current map
+  float *top = reinterpret_cast<float *>(is_cur + 64);    // [256][K'] per-thread descending lists
+  __shared__ float red_c[8], red_t[8];
+  const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
   const int slice = blockIdx.y;
   const int b = slice / lv.n_heads, h = slice % lv.n_heads;
-  const int qi = blockIdx.x * stride;
   const int L = lv.hist_len[slice] + n_k;
-  if (threadIdx.x < CH) {
+  const int r0 = blockIdx.x * 64;
+  const int Kp = topk_prime;
+  for (int idx = tid; idx < 64 * CH; idx += 256) {
+    const int r = idx / CH, c = idx % CH;
     float v[VN];
-    Vec16<T>::load(row_ptr<T>(Q, b, h, qi) + threadIdx.x * VN, v);
+    if (r0 + r < n_rows) {
+      Vec16<T>::load(row_ptr<T>(Q, b, h, (r0 + r) * stride) + c * VN, v);
+    } else {
 #pragma unroll
-    for (int e = 0; e < VN; ++e) qs[threadIdx.x * VN + e] = v[e];
+      for (int e = 0; e < VN; ++e) v[e] = 0.f;
+    }
+#pragma unroll
+    for (int e = 0; e < VN; ++e) Qs[r * LD + c * VN + e] = v[e];
+  }
+  float *mine = top + (size_t)tid * (Kp > 0 ? Kp : 1);
+  for (int e = 0; e < Kp; ++e) mine[e] = -INFINITY;
+  // row statistics of the 4 threads that share a row (row = tid >> 2): kept redundantly in each of them
+  const int row = tid >> 2, part = tid & 3;
+  float m_run = -INFINITY, z_run = 0.f, cur_run = 0.f;
+  float thr = Kp > 0 ? -INFINITY : INFINITY;           // the smallest member of this thread's list (nothing enters when K' = 0)
+  for (int j0 = 0; j0 < L; j0 += 64) {
+    __syncthreads();
+    load_tile_rows<T, D>(Ks, LD, lv, lv.k_pool, slice, j0, L);
+    if (tid < 64) is_cur[tid] = (j0 + tid < L) ? (lv.pos_pool[slot_row(lv, slice, j0 + tid)] >= n_prev ? 1 : 0) : 0;
+    __syncthreads();
+    float s[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) s[i][j] = 0.f;
+    for (int c = 0; c < D; c += 4) {
+      float4 q[4], k[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) q[i] = *reinterpret_cast<const float4 *>(&Qs[(ty + 16 * i) * LD + c]);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) k[j] = *reinterpret_cast<const float4 *>(&Ks[(tx + 16 * j) * LD + c]);
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          s[i][j] = fmaf(q[i].x, k[j].x, s[i][j]);
+          s[i][j] = fmaf(q[i].y, k[j].y, s[i][j]);
+          s[i][j] = fmaf(q[i].z, k[j].z, s[i][j]);
+          s[i][j] = fmaf(q[i].w, k[j].w, s[i][j]);
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        Ss[(ty + 16 * i) * LDS + tx + 16 * j] = (j0 + tx + 16 * j < L) ? s[i][j] * scale : -INFINITY;
+    __syncthreads();
+    {
+      const float *srow = Ss + row * LDS + part * 16;
+      float mx = -INFINITY;
+#pragma unroll
+      for (int e = 0; e < 16; ++e) mx = fmaxf(mx, srow[e]);
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+      const float m_new = fmaxf(m_run, mx);            // finite: every tile holds at least one entry
+      float sum = 0.f, cur = 0.f;
+#pragma unroll
+      for (int e = 0; e < 16; ++e) {
+        const float v = srow[e];
+        const float pe = expf(v - m_new);              // 0 for the padding beyond L
+        sum += pe;
+        if (is_cur[part * 16 + e]) {
+          cur += pe;
+        } else if (v > thr) {                          // a history logit that enters this thread's K' largest
+          int at = Kp - 1;
+          while (at > 0 && mine[at - 1] < v) { mine[at] = mine[at - 1]; --at; }
+          mine[at] = v;
+          thr = mine[Kp - 1];
+        }
+      }
+      sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+      sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+      cur += __shfl_xor_sync(0xffffffffu, cur, 1);
+      cur += __shfl_xor_sync(0xffffffffu, cur, 2);
+      const float a = expf(m_run - m_new);             // 0 at the first tile
+      z_run = z_run * a + sum;
+      cur_run = cur_run * a + cur;
+      m_run = m_new;
+    }
   }
   __syncthreads();
-  float mx = -INFINITY;
-  for (int i = threadIdx.x; i < L; i += blockDim.x) {
-    const size_t row = slot_row(lv, slice, i);
-    const T *kr = reinterpret_cast<const T *>(lv.k_pool + row * lv.row_bytes);
-    float dot = 0.f;
-#pragma unroll 4
-    for (int c = 0; c < CH; ++c) {
-      float v[VN];
-      Vec16<T>::load(kr + c * VN, v);
-#pragma unroll
-      for (int e = 0; e < VN; ++e) dot = fmaf(qs[c * VN + e], v[e], dot);
+  float c_i = 0.f, t_i = 0.f;
+  if (part == 0 && r0 + row < n_rows) {
+    c_i = cur_run / z_run;
+    // four-way merge of the row's four descending lists: K' largest history logits -> their weights
+    const float *l0 = top + (size_t)(tid + 0) * (Kp > 0 ? Kp : 1), *l1 = top + (size_t)(tid + 1) * (Kp > 0 ? Kp : 1);
+    const float *l2 = top + (size_t)(tid + 2) * (Kp > 0 ? Kp : 1), *l3 = top + (size_t)(tid + 3) * (Kp > 0 ? Kp : 1);
+    int i0 = 0, i1 = 0, i2 = 0, i3 = 0;
+    float tsum = 0.f;
+    for (int e = 0; e < Kp; ++e) {
+      const float v0 = i0 < Kp ? l0[i0] : -INFINITY, v1 = i1 < Kp ? l1[i1] : -INFINITY;
+      const float v2 = i2 < Kp ? l2[i2] : -INFINITY, v3 = i3 < Kp ? l3[i3] : -INFINITY;
+      const float best = fmaxf(fmaxf(v0, v1), fmaxf(v2, v3));
+      if (best == -INFINITY) break;                    // history exhausted
+      tsum += expf(best - m_run);
+      if (best == v0) ++i0; else if (best == v1) ++i1; else if (best == v2) ++i2; else ++i3;
     }
-    dot *= scale;
-    p[i] = dot;
-    mx = fmaxf(mx, dot);
+    t_i = tsum / z_run;
   }
-  mx = block_reduce_max(mx, red);
-  float sum = 0.f;
-  for (int i = threadIdx.x; i < L; i += blockDim.x) {
-    const float e = expf(p[i] - mx);
-    p[i] = e;
-    sum += e;
+  // the block's sums, in a fixed order
+  for (int o = 16; o > 0; o >>= 1) {
+    c_i += __shfl_xor_sync(0xffffffffu, c_i, o);
+    t_i += __shfl_xor_sync(0xffffffffu, t_i, o);
   }
-  sum = block_reduce_sum(sum, red);
-  const float inv = 1.f / sum;
-  float cur = 0.f;
-  for (int i = threadIdx.x; i < L; i += blockDim.x) {
-    const int ps = lv.pos_pool[slot_row(lv, slice, i)];
-    const float a = p[i] * inv;
-    if (ps >= n_prev) { cur += a; p[i] = -1.f; } else { p[i] = a; }
-  }
-  cur = block_reduce_sum(cur, red);
-  float top = 0.f;
-  for (int round = 0; round < topk_prime; ++round) {
-    float bv = -1.f;
-    int bi = -1;
-    for (int i = threadIdx.x; i < L; i += blockDim.x)
-      if (p[i] > bv) { bv = p[i]; bi = i; }
-    for (int o = 16; o > 0; o >>= 1) {
-      const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-      const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-      if (ov > bv || (ov == bv && oi >= 0 && (bi < 0 || oi < bi))) { bv = ov; bi = oi; }
-    }
-    __syncthreads();
-    if ((threadIdx.x & 31) == 0) { best_v[threadIdx.x >> 5] = bv; best_i[threadIdx.x >> 5] = bi; }
-    __syncthreads();
-    bv = best_v[0]; bi = best_i[0];
-    for (int w = 1; w < 8; ++w)
-      if (best_v[w] > bv || (best_v[w] == bv && best_i[w] >= 0 && (bi < 0 || best_i[w] < bi))) { bv = best_v[w]; bi = best_i[w]; }
-    if (bi < 0 || bv < 0.f) break;   // history exhausted (uniform across the block)
-    top += bv;
-    __syncthreads();
-    if (threadIdx.x == 0) p[bi] = -1.f;
-    __syncthreads();
-  }
-  if (threadIdx.x == 0) {
-    atomicAdd(&acc[0], (double)cur);
-    atomicAdd(&acc[1], (double)top);
+  if ((tid & 31) == 0) { red_c[tid >> 5] = c_i; red_t[tid >> 5] = t_i; }
+  __syncthreads();
+  if (tid == 0) {
+    float cs = 0.f, ts = 0.f;
+    for (int w = 0; w < 8; ++w) { cs += red_c[w]; ts += red_t[w]; }
+    atomicAdd(&acc[0], (double)cs);
+    atomicAdd(&acc[1], (double)ts);
     // the same sums per slice, behind the two totals
-    atomicAdd(&acc[2 + 2 * blockIdx.y], (double)cur);
-    atomicAdd(&acc[3 + 2 * blockIdx.y], (double)top);
+    atomicAdd(&acc[2 + 2 * blockIdx.y], (double)cs);
+    atomicAdd(&acc[3 + 2 * blockIdx.y], (double)ts);
   }
 }
 

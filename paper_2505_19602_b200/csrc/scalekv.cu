@@ -104,8 +104,16 @@ scalekv_status make_plan(const scalekv_config *c, Plan &p, std::string &err) {
   p.budgets.assign(c->budgets, c->budgets + (size_t)p.n_layers * p.K);
   if (c->window_patches < 0 || c->window_patches > c->max_window) { err = "window_patches must lie in [0, max_window]"; return SCALEKV_ERR_INVALID_ARG; }
   p.windows.assign(p.K, std::vector<int>());
+  if (c->window_kind != SCALEKV_WINDOW_CENTROIDS && c->window_kind != SCALEKV_WINDOW_LAST) { err = "unknown window_kind"; return SCALEKV_ERR_INVALID_ARG; }
   if (c->window_patches > 0)
-    for (int k = 0; k < p.K; ++k) p.windows[k] = centroid_window(c->scale_h[k], c->scale_w[k], c->window_patches);
+    for (int k = 0; k < p.K; ++k) {
+      if (c->window_kind == SCALEKV_WINDOW_LAST) {
+        const int m = std::min(c->window_patches, p.n[k]);
+        for (int i = 0; i < m; ++i) p.windows[k].push_back(p.n[k] - m + i);
+      } else {
+        p.windows[k] = centroid_window(c->scale_h[k], c->scale_w[k], c->window_patches);
+      }
+    }
   p.layers.resize(p.n_layers);
   int trans_max = 0, len_max = 0;
   size_t pt = 0;
@@ -448,9 +456,9 @@ scalekv_status scalekv_init(const scalekv_config *cfg, scalekv_ctx **out) {
     if (cfg->dtype == SCALEKV_BF16) {
       ok = ok && set_smem(attend_simt_kernel<__nv_bfloat16, 128>, (64 * 132 * 2 + 64 * 65 + 192) * 4);
       ok = ok && set_smem(score_logits_kernel<__nv_bfloat16, 128>, 2 * 64 * 132 * 4);
-      ok = ok && set_smem(layer_stats_kernel<__nv_bfloat16, 128>, (size_t)(128 + p.ld_s) * 4);
+      ok = ok && set_smem(layer_stats_kernel<__nv_bfloat16, 128>, layer_stats_smem_bytes<128>(64));
     } else {
-      ok = ok && set_smem(layer_stats_kernel<float, 64>, (size_t)(64 + p.ld_s) * 4);
+      ok = ok && set_smem(layer_stats_kernel<float, 64>, layer_stats_smem_bytes<64>(64));
       ok = ok && set_smem(attend_simt_kernel<float, 64>, (64 * 68 * 2 + 64 * 65 + 192) * 4);
       ok = ok && set_smem(score_logits_kernel<float, 64>, 2 * 64 * 68 * 4);
     }
@@ -891,20 +899,19 @@ scalekv_status scalekv_layer_stats_ex(scalekv_ctx *ctx, int32_t layer, scalekv_t
   if (st0 != SCALEKV_OK) return st0;
   const int nk = ctx->pending[layer];
   const int k = ctx->next_scale[layer] - 1;
-  const int L = ctx->hist[layer] + nk;
   const int rows = (nk + query_stride - 1) / query_stride;
   double *acc = reinterpret_cast<double *>(ctx->ws + p.off_acc);
   const size_t acc_bytes = 16 + (size_t)p.n_slices * 16;
   CU(cudaMemsetAsync(acc, 0, acc_bytes, ctx->s_main));
   {
     Scope sc(ctx, ctx->s_main, kOther);
-    dim3 grid(rows, p.n_slices);
+    dim3 grid((rows + 63) / 64, p.n_slices);
     if (ctx->dtype == SCALEKV_BF16)
-      layer_stats_kernel<__nv_bfloat16, 128><<<grid, 256, (size_t)(128 + L) * 4, ctx->s_main>>>(
-          layer_view(ctx, layer), tview(Q), nk, p.N[k], query_stride, topk_prime, ctx->scale, acc);
+      layer_stats_kernel<__nv_bfloat16, 128><<<grid, 256, layer_stats_smem_bytes<128>(topk_prime), ctx->s_main>>>(
+          layer_view(ctx, layer), tview(Q), nk, p.N[k], query_stride, rows, topk_prime, ctx->scale, acc);
     else
-      layer_stats_kernel<float, 64><<<grid, 256, (size_t)(64 + L) * 4, ctx->s_main>>>(
-          layer_view(ctx, layer), tview(Q), nk, p.N[k], query_stride, topk_prime, ctx->scale, acc);
+      layer_stats_kernel<float, 64><<<grid, 256, layer_stats_smem_bytes<64>(topk_prime), ctx->s_main>>>(
+          layer_view(ctx, layer), tview(Q), nk, p.N[k], query_stride, rows, topk_prime, ctx->scale, acc);
   }
   scalekv_status st = check_launch(ctx, "layer_stats");
   if (st != SCALEKV_OK) return st;
@@ -979,6 +986,31 @@ scalekv_status scalekv_make_budgets(const uint8_t *is_drafter, int32_t L, int32_
     const double bd = (b_uniform * L - nr * br) / nd;
     for (int l = 0; l < L; ++l)
       budgets_out[(size_t)l * K + k] = (int32_t)std::floor((is_drafter[(size_t)l * K + k] ? bd : br) + 0.5);
+  }
+  return SCALEKV_OK;
+}
+
+scalekv_status scalekv_window_last(int32_t h, int32_t w, int32_t n_obs, int32_t *pos, int32_t *count) {
+  if (h < 1 || w < 1 || n_obs < 1 || !pos || !count) return SCALEKV_ERR_INVALID_ARG;
+  const long long n = (long long)h * w;
+  const int m = (int)std::min<long long>(n_obs, n);
+  for (int i = 0; i < m; ++i) pos[i] = (int32_t)(n - m + i);
+  *count = m;
+  return SCALEKV_OK;
+}
+
+scalekv_status scalekv_policy_budgets(int32_t shape, int32_t L, int32_t K, double b_mean, double beta, int32_t *budgets_out) {
+  if (!budgets_out || L < 1 || K < 1 || !(b_mean >= 0.0)) return SCALEKV_ERR_INVALID_ARG;
+  if (shape != SCALEKV_BUDGETS_UNIFORM && shape != SCALEKV_BUDGETS_PYRAMID) return SCALEKV_ERR_INVALID_ARG;
+  if (shape == SCALEKV_BUDGETS_PYRAMID && !(beta >= 1.0)) return SCALEKV_ERR_INVALID_ARG;
+  for (int l = 0; l < L; ++l) {
+    double b = b_mean;
+    if (shape == SCALEKV_BUDGETS_PYRAMID && L > 1) {
+      const double b_min = b_mean / beta, b_max = 2.0 * b_mean - b_min;
+      b = b_max - (b_max - b_min) * l / (L - 1);
+    }
+    const int32_t v = (int32_t)std::floor(b + 0.5);
+    for (int k = 0; k < K; ++k) budgets_out[(size_t)l * K + k] = v;
   }
   return SCALEKV_OK;
 }

@@ -73,12 +73,14 @@ class PassInputs:
         return total
 
 
-def run_pass(kv: binding.ScaleKV, inputs: PassInputs, windows, compress_last=False, marks=None, three_calls=False):
+def run_pass(kv: binding.ScaleKV, inputs: PassInputs, windows, compress_last=False, marks=None, three_calls=False, select=None):
     """One pass: reset, then for every scale and layer append -> attend -> compress (one scalekv_step per
     layer and scale, or the three calls one by one with three_calls=True: the same launches either way).
 
     marks: a list that receives CUDA events recorded on stream_main before the reset, after it, and after
     every scale-step (2 + n_scales events), for per-scale-step latencies.
+    select: options of scalekv_compress_ex (policy, pool_kernel, n_sink) for the comparison policies; the
+    compress of every step then goes through that call.
     """
     wl = inputs.wl
 
@@ -100,6 +102,12 @@ def run_pass(kv: binding.ScaleKV, inputs: PassInputs, windows, compress_last=Fal
         wp = kv.window_array(windows[k]) if (do_compress and windows[k] is not None) else None
         for l in range(wl.n_layers):
             Q, K, V = inputs.data[(l, k)]
+            if select is not None:
+                kv.scalekv_append(l, k, K, V)
+                kv.scalekv_attend(l, Q, O)
+                if do_compress:
+                    kv.scalekv_compress_ex(l, Q, windows[k], qw_is_full_map=True, **select)
+                continue
             if not three_calls:
                 kv.scalekv_step(l, k, Q, K, V, O, window_pos=wp, whole_map=do_compress and wp is None)
                 continue
@@ -113,7 +121,7 @@ def run_pass(kv: binding.ScaleKV, inputs: PassInputs, windows, compress_last=Fal
         mark()
 
 
-def pass_work(wl: synth.Workload, budgets, windows):
+def pass_work(wl: synth.Workload, budgets, windows, recent=False):
     """Algorithmic work of one pass, from the schedule alone.
 
     attend_flop       4 n_k L d per slice-step.
@@ -141,6 +149,7 @@ def pass_work(wl: synth.Workload, budgets, windows):
         for k in range(wl.n_scales):
             L = hist + n[k]
             w = len(windows[k]) if windows[k] is not None else n[k]
+            wk = 0 if recent else w          # the positional rules have no window: their budget is the whole cache
             f = 4 * n[k] * L * d * slices
             out["attend_flop"] += f
             per_scale_flop[k] += f
@@ -152,18 +161,18 @@ def pass_work(wl: synth.Workload, budgets, windows):
             out["attend_launches"] += 1
             if k + 1 == wl.n_scales:
                 break
-            cand = L - w
+            cand = L - wk
             b = budgets[l][k]
             if b != binding.KEEP_ALL and b < cand:
                 if not fused:
                     out["score_bytes"] += L * d * esz * slices
-                out["score_bytes"] += (4 * w * L + 4 * L + 4 * L + 4 * L) * slices
-                out["select_bytes"] += (4 * L + 4 * (b + w)) * slices
-                out["compact_bytes"] += (b + w) * (2 * 2 * d * esz + 8) * slices
+                out["score_bytes"] += (4 * wk * L + 4 * L + 4 * L + 4 * L) * slices
+                out["select_bytes"] += (4 * L + 4 * (b + wk)) * slices
+                out["compact_bytes"] += (b + wk) * (2 * 2 * d * esz + 8) * slices
                 # the one-launch compress: logits and positions in, scores out, the survivors' rows moved
-                out["compress_bytes"] += ((4 * w * L + 4 * L + 4 * L) + (b + w) * (2 * 2 * d * esz + 8)) * slices
+                out["compress_bytes"] += ((4 * wk * L + 4 * L + (0 if recent else 4 * L)) + (b + wk) * (2 * 2 * d * esz + 8)) * slices
                 out["compress_launches"] += 1
-                hist = b + w
+                hist = b + wk
             else:
                 hist = L
     out["per_scale_flop"] = per_scale_flop

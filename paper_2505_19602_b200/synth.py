@@ -27,6 +27,7 @@ import torch
 SIDES_4 = (1, 2, 4, 8)
 SIDES_13 = (1, 2, 4, 6, 8, 12, 16, 20, 24, 32, 40, 48, 64)
 SIDES_16 = SIDES_13 + (80, 96, 128)
+SIDES_19 = SIDES_16 + (160, 192, 256)      # a 4K-class image at the same 16 x downsampling: 170 521 tokens
 
 
 @dataclass
@@ -72,6 +73,9 @@ WORKLOADS = {
     "hires": Workload("hires", 32, 4, 16, 128, "bf16", SIDES_16, seed=5, n_drafters=8),
     # the headline pass with the batch doubled, as under classifier-free guidance (a conditional and an
     # unconditional branch per image run through the same layers)
+    # beyond configs[4]: the "ultra-high resolutions such as 4K" the paper names as the method's target (Sec. 4.3):
+    # 19 scales up to 256 x 256; a slice outgrows one CTA's shared memory, so select and compact work from global memory
+    "uhd4k": Workload("uhd4k", 32, 1, 16, 128, "bf16", SIDES_19, seed=7, n_drafters=8),
     "pass2b_cfg": Workload("pass2b_cfg", 32, 16, 16, 128, "bf16", SIDES_13, seed=6, n_drafters=8),
 }
 

@@ -35,6 +35,9 @@ class ParityRun:
         self.max_lse_err = 0.0
         self.evictions = 0
         self.separate_kernels = False  # compress as three launches (the path long slices take) instead of one
+        self.policy = "score"          # "score": observation-window importance; "recent": positional (sliding window, sinks)
+        self.pool_kernel = 1           # width of the pooling of the importance along the keys (score policy)
+        self.n_sink = 0                # always-kept lowest positions (recent policy)
         self.compared = 0             # slice-steps whose attention output was compared
         self.rel_bound_used = 0       # ... of which the relative branch of the bf16 bound (|O| > 2.56) decided
 
@@ -53,8 +56,9 @@ class ParityRun:
                 O = kv.scalekv_attend(l, Qd, lse=lse)
                 do_compress = (k + 1 < len(self.n)) or self.compress_last
                 if do_compress:
-                    if self.separate_kernels:
-                        kv.scalekv_compress_ex(l, Qd, wpos, qw_is_full_map=True, separate_kernels=True)
+                    if self.separate_kernels or self.policy != "score" or self.pool_kernel > 1:
+                        kv.scalekv_compress_ex(l, Qd, wpos, qw_is_full_map=True, policy=self.policy, pool_kernel=self.pool_kernel,
+                                               n_sink=self.n_sink, separate_kernels=self.separate_kernels)
                     elif wpos is None:
                         kv.scalekv_compress(l, Qd, None)
                     else:
@@ -109,7 +113,14 @@ class ParityRun:
             def steps():
                 for l in range(n_layers):
                     Qd, Kd, Vd = dev[l]
-                    kv.scalekv_step(l, k, Qd, Kd, Vd, O[l], window_pos=wp, whole_map=do_compress and wp is None, lse=lse[l])
+                    if self.policy == "score" and self.pool_kernel == 1:
+                        kv.scalekv_step(l, k, Qd, Kd, Vd, O[l], window_pos=wp, whole_map=do_compress and wp is None, lse=lse[l])
+                        continue
+                    kv.scalekv_append(l, k, Kd, Vd)
+                    kv.scalekv_attend(l, Qd, O[l], lse=lse[l])
+                    if do_compress:
+                        kv.scalekv_compress_ex(l, Qd, wpos, qw_is_full_map=True, policy=self.policy, pool_kernel=self.pool_kernel,
+                                               n_sink=self.n_sink)
 
             if mode == "graph":
                 g = torch.cuda.CUDAGraph()
@@ -213,11 +224,19 @@ class ParityRun:
         if not do_compress:
             return
         nk = self.n[k]
-        w_list = list(range(nk)) if wpos is None else list(wpos)
         budget = self.budgets[l][k]
         L = len(cache)
         before_pos = cache.pos.copy()
-        s = cache.scores(Q[w_list])
+        if self.policy == "recent":
+            # positional rule: the budget counts the whole cache, sinks included; nothing to score, no ties
+            keep = orc.select_recent(cache.pos, budget, self.n_sink)
+            got_pos = kv.scalekv_export_slice(l, b, h).numpy().astype(np.int64)
+            assert np.array_equal(got_pos, cache.pos[keep]), f"slice {key} scale {k}: positional rule kept other entries"
+            self.evictions += int(len(keep) < L)
+            cache.adopt(keep)
+            return
+        w_list = list(range(nk)) if wpos is None else list(wpos)
+        s = orc.pool_scores(cache.scores(Q[w_list]), self.pool_kernel)
         keep = orc.select(s, cache.pos, cache.N[k], w_list, budget)
         want_pos = cache.pos[keep]
         if not exported:
@@ -254,5 +273,5 @@ class ParityRun:
         assert np.array_equal(to64(Vg), cache.V), f"slice {key} scale {k}: compacted V rows differ"
         if kprime < cand:
             sg = kv.scalekv_export_scores(b, h).numpy().astype(np.float64) if scores_fresh else None
-            if sg is not None and len(sg) == L:
+            if sg is not None and len(sg) == L and self.pool_kernel == 1:
                 assert np.all(np.abs(sg - s) <= 2e-4 * s + 1e-9), "importance scores differ"

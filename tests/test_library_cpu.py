@@ -103,3 +103,12 @@ def test_budget_tokens_matches_oracle(lib):
             assert binding.scalekv_budget_tokens(f, sides) == orc.budget_tokens(f, n), (sides, f)
     assert binding.scalekv_budget_tokens(0.30, SIDES_13) == 1928        # 1927.5 rounds up
     assert binding.scalekv_budget_tokens(0.5, (1, 1, 1)) == 1 and binding.scalekv_budget_tokens(0.25, (1, 1, 1)) == 1
+
+
+def test_comparison_policy_helpers_match_oracle(lib):
+    for h, w, n in ((3, 5, 16), (8, 8, 16), (6, 10, 4), (1, 1, 16), (64, 64, 16)):
+        assert binding.scalekv_window_last(h, w, n) == orc.window_last(h, w, n)
+    for shape in ("uniform", "pyramid"):
+        for L, b, beta in ((32, 627, 20.0), (40, 1300.5, 20.0), (5, 100, 4.0), (1, 77, 20.0), (6, 50, 1.0)):
+            assert np.array_equal(binding.scalekv_policy_budgets(shape, L, 4, b, beta), orc.policy_budgets(shape, L, 4, b, beta))
+

@@ -517,3 +517,23 @@ def test_normalized_current_attention_closed_forms():
     assert abs(orc.normalized_current_attention(Q, K, pos, n_prev, query_stride=3) - total / 4) < 1e-12
     sc, _, cnt = orc.layer_stats_slice(Q, K, pos, n_prev, 4, query_stride=3)
     assert abs(orc.normalized_current_attention(Q, K, pos, n_prev, query_stride=3) - sc / cnt * L / nk) < 1e-12
+
+
+def test_comparison_policy_helpers_closed_forms():
+    """window_last: the tail of the raster order.  policy_budgets: "pyramid" is an arithmetic series over the
+    layers whose mean is b_mean (so the total equals the uniform table's up to rounding), strictly falling, from
+    2 b_mean - b_mean / beta down to b_mean / beta; beta = 1, one layer and "uniform" all give b_mean."""
+    assert orc.window_last(3, 5, 16) == list(range(15)) and orc.window_last(8, 8, 16) == list(range(48, 64))
+    assert orc.window_last(6, 10, 4) == [56, 57, 58, 59] and orc.window_last(1, 1, 16) == [0]
+    for L, b, beta in ((32, 627, 20.0), (40, 1300, 20.0), (5, 100, 4.0), (2, 11, 3.0)):
+        t = orc.policy_budgets("pyramid", L, 3, b, beta)
+        assert t.shape == (L, 3) and np.all(t[:, 0] == t[:, 1]) and np.all(t[:, 0] == t[:, 2])
+        col = t[:, 0]
+        assert abs(int(col.sum()) - L * b) <= L // 2 + 1          # rounding residue of an exact series sum L * b
+        assert np.all(np.diff(col) < 0)
+        assert col[0] == math.floor(2 * b - b / beta + 0.5) and col[-1] == math.floor(b / beta + 0.5)
+        assert abs((col[0] + col[-1]) / 2 - b) <= 1
+    assert np.all(orc.policy_budgets("pyramid", 6, 2, 50, 1.0) == 50)
+    assert np.all(orc.policy_budgets("pyramid", 1, 4, 77, 20.0) == 77)
+    assert np.all(orc.policy_budgets("uniform", 7, 3, 642.5) == 643)
+

@@ -1085,3 +1085,87 @@ def test_compress_as_three_launches_matches_oracle():
     run.run()
     assert run.evictions >= 40 and run.resyncs == 0
     kv.close()
+
+
+@pytest.mark.parametrize("policy", ["sliding", "sinks", "snapkv", "pyramid"])
+@pytest.mark.parametrize("mode", ["synced", "pipelined"])
+def test_comparison_policies_match_oracle(policy, mode):
+    """The four comparison rules of Sec. 4.1 as configurations of the same store, each against its oracle
+    statement on the ragged five-layer case, step by step and in the benchmark's pipelined mode: sliding window
+    and sinks + recent (positional), the SnapKV-like rule (observed by the last 16 rows of the map, importance
+    pooled over 7 neighbouring keys, uniform table) and pyramid budgets (the same rule, the table falling with
+    the layer index)."""
+    sides, _, wl = _ragged_five_layer_case()
+    K = len(sides)
+    if policy in ("sliding", "sinks"):
+        table = binding.scalekv_policy_budgets("uniform", 5, K, 76)
+        window = lambda k: binding.scalekv_window_centroids(sides[k], sides[k], 16)     # ignored by the positional rules
+        kind = "centroids"
+    else:
+        table = binding.scalekv_policy_budgets("uniform" if policy == "snapkv" else "pyramid", 5, K, 60, 6.0)
+        assert np.array_equal(table, orc.policy_budgets("uniform" if policy == "snapkv" else "pyramid", 5, K, 60, 6.0))
+        window = lambda k: orc.window_last(sides[k], sides[k], 16)
+        kind = "last"
+    budgets = [[int(x) for x in row] for row in table]
+    kv = binding.ScaleKV(5, 2, 2, 128, "bf16", sides, sides, budgets, max_window=16, window_kind=kind)
+    run = ParityRun(kv, "bf16", sides, budgets, lambda l, k: synth.scale_inputs(wl, l, k), window, all_slices(5, 2, 2))
+    if policy in ("sliding", "sinks"):
+        run.policy, run.n_sink = "recent", (4 if policy == "sinks" else 0)
+    else:
+        run.pool_kernel = 7
+    run = run.run() if mode == "synced" else run.run_pipelined("eager")
+    print(policy, mode, run.summary())
+    assert run.evictions >= 30
+    if policy == "pyramid":
+        lens = [kv.scalekv_lengths(l)[0][0] for l in range(5)]
+        assert lens == sorted(lens, reverse=True) and lens[0] > lens[-1]         # the store really is pyramid-shaped
+    kv.close()
+
+
+def test_refiner_decay_table_on_the_headline_shape():
+    """The paper's own budget constants on the 13-scale shape: 650 tokens per head and layer on average,
+    B_r(0) = 600, refiner decay delta = 70 (Sec. 4.3, "Impact of Refiner Budget Decay Rate"; Eq. 4), with 8
+    drafters per ranked scale.  The table differs from scale to scale and the refiners' budget is clamped at 0
+    from scale 9 on (only the window survives); all 32 layers run pipelined like the benchmark, the oracle
+    follows 8 slices."""
+    wl = synth.WORKLOADS["pass2b"]
+    planted = synth.drafter_layers(wl)
+    roles = np.zeros((wl.n_layers, wl.n_scales), dtype=bool)
+    roles[planted, 1:wl.n_scales - 1] = True                                      # scales 1 and K are not ranked
+    table = binding.scalekv_make_budgets(roles, 650, 600, 70)
+    assert np.array_equal(table, orc.make_budgets(roles, 650, 600, 70))
+    refiner = [l for l in range(wl.n_layers) if l not in planted][0]
+    assert table[refiner, 1] == 460 and table[refiner, 8] == 0 and table[planted[0], 8] == 2600 and table[refiner, 0] == 650
+    budgets = [[int(x) for x in row] for row in table]
+    kv = binding.ScaleKV(wl.n_layers, wl.batch, wl.n_heads, 128, "bf16", wl.sides, wl.sides, budgets, max_window=16)
+    slices = sampled_slices(wl, planted, 8)
+    run = ParityRun(kv, "bf16", wl.sides, budgets, lambda l, k: synth.scale_inputs(wl, l, k, device="cuda"),
+                    lambda k: orc.window_centroids(wl.sides[k], wl.sides[k], 16), slices, check_lse=True,
+                    max_rows=1024).run_pipelined("eager")
+    print("650 / 600 / delta 70:", run.summary())
+    assert run.evictions > 0
+    assert kv.scalekv_lengths(refiner)[0][0] == 16 + wl.n_tokens[-1]              # window of scale 12 + the last map
+    kv.close()
+
+
+def test_4k_class_schedule_sampled_slices():
+    """A schedule beyond configs[4]: 19 scales up to 256 x 256 (170 521 tokens, a cache of up to 98 000 entries
+    per slice).  A slice no longer fits one CTA's shared memory, so the selection streams its keys from global
+    memory and the pruning reads its keep list there.  One drafter and one refiner layer at the 10 % point
+    (30.77 % / 3.077 % of the cached tokens), two heads, pipelined; attention compared on 192 rows per map."""
+    sides = synth.SIDES_19
+    wl = synth.Workload("uhd4k-2", 2, 1, 2, 128, "bf16", sides, seed=7, n_drafters=1)
+    n = wl.n_tokens
+    bd, br = orc.budget_tokens(0.3077, n), orc.budget_tokens(0.03077, n)
+    assert bd == binding.scalekv_budget_tokens(0.3077, sides) and bd > 30000
+    planted = synth.drafter_layers(wl)
+    budgets = [[bd if l in planted else br] * wl.n_scales for l in range(2)]
+    kv = binding.ScaleKV(2, 1, 2, 128, "bf16", sides, sides, budgets, max_window=16)
+    run = ParityRun(kv, "bf16", sides, budgets, lambda l, k: synth.scale_inputs(wl, l, k, device="cuda"),
+                    lambda k: orc.window_centroids(sides[k], sides[k], 16), all_slices(2, 1, 2), check_lse=True,
+                    max_rows=192).run_pipelined("eager")
+    print("4K-class:", run.summary())
+    assert run.evictions > 0
+    assert kv.scalekv_lengths(planted[0])[0][0] == bd + 16 + n[-1]
+    kv.close()
+
