@@ -95,8 +95,8 @@ typedef struct {
 
 /* Bytes of pool and workspace that scalekv_init needs for this configuration (pointers in cfg
  * are ignored).  The pool holds, per layer, ceil(cap_l / page_tokens) persistent pages per slice,
- * cap_l being the largest cache a compress leaves behind, plus two transient page sets (even /
- * odd layers) that hold the part of the current map that exceeds cap_l until that layer's
+ * cap_l being the largest cache a compress leaves behind, plus four transient page sets (layer l
+ * uses set l mod 4) that hold the part of the current map that exceeds cap_l until that layer's
  * compress; page tables; per-slice lengths.  No CUDA call is made. */
 scalekv_status scalekv_query_sizes(const scalekv_config *cfg, size_t *pool_bytes, size_t *workspace_bytes);
 
@@ -128,9 +128,9 @@ scalekv_status scalekv_destroy(scalekv_ctx *ctx);
  * next append) copies first with a kernel of its own.  K and V must therefore stay unmodified
  * until stream_main has passed the layer's next call.  For f32 x 64 the copy is enqueued here.
  * Ordered on stream_main after this layer's previous compress.
- * Layers of equal parity (0, 2, 4, .. / 1, 3, 5, ..) share one transient page set, which holds the part of a
+ * Layers l, l + 4, l + 8, .. share one transient page set, which holds the part of a
  * current map that exceeds the layer's persistent capacity, and one buffer of recorded window logits.  An append
- * therefore returns SCALEKV_ERR_BAD_STATE, and touches nothing, while another layer of the same parity still
+ * therefore returns SCALEKV_ERR_BAD_STATE, and touches nothing, while another layer of the same set still
  * holds an appended map that reaches into the transient pages and has not been compressed; otherwise it waits
  * (on stream_main) for that layer's last compress.  The one exception is a map of the LAST scale that has been
  * attended: no later step reads it, so its transient rows are given up, and that layer then refuses compress and

@@ -161,7 +161,9 @@ __device__ __forceinline__ void tma_store_4d(const CUtensorMap *tm, uint32_t src
                : "memory");
 }
 __device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+// waits until the bulk stores committed so far have READ their shared-memory source (the CTA may then leave; the
+// writes to global memory complete on their own)
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 // orders this thread's shared-memory writes before later reads of the asynchronous (TMA) proxy
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
@@ -489,10 +491,18 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
+  // Everybody but the TMA warp waits here for the barriers (initialised by that warp's first thread) and for the
+  // TMEM allocation.  The TMA warp needs neither the TMEM address nor anybody else: it only announces that the
+  // barriers are ready and goes on to issue the first loads while the allocation is still under way.
   tc_fence_before();
-  __syncthreads();
+  if (warp == 0) {
+    __syncwarp();
+    asm volatile("bar.arrive 1, %0;" ::"n"(kThreads) : "memory");
+  } else {
+    asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory");
+  }
   tc_fence_after();
-  const uint32_t tmem = *tmem_slot;
+  const uint32_t tmem = warp == 0 ? 0u : *tmem_slot;
 
   if (warp < 4) {
   if (warp == 0) {
@@ -802,7 +812,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       if (prm.lse != nullptr && qi < n_k) prm.lse[(size_t)slice * n_k + qi] = (m + log2f(l)) * 0.6931471805599453f;
       if (wrank >= 0) prm.win_lse[(size_t)slice * prm.w + wrank] = m + log2f(l);
     }
-    if (quarter == 0) tma_store_wait_all();   // (a lane that issued nothing has nothing to wait for)
+    if (quarter == 0) tma_store_wait_read();   // (a lane that issued nothing has nothing to wait for)
     tc_fence_before();
   }
   __syncthreads();

@@ -20,6 +20,12 @@ using namespace scalekv;
 
 namespace {
 
+// Layers l, l + kSets, l + 2 kSets, ... share one transient page set and one buffer of recorded window logits: the
+// part of a current map beyond a layer's persistent capacity only lives from that layer's attend to its compress,
+// and with four sets the compress of layer l has the attends of three more layers to hide under before layer
+// l + 4 needs the set back (with two, the chain attend(l) -> compress(l) -> attend(l + 2) bounds the scales whose
+// kernels are short).
+constexpr int kSets = 4;
 constexpr int kNumClasses = 7;
 enum KernelClass { kAppend = 0, kAttend = 1, kScore = 2, kSelect = 3, kCompact = 4, kOther = 5, kCompress = 6 };
 
@@ -41,7 +47,7 @@ struct Plan {
   std::vector<std::vector<int>> windows;   // per scale: rows whose logits attend records (empty: none)
   std::vector<LayerPlan> layers;
   int trans_pages_per_slice = 0;    // size of one transient set per slice
-  int trans_first[2] = {0, 0};
+  int trans_first[kSets] = {0, 0, 0, 0};
   long long n_pages = 0;
   int ld_s = 0;                     // padded max length (leading dimension of per-slice scratch)
   int ld_l = 0;                     // leading dimension of a logit row: room for the history rounded up to a key tile and a ragged last tile
@@ -141,8 +147,7 @@ scalekv_status make_plan(const scalekv_config *c, Plan &p, std::string &err) {
     len_max = std::max(len_max, lp.max_len);
   }
   p.trans_pages_per_slice = trans_max;
-  p.trans_first[0] = (int)page; page += (long long)p.n_slices * trans_max;
-  p.trans_first[1] = (int)page; page += (long long)p.n_slices * trans_max;
+  for (int t = 0; t < kSets; ++t) { p.trans_first[t] = (int)page; page += (long long)p.n_slices * trans_max; }
   if (page > 0x7fffffffLL / p.P) { err = "store too large for 32-bit row indices"; return SCALEKV_ERR_CAPACITY; }
   p.n_pages = page;
   p.pt_elems = pt;
@@ -158,9 +163,9 @@ scalekv_status make_plan(const scalekv_config *c, Plan &p, std::string &err) {
   p.off_status = o; o = align_up(o + 256, 1024);
   p.pool_bytes = o;
   o = 0;
-  p.logits_elems = (size_t)p.n_slices * p.max_window * p.ld_l;   // one buffer per layer parity
-  p.off_logits = o; o = align_up(o + 2 * p.logits_elems * 4, 1024);
-  p.off_wlse = o; o = align_up(o + 2 * (size_t)p.n_slices * p.max_window * 4, 1024);   // one per layer parity
+  p.logits_elems = (size_t)p.n_slices * p.max_window * p.ld_l;   // one buffer per set
+  p.off_logits = o; o = align_up(o + kSets * p.logits_elems * 4, 1024);
+  p.off_wlse = o; o = align_up(o + kSets * (size_t)p.n_slices * p.max_window * 4, 1024);   // one per set
   p.off_scores = o; o = align_up(o + (size_t)p.n_slices * p.ld_s * 4, 1024);
   p.off_keys = o; o = align_up(o + (size_t)p.n_slices * p.ld_s * 4, 1024);
   p.off_keep = o; o = align_up(o + (size_t)p.n_slices * p.ld_s * 4, 1024);
@@ -205,7 +210,7 @@ struct scalekv_ctx {
   bool compact_smem_ok = false;    // the separate compact kernel can stage a slice's keep list in shared memory
   size_t fused_smem = 0;
   bool side_dirty = false;         // stream_side has work that stream_main has not joined yet
-  int set_owner[2] = {-1, -1};     // layer that last appended into the transient page set / logit buffer of each parity
+  int set_owner[kSets] = {-1, -1, -1, -1};   // layer that last appended into each transient page set / logit buffer
   int64_t launches = 0;
   int scores_len = 0;              // length of the score vectors left by the last evicting compress
   bool profile = false;            // launches are bracketed by events
@@ -415,7 +420,7 @@ scalekv_status scalekv_init(const scalekv_config *cfg, scalekv_ctx **out) {
   cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, cfg->device);
   cudaDeviceGetAttribute(&minor, cudaDevAttrComputeCapabilityMinor, cfg->device);
   if (major != 10) return bail(SCALEKV_ERR_UNSUPPORTED);
-  // page tables: persistent pages first, then the transient set of the layer's parity
+  // page tables: persistent pages first, then the transient set the layer shares (layer mod kSets)
   ctx->page_table_host.resize(p.pt_elems);
   for (int l = 0; l < p.n_layers; ++l) {
     const LayerPlan &lp = p.layers[l];
@@ -423,7 +428,7 @@ scalekv_status scalekv_init(const scalekv_config *cfg, scalekv_ctx **out) {
       for (int j = 0; j < lp.total_pages; ++j) {
         int page = j < lp.persist_pages
                        ? lp.first_page + s * lp.persist_pages + j
-                       : p.trans_first[l & 1] + s * p.trans_pages_per_slice + (j - lp.persist_pages);
+                       : p.trans_first[l % kSets] + s * p.trans_pages_per_slice + (j - lp.persist_pages);
         ctx->page_table_host[lp.page_table_off + (size_t)s * lp.total_pages + j] = page;
       }
   }
@@ -510,7 +515,7 @@ scalekv_status scalekv_reset(scalekv_ctx *ctx) {
   std::fill(ctx->in_store.begin(), ctx->in_store.end(), 1);
   std::fill(ctx->logits_of.begin(), ctx->logits_of.end(), -1);
   std::fill(ctx->ev_compress_live.begin(), ctx->ev_compress_live.end(), 0);
-  ctx->set_owner[0] = ctx->set_owner[1] = -1;
+  for (int t = 0; t < kSets; ++t) ctx->set_owner[t] = -1;
   ctx->side_dirty = ctx->s_side != ctx->s_main;   // the side stream was sent behind the reset: a capture has to join it again
   std::fill(ctx->map_lost.begin(), ctx->map_lost.end(), 0);
   return SCALEKV_OK;
@@ -544,11 +549,11 @@ scalekv_status scalekv_append(scalekv_ctx *ctx, int32_t layer, int32_t scale, sc
   if (scale != ctx->next_scale[layer])
     return fail(ctx, SCALEKV_ERR_BAD_STATE, "layer %d expects scale %d, got %d", layer, ctx->next_scale[layer], scale);
   if (!tensor_ok(K, p.esize) || !tensor_ok(V, p.esize)) return fail(ctx, SCALEKV_ERR_INVALID_ARG, "K/V null or rows not 16-byte aligned");
-  // The transient page set and the logit buffer of this layer's parity are shared with every other layer of
-  // that parity.  Their last user (the owner) must be through with them: a pending map of the owner whose
+  // The transient page set and the logit buffer of this layer's set (layer mod kSets) are shared with every other
+  // layer of that set.  Their last user (the owner) must be through with them: a pending map of the owner whose
   // rows reach into the transient pages would be overwritten, so that order of calls is refused; otherwise
   // stream_main waits for the owner's last compress (and for this layer's own).
-  const int par = layer & 1;
+  const int par = layer % kSets;
   const int owner = ctx->set_owner[par];
   if (owner >= 0 && owner != layer && ctx->pending[owner] != 0) {
     const LayerPlan &op = p.layers[owner];
@@ -614,8 +619,8 @@ scalekv_status scalekv_attend(scalekv_ctx *ctx, int32_t layer, scalekv_tensor Q,
       if (fused) { kc = tview(ctx->pend_k[layer]); vc = tview(ctx->pend_v[layer]); }
       const int k = ctx->next_scale[layer] - 1;
       const std::vector<int> &win = p.windows[k];
-      float *wl = win.empty() ? nullptr : reinterpret_cast<float *>(ctx->ws + p.off_logits) + (size_t)(layer & 1) * p.logits_elems;
-      float *wlse = reinterpret_cast<float *>(ctx->ws + p.off_wlse) + (size_t)(layer & 1) * p.n_slices * p.max_window;
+      float *wl = win.empty() ? nullptr : reinterpret_cast<float *>(ctx->ws + p.off_logits) + (size_t)(layer % kSets) * p.logits_elems;
+      float *wlse = reinterpret_cast<float *>(ctx->ws + p.off_wlse) + (size_t)(layer % kSets) * p.n_slices * p.max_window;
       if (!ctx->tc.launch(lv, tview(Q), tview(O), lse, nk, fused ? &kc : nullptr, fused ? &vc : nullptr, p.N[k], ctx->scale, wl,
                           wlse, p.ld_l, win.data(), (int)win.size(), ctx->s_main, e))
         return fail(ctx, SCALEKV_ERR_CUDA, "attend launch: %s", e.c_str());
@@ -721,7 +726,7 @@ scalekv_status scalekv_compress_ex(scalekv_ctx *ctx, int32_t layer, scalekv_tens
     if (st != SCALEKV_OK) return st;
   } else {
     LayerView lv = layer_view(ctx, layer);
-    float *logits = reinterpret_cast<float *>(ctx->ws + p.off_logits) + (size_t)(layer & 1) * p.logits_elems;
+    float *logits = reinterpret_cast<float *>(ctx->ws + p.off_logits) + (size_t)(layer % kSets) * p.logits_elems;
     float *scores = reinterpret_cast<float *>(ctx->ws + p.off_scores);
     int *keep = reinterpret_cast<int *>(ctx->ws + p.off_keep);
     int *kept = reinterpret_cast<int *>(ctx->ws + p.off_kept);
@@ -735,9 +740,9 @@ scalekv_status scalekv_compress_ex(scalekv_ctx *ctx, int32_t layer, scalekv_tens
     bool recorded = recent || (ctx->logits_of[layer] == k && (int)p.windows[k].size() == wa.w);
     for (int j = 0; !recent && recorded && j < wa.w; ++j) recorded = p.windows[k][j] == wa.pos[j];
     if (!recorded) {
-      // this writes the logit buffer of the layer's parity: if another layer of that parity has appended since, what
+      // this writes the logit buffer of the layer's set: if another layer of that set has appended since, what
       // its attend recorded there is lost (its compress scores from K too), and its attend must be through first
-      const int ow = ctx->set_owner[layer & 1];
+      const int ow = ctx->set_owner[layer % kSets];
       if (ow >= 0 && ow != layer) {
         ctx->logits_of[ow] = -1;
         if (s != ctx->s_main && ctx->attended[ow]) CU(cudaStreamWaitEvent(s, ctx->ev_attend[ow], 0));
@@ -754,7 +759,7 @@ scalekv_status scalekv_compress_ex(scalekv_ctx *ctx, int32_t layer, scalekv_tens
                                                                          ctx->scale);
     }
     ctx->logits_of[layer] = -1;
-    float *wlse = reinterpret_cast<float *>(ctx->ws + p.off_wlse) + (size_t)(layer & 1) * p.n_slices * p.max_window;
+    float *wlse = reinterpret_cast<float *>(ctx->ws + p.off_wlse) + (size_t)(layer % kSets) * p.n_slices * p.max_window;
     if (!recorded) {
       Scope sc(ctx, s, kScore);
       row_lse_kernel<<<p.n_slices, 1024, 0, s>>>(lv, wa, logits, p.ld_l, wlse);
