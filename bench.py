@@ -28,11 +28,14 @@ if ROOT not in sys.path:
 
 METRIC = "scale_steps_per_sec"
 # DRAM traffic of the attend kernel: (dram__bytes_read.sum + dram__bytes_write.sum) / algorithmic bytes over the two
-# launches of an ncu capture of one layer of the headline workload, its two largest scales (1548.8 MB measured against
-# 1676 MB algorithmic: part of the appended rows is still in L2 when a launch ends).  The capture runs one layer of the
-# workload; traffic grows in proportion to the bytes a launch must move, so the roofline object reports this ratio times
-# the average algorithmic bytes per launch.  Set to None when the kernel changes after the capture.
-ATTEND_TRAFFIC_RATIO = 1548.8 / 1676.0
+# launches of an ncu capture of one layer of the headline workload, its two largest scales (592.2 + 956.3 = 1548.5 MB
+# measured against 1676 MB algorithmic: part of the appended rows is still in L2 when a launch ends).  The capture runs
+# one layer of the workload; traffic grows in proportion to the bytes a launch must move, so the roofline object reports
+# this ratio times the average algorithmic bytes per launch.  Captured on the kernel as of the commit named below
+# (profiles/attend_tc_kernel_pass2b_1layer.md); set ATTEND_TRAFFIC_RATIO to None when attend_tc.cuh changes after it.
+ATTEND_TRAFFIC_RATIO = 1548.5 / 1676.0
+ATTEND_TRAFFIC_SOURCE = ("ncu capture of attend_tc_kernel at commit ac51e08 (one layer, scales 12 and 13), scaled to the "
+                         "average launch by algorithmic bytes")
 UNIT = "scale-steps/s"
 E2E_HOST_LAYERS = 4
 
@@ -456,7 +459,8 @@ def run_scalekv(args):
                 "frac": (att_tflops / peak_tf) if peak_tf else None,
                 "traffic": (ATTEND_TRAFFIC_RATIO * work["attend_min_bytes"] / max(work["attend_launches"], 1)
                             if ATTEND_TRAFFIC_RATIO and wl.dtype == "bf16" else None),
-                "traffic_unit": "bytes per launch (average launch; ncu capture of one layer scaled by algorithmic bytes)",
+                "traffic_unit": "bytes per launch (average launch)",
+                "traffic_source": ATTEND_TRAFFIC_SOURCE if (ATTEND_TRAFFIC_RATIO and wl.dtype == "bf16") else None,
                 "peak_source": f"{peaks['source']} bf16 sustained (kernel timed inside a long step)",
                 "avg_launch_ms": att_ms / max(att_n, 1),
                 "flop_per_launch_avg": work["attend_flop"] / max(work["attend_launches"], 1),

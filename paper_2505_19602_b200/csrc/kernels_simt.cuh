@@ -864,22 +864,46 @@ __global__ void __launch_bounds__(1024) compress_fused_kernel(LayerView lv, Wind
 // ------------------------------------------------------------------------------------------
 // layer statistics (Eq. 2): for sampled query rows i of the current map, alpha_i = softmax row over all L
 // entries, c_i = mass on the current map, t_i = sum of the K' largest alpha_ij over the history.
-// A CTA of 256 threads owns 64 sampled rows of one slice and streams the slice's keys in tiles of 64, so a
-// key tile is read once for 64 rows.  Per tile: logits by fp32 FMA (thread (ty, tx) owns rows ty + 16 i,
-// columns tx + 16 j), staged in shared memory; then four threads per row, 16 columns each, fold the tile into
-// the row's running maximum, normaliser and current-map mass (online softmax statistics) and into their own
-// descending list of the K' largest history logits seen in their columns (the K' largest weights are the K'
-// largest logits).  Nothing of length L is kept.  At the end one thread per row merges the four lists (K'
-// steps of a four-way merge) and the block adds its rows' c_i and t_i to the accumulators.
-// grid (ceil(n_rows / 64), n_slices); dynamic shared memory: layer_stats_smem_bytes<D>(K').
+// A CTA of 256 threads owns 64 sampled rows of one slice and streams a range of the slice's keys in tiles of
+// 64, so a key tile is read once for 64 rows.  Per tile: logits by fp32 FMA (thread (ty, tx) owns rows
+// ty + 16 i, columns tx + 16 j), staged in shared memory; then four threads per row, 16 columns each, fold the
+// tile into the row's running maximum, normaliser and current-map mass (online softmax statistics) and into
+// their own descending list of the K' largest history logits seen in their columns (the K' largest weights
+// are the K' largest logits).  Nothing of length L is kept.  At the end one thread per row merges the four
+// lists (K' steps of a four-way merge).
+// The calibration runs few slices (one image), so the keys of a slice are split over gridDim.z CTAs to fill
+// the GPU: with one split the block adds its rows' c_i and t_i to the accumulators itself; with several every
+// CTA writes, per row, (maximum, normaliser, current mass, K' largest logits) to `partial` and
+// layer_stats_merge_kernel combines the splits.
+// grid (ceil(n_rows / 64), n_slices, n_split); dynamic shared memory: layer_stats_smem_bytes<D>(K').
 // ------------------------------------------------------------------------------------------
 template <int D> __host__ __device__ constexpr size_t layer_stats_smem_bytes(int topk) {
   return (size_t)(2 * 64 * (D + 4) + 64 * 65 + 64 + 256 * (topk > 0 ? topk : 1)) * 4;
 }
+constexpr int kStatsRec = 4 + 64;        // floats per (split, row) record: m, z, cur, unused, then up to 64 logits
+
+__device__ __forceinline__ void stats_block_accumulate(float c_i, float t_i, double *acc, float *red_c, float *red_t) {
+  const int tid = threadIdx.x;
+  for (int o = 16; o > 0; o >>= 1) {
+    c_i += __shfl_xor_sync(0xffffffffu, c_i, o);
+    t_i += __shfl_xor_sync(0xffffffffu, t_i, o);
+  }
+  if ((tid & 31) == 0) { red_c[tid >> 5] = c_i; red_t[tid >> 5] = t_i; }
+  __syncthreads();
+  if (tid == 0) {
+    float cs = 0.f, ts = 0.f;
+    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) { cs += red_c[w]; ts += red_t[w]; }   // fixed order
+    atomicAdd(&acc[0], (double)cs);
+    atomicAdd(&acc[1], (double)ts);
+    // the same sums per slice, behind the two totals
+    atomicAdd(&acc[2 + 2 * blockIdx.y], (double)cs);
+    atomicAdd(&acc[3 + 2 * blockIdx.y], (double)ts);
+  }
+}
 
 template <typename T, int D>
 __global__ void __launch_bounds__(256) layer_stats_kernel(LayerView lv, TensorView Q, int n_k, int n_prev, int stride, int n_rows,
-                                                          int topk_prime, float scale, double *acc) {
+                                                          int topk_prime, float scale, double *acc, float *partial) {
   constexpr int LD = D + 4, LDS = 65;
   constexpr int CH = D * (int)sizeof(T) / 16;
   constexpr int VN = Vec16<T>::N;
@@ -896,6 +920,9 @@ __global__ void __launch_bounds__(256) layer_stats_kernel(LayerView lv, TensorVi
   const int L = lv.hist_len[slice] + n_k;
   const int r0 = blockIdx.x * 64;
   const int Kp = topk_prime;
+  const int n_split = gridDim.z;
+  const int tiles = (L + 63) >> 6;
+  const int t_lo = (int)((long long)tiles * blockIdx.z / n_split), t_hi = (int)((long long)tiles * (blockIdx.z + 1) / n_split);
   for (int idx = tid; idx < 64 * CH; idx += 256) {
     const int r = idx / CH, c = idx % CH;
     float v[VN];
@@ -908,13 +935,15 @@ __global__ void __launch_bounds__(256) layer_stats_kernel(LayerView lv, TensorVi
 #pragma unroll
     for (int e = 0; e < VN; ++e) Qs[r * LD + c * VN + e] = v[e];
   }
-  float *mine = top + (size_t)tid * (Kp > 0 ? Kp : 1);
+  const int Ks_ = Kp > 0 ? Kp : 1;
+  float *mine = top + (size_t)tid * Ks_;
   for (int e = 0; e < Kp; ++e) mine[e] = -INFINITY;
   // row statistics of the 4 threads that share a row (row = tid >> 2): kept redundantly in each of them
   const int row = tid >> 2, part = tid & 3;
   float m_run = -INFINITY, z_run = 0.f, cur_run = 0.f;
   float thr = Kp > 0 ? -INFINITY : INFINITY;           // the smallest member of this thread's list (nothing enters when K' = 0)
-  for (int j0 = 0; j0 < L; j0 += 64) {
+  for (int t = t_lo; t < t_hi; ++t) {
+    const int j0 = t << 6;
     __syncthreads();
     load_tile_rows<T, D>(Ks, LD, lv, lv.k_pool, slice, j0, L);
     if (tid < 64) is_cur[tid] = (j0 + tid < L) ? (lv.pos_pool[slot_row(lv, slice, j0 + tid)] >= n_prev ? 1 : 0) : 0;
@@ -981,39 +1010,65 @@ __global__ void __launch_bounds__(256) layer_stats_kernel(LayerView lv, TensorVi
   }
   __syncthreads();
   float c_i = 0.f, t_i = 0.f;
-  if (part == 0 && r0 + row < n_rows) {
-    c_i = cur_run / z_run;
-    // four-way merge of the row's four descending lists: K' largest history logits -> their weights
-    const float *l0 = top + (size_t)(tid + 0) * (Kp > 0 ? Kp : 1), *l1 = top + (size_t)(tid + 1) * (Kp > 0 ? Kp : 1);
-    const float *l2 = top + (size_t)(tid + 2) * (Kp > 0 ? Kp : 1), *l3 = top + (size_t)(tid + 3) * (Kp > 0 ? Kp : 1);
+  if (part == 0) {
+    // four-way merge of the row's four descending lists: the K' largest history logits of this key range
+    const float *l0 = top + (size_t)(tid + 0) * Ks_, *l1 = top + (size_t)(tid + 1) * Ks_;
+    const float *l2 = top + (size_t)(tid + 2) * Ks_, *l3 = top + (size_t)(tid + 3) * Ks_;
+    float *rec = nullptr;
+    if (n_split > 1) {
+      rec = partial + ((((size_t)slice * gridDim.x + blockIdx.x) * n_split + blockIdx.z) * 64 + row) * kStatsRec;
+      rec[0] = m_run; rec[1] = z_run; rec[2] = cur_run;
+    }
     int i0 = 0, i1 = 0, i2 = 0, i3 = 0;
     float tsum = 0.f;
     for (int e = 0; e < Kp; ++e) {
       const float v0 = i0 < Kp ? l0[i0] : -INFINITY, v1 = i1 < Kp ? l1[i1] : -INFINITY;
       const float v2 = i2 < Kp ? l2[i2] : -INFINITY, v3 = i3 < Kp ? l3[i3] : -INFINITY;
       const float best = fmaxf(fmaxf(v0, v1), fmaxf(v2, v3));
-      if (best == -INFINITY) break;                    // history exhausted
+      if (rec) rec[4 + e] = best;                      // (-inf once the range's history is exhausted)
+      if (best == -INFINITY) { if (!rec) break; else continue; }
       tsum += expf(best - m_run);
       if (best == v0) ++i0; else if (best == v1) ++i1; else if (best == v2) ++i2; else ++i3;
     }
-    t_i = tsum / z_run;
+    if (r0 + row < n_rows) { c_i = cur_run / z_run; t_i = tsum / z_run; }
   }
-  // the block's sums, in a fixed order
-  for (int o = 16; o > 0; o >>= 1) {
-    c_i += __shfl_xor_sync(0xffffffffu, c_i, o);
-    t_i += __shfl_xor_sync(0xffffffffu, t_i, o);
+  if (n_split == 1) stats_block_accumulate(c_i, t_i, acc, red_c, red_t);
+}
+
+// Combines the key-range splits of layer_stats_kernel: per row the maxima, normalisers and current masses by
+// the usual rescaling, the K' largest history logits by an n_split-way merge of the splits' descending lists.
+// grid (ceil(n_rows / 64), n_slices), 64 threads, one row per thread.
+__global__ void __launch_bounds__(64) layer_stats_merge_kernel(const float *partial, int n_split, int n_rows, int topk_prime,
+                                                               double *acc) {
+  __shared__ float red_c[2], red_t[2];
+  const int row = threadIdx.x;
+  const float *base = partial + (((size_t)blockIdx.y * gridDim.x + blockIdx.x) * n_split * 64 + row) * kStatsRec;
+  const size_t step = (size_t)64 * kStatsRec;          // from one split's record of this row to the next
+  float m = -INFINITY;
+  for (int s = 0; s < n_split; ++s) m = fmaxf(m, base[s * step]);
+  float z = 0.f, cur = 0.f;
+  for (int s = 0; s < n_split; ++s) {
+    const float a = expf(base[s * step] - m);
+    z += base[s * step + 1] * a;
+    cur += base[s * step + 2] * a;
   }
-  if ((tid & 31) == 0) { red_c[tid >> 5] = c_i; red_t[tid >> 5] = t_i; }
-  __syncthreads();
-  if (tid == 0) {
-    float cs = 0.f, ts = 0.f;
-    for (int w = 0; w < 8; ++w) { cs += red_c[w]; ts += red_t[w]; }
-    atomicAdd(&acc[0], (double)cs);
-    atomicAdd(&acc[1], (double)ts);
-    // the same sums per slice, behind the two totals
-    atomicAdd(&acc[2 + 2 * blockIdx.y], (double)cs);
-    atomicAdd(&acc[3 + 2 * blockIdx.y], (double)ts);
+  int head[16];
+  for (int s = 0; s < 16; ++s) head[s] = 0;
+  float tsum = 0.f;
+  for (int e = 0; e < topk_prime; ++e) {
+    float best = -INFINITY;
+    int who = -1;
+    for (int s = 0; s < n_split; ++s) {
+      const float v = head[s] < topk_prime ? base[s * step + 4 + head[s]] : -INFINITY;
+      if (v > best) { best = v; who = s; }
+    }
+    if (who < 0) break;                                // history exhausted
+    tsum += expf(best - m);
+    ++head[who];
   }
+  float c_i = 0.f, t_i = 0.f;
+  if (blockIdx.x * 64 + row < n_rows) { c_i = cur / z; t_i = tsum / z; }
+  stats_block_accumulate(c_i, t_i, acc, red_c, red_t);
 }
 
 }  // namespace scalekv

@@ -26,6 +26,9 @@ namespace {
 // l + 4 needs the set back (with two, the chain attend(l) -> compress(l) -> attend(l + 2) bounds the scales whose
 // kernels are short).
 constexpr int kSets = 4;
+// layer_stats splits a slice's keys over several CTAs while the launch would otherwise leave SMs idle; this many CTAs
+// bound the scratch of their partial results (about 10 MB)
+constexpr int kStatsMaxCtas = 592;
 constexpr int kNumClasses = 7;
 enum KernelClass { kAppend = 0, kAttend = 1, kScore = 2, kSelect = 3, kCompact = 4, kOther = 5, kCompress = 6 };
 
@@ -56,7 +59,7 @@ struct Plan {
   size_t off_k, off_v, off_pos, off_pt, off_len, off_status, pool_bytes;
   size_t pt_elems, logits_elems;
   // workspace layout
-  size_t off_logits, off_wlse, off_scores, off_keys, off_keep, off_kept, off_hbud, off_acc, ws_bytes;
+  size_t off_logits, off_wlse, off_scores, off_keys, off_keep, off_kept, off_hbud, off_acc, off_stats, ws_bytes;
 };
 
 // Raster indices of the observation window of an h x w map (see scalekv_window_centroids).
@@ -172,6 +175,7 @@ scalekv_status make_plan(const scalekv_config *c, Plan &p, std::string &err) {
   p.off_kept = o; o = align_up(o + (size_t)p.n_slices * 4, 1024);
   p.off_hbud = o; o = align_up(o + (size_t)p.n_slices * 4, 1024);
   p.off_acc = o; o = align_up(o + 16 + (size_t)p.n_slices * 16, 1024);
+  p.off_stats = o; o = align_up(o + (size_t)kStatsMaxCtas * 64 * kStatsRec * 4, 1024);   // key-range partials of layer_stats
   p.ws_bytes = o;
   return SCALEKV_OK;
 }
@@ -908,15 +912,25 @@ scalekv_status scalekv_layer_stats_ex(scalekv_ctx *ctx, int32_t layer, scalekv_t
   double *acc = reinterpret_cast<double *>(ctx->ws + p.off_acc);
   const size_t acc_bytes = 16 + (size_t)p.n_slices * 16;
   CU(cudaMemsetAsync(acc, 0, acc_bytes, ctx->s_main));
+  // few slices and few sampled rows leave most SMs idle: split every slice's keys over enough CTAs to fill them
+  const int row_blocks = (rows + 63) / 64;
+  const int tiles = (ctx->hist[layer] + nk + 63) / 64;
+  int n_split = 1;
+  while (n_split < 16 && row_blocks * p.n_slices * n_split * 2 <= kStatsMaxCtas && n_split * 2 <= tiles) n_split *= 2;
+  float *partial = reinterpret_cast<float *>(ctx->ws + p.off_stats);
   {
     Scope sc(ctx, ctx->s_main, kOther);
-    dim3 grid((rows + 63) / 64, p.n_slices);
+    dim3 grid(row_blocks, p.n_slices, n_split);
     if (ctx->dtype == SCALEKV_BF16)
       layer_stats_kernel<__nv_bfloat16, 128><<<grid, 256, layer_stats_smem_bytes<128>(topk_prime), ctx->s_main>>>(
-          layer_view(ctx, layer), tview(Q), nk, p.N[k], query_stride, rows, topk_prime, ctx->scale, acc);
+          layer_view(ctx, layer), tview(Q), nk, p.N[k], query_stride, rows, topk_prime, ctx->scale, acc, partial);
     else
       layer_stats_kernel<float, 64><<<grid, 256, layer_stats_smem_bytes<64>(topk_prime), ctx->s_main>>>(
-          layer_view(ctx, layer), tview(Q), nk, p.N[k], query_stride, rows, topk_prime, ctx->scale, acc);
+          layer_view(ctx, layer), tview(Q), nk, p.N[k], query_stride, rows, topk_prime, ctx->scale, acc, partial);
+  }
+  if (n_split > 1) {
+    Scope sc(ctx, ctx->s_main, kOther);
+    layer_stats_merge_kernel<<<dim3(row_blocks, p.n_slices), 64, 0, ctx->s_main>>>(partial, n_split, rows, topk_prime, acc);
   }
   scalekv_status st = check_launch(ctx, "layer_stats");
   if (st != SCALEKV_OK) return st;
