@@ -942,17 +942,42 @@ __global__ void __launch_bounds__(256) layer_stats_kernel(LayerView lv, TensorVi
   const int row = tid >> 2, part = tid & 3;
   float m_run = -INFINITY, z_run = 0.f, cur_run = 0.f;
   float thr = Kp > 0 ? -INFINITY : INFINITY;           // the smallest member of this thread's list (nothing enters when K' = 0)
+  // the next key tile (and its positions) travels from global memory into registers while the current one is worked on
+  constexpr int PIECES = 64 * CH / 256;                // 16-byte pieces of a tile per thread
+  uint4 nxt[PIECES];
+  int nxt_pos = 0;
+  auto fetch = [&](int t) {
+    const int j0 = t << 6;
+#pragma unroll
+    for (int u = 0; u < PIECES; ++u) {
+      const int idx = tid + u * 256, r = idx / CH, c = idx % CH;
+      nxt[u] = make_uint4(0u, 0u, 0u, 0u);
+      if (j0 + r < L) nxt[u] = reinterpret_cast<const uint4 *>(lv.k_pool + slot_row(lv, slice, j0 + r) * lv.row_bytes)[c];
+    }
+    if (tid < 64) nxt_pos = (j0 + tid < L) ? lv.pos_pool[slot_row(lv, slice, j0 + tid)] : -1;
+  };
+  if (t_lo < t_hi) fetch(t_lo);
   for (int t = t_lo; t < t_hi; ++t) {
     const int j0 = t << 6;
     __syncthreads();
-    load_tile_rows<T, D>(Ks, LD, lv, lv.k_pool, slice, j0, L);
-    if (tid < 64) is_cur[tid] = (j0 + tid < L) ? (lv.pos_pool[slot_row(lv, slice, j0 + tid)] >= n_prev ? 1 : 0) : 0;
+#pragma unroll
+    for (int u = 0; u < PIECES; ++u) {
+      const int idx = tid + u * 256, r = idx / CH, c = idx % CH;
+      float v[VN];
+      Vec16<T>::load(reinterpret_cast<const T *>(&nxt[u]), v);
+#pragma unroll
+      for (int e = 0; e < VN; e += 4)                  // 16-byte stores (LD and VN are multiples of 4)
+        *reinterpret_cast<float4 *>(&Ks[r * LD + c * VN + e]) = make_float4(v[e], v[e + 1], v[e + 2], v[e + 3]);
+    }
+    if (tid < 64) is_cur[tid] = nxt_pos >= n_prev ? 1 : 0;
     __syncthreads();
+    if (t + 1 < t_hi) fetch(t + 1);
     float s[4][4];
 #pragma unroll
     for (int i = 0; i < 4; ++i)
 #pragma unroll
       for (int j = 0; j < 4; ++j) s[i][j] = 0.f;
+#pragma unroll 4
     for (int c = 0; c < D; c += 4) {
       float4 q[4], k[4];
 #pragma unroll
