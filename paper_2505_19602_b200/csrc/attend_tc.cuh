@@ -16,8 +16,7 @@
 //                         the two tiles' chains  S -> softmax -> PV  run concurrently, each hiding the other's
 //                         hand-over latencies.  A thread sweeps its row of an S tile once, in four chunks of 32
 //                         columns (tcgen05.ld, the next chunk in flight): p = exp2(s * c - m) against a lazy
-//                         reference m with packed f32x2 arithmetic (a share of the exponentials on the FMA
-//                         pipe), the chunk's sum, and P as bf16 pairs written over the first 64 columns of the
+//                         reference m with packed f32x2 arithmetic, the chunk's sum, and P as bf16 pairs written over the first 64 columns of the
 //                         row's S buffer (tcgen05.st; a chunk's P only covers columns already read), from
 //                         where the PV product takes its A operand.  Only when a chunk's sum shows that an
 //                         exponent left the lazy band (2^8) does the warp raise the reference: the chunk is
@@ -63,7 +62,10 @@ constexpr uint32_t kOffTmemSlot = 208;            // inside the barrier area, be
 static_assert(bCount * 8 <= kOffTmemSlot, "barriers overlap the TMEM slot");
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColS = 0, kColO = 256;       // S/P buffers at 0 and 128, O accumulators at 256 and 384
-constexpr int kPolyPairs = 1;                   // of every 4 pairs of exponentials, this many run on the FMA pipe
+// Of every 4 pairs of exponentials, this many are computed on the FMA pipe (exp2_poly_pair) instead of the MUFU.
+// 0: measured in whole passes under the power cap, every exponential on the MUFU is 2-3 % faster than one pair in
+// four on the FMA pipe (the polynomial costs seven times the instructions), although an isolated launch shows no difference.
+constexpr int kPolyPairs = 0;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
