@@ -7,9 +7,10 @@
 //                         128B-swizzled shared memory: history tiles page by page through the slice's
 //                         page table, tiles of a not yet appended current map from the caller's tensors.
 //   warp 1 (one thread) : tcgen05.mma issuer; owns the TMEM allocation (512 columns: two S/P buffers
-//                         and two O accumulators).  With two query tiles the issue order per key tile
-//                         j is  S_A(j), PV_B(j-1), S_B(j), PV_A(j): while one tile's softmax runs, the
-//                         tensor pipe works for the other tile.  With one query tile the two S buffers
+//                         and two O accumulators).  With two query tiles the issue order is
+//                         S_A(0), S_B(0), then per key tile j  PV_A(j), S_A(j+1), PV_B(j), S_B(j+1): while one
+//                         tile's softmax runs, the tensor pipe works for the other tile, and a tile's next S
+//                         product follows its PV product without a wait in between.  With one query tile the two S buffers
 //                         alternate and S(j+1) is issued ahead of PV(j).
 //   warps 4-7, 8-11     : softmax, one warpgroup per query tile (warps 4-7 tile A, warps 8-11 tile B), one
 //                         thread per query row (TMEM lane), so that no row state is shared between threads and
@@ -46,6 +47,11 @@ namespace scalekv {
 namespace tc {
 
 constexpr int kChunks = 4;                       // tcgen05.ld x32 loads per softmax thread (= query row) and S tile
+// With two query tiles a PV product is issued in two parts: the steps over the keys of the first kEarlyChunks chunks
+// as soon as their P is stored, under the sweep of the remaining chunks, and the rest when the tile's P is complete.
+// What stands between the end of a sweep and the tile's next S tile is then 2 (4 - kEarlyChunks) + 8 MMAs, not 16.
+constexpr int kEarlyChunks = 3;
+static_assert(kEarlyChunks >= 1 && kEarlyChunks < kChunks, "both parts of a PV product need at least one chunk");
 constexpr int kThreads = 128 + 2 * 128;          // warps: TMA, MMA, 2 x append, one softmax warpgroup per query tile
 constexpr int kStages = 5;                       // one ring for the K and V tiles: K_0, V_0, K_1, V_1, ...
 constexpr uint32_t kTileBytes = 128 * 128 * 2;   // one 128 x 128 bf16 operand tile
@@ -57,7 +63,7 @@ constexpr uint32_t kSmemBytes = kOffBar + 256;
 static_assert(kSmemBytes <= 232448, "more shared memory than a CTA can have");
 // barrier slots (8 bytes each): one full/empty pair per ring stage, one S/P/PV barrier per S buffer or query tile
 enum { bQFull = 0, bFull = 1, bEmpty = bFull + kStages, bSFull = bEmpty + kStages, bPFull = bSFull + 2, bPvDone = bPFull + 2,
-       bFinal = bPvDone + 2, bOut = bFinal + 2, bCount = bOut + 2 };
+       bFinal = bPvDone + 2, bOut = bFinal + 2, bPEarly = bOut + 2, bPvEarly = bPEarly + 2, bCount = bPvEarly + 2 };
 constexpr uint32_t kOffTmemSlot = 208;            // inside the barrier area, behind the barriers
 static_assert(bCount * 8 <= kOffTmemSlot, "barriers overlap the TMEM slot");
 constexpr uint32_t kTmemCols = 512;
@@ -223,6 +229,27 @@ __device__ __forceinline__ void tc_mma_ts_x8(uint32_t d_tmem, uint32_t a_tmem, u
       "n"(p_col(5)), "n"(p_col(6)), "n"(p_col(7))
       : "memory");
 }
+// The first N of the eight steps (a_tmem and b_lo address the first of them).
+template <int N>
+__device__ __forceinline__ void tc_mma_ts_n(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t hi, uint32_t idesc,
+                                            uint32_t accumulate_first) {
+  static_assert(N >= 1 && N <= 8, "one to eight steps");
+  asm volatile(
+      "{\n\t.reg .pred e, pf, pt, q;\n\t.reg .b64 db;\n\t.reg .b32 at, bl, nn;\n\t"
+      "elect.sync _|e, 0xffffffff;\n\tsetp.ne.b32 pf, %5, 0;\n\tsetp.eq.b32 pt, 0, 0;\n\tmov.u32 nn, %13;\n\t"
+      "mov.b64 db, {%2, %3};\n\t@e tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, pf;\n\t"
+      "setp.gt.and.u32 q, nn, 1, e;\n\tadd.u32 at, %1, %6;\n\tadd.u32 bl, %2, 128;\n\tmov.b64 db, {bl, %3};\n\t@q tcgen05.mma.cta_group::1.kind::f16 [%0], [at], db, %4, pt;\n\t"
+      "setp.gt.and.u32 q, nn, 2, e;\n\tadd.u32 at, %1, %7;\n\tadd.u32 bl, %2, 256;\n\tmov.b64 db, {bl, %3};\n\t@q tcgen05.mma.cta_group::1.kind::f16 [%0], [at], db, %4, pt;\n\t"
+      "setp.gt.and.u32 q, nn, 3, e;\n\tadd.u32 at, %1, %8;\n\tadd.u32 bl, %2, 384;\n\tmov.b64 db, {bl, %3};\n\t@q tcgen05.mma.cta_group::1.kind::f16 [%0], [at], db, %4, pt;\n\t"
+      "setp.gt.and.u32 q, nn, 4, e;\n\tadd.u32 at, %1, %9;\n\tadd.u32 bl, %2, 512;\n\tmov.b64 db, {bl, %3};\n\t@q tcgen05.mma.cta_group::1.kind::f16 [%0], [at], db, %4, pt;\n\t"
+      "setp.gt.and.u32 q, nn, 5, e;\n\tadd.u32 at, %1, %10;\n\tadd.u32 bl, %2, 640;\n\tmov.b64 db, {bl, %3};\n\t@q tcgen05.mma.cta_group::1.kind::f16 [%0], [at], db, %4, pt;\n\t"
+      "setp.gt.and.u32 q, nn, 6, e;\n\tadd.u32 at, %1, %11;\n\tadd.u32 bl, %2, 768;\n\tmov.b64 db, {bl, %3};\n\t@q tcgen05.mma.cta_group::1.kind::f16 [%0], [at], db, %4, pt;\n\t"
+      "setp.gt.and.u32 q, nn, 7, e;\n\tadd.u32 at, %1, %12;\n\tadd.u32 bl, %2, 896;\n\tmov.b64 db, {bl, %3};\n\t@q tcgen05.mma.cta_group::1.kind::f16 [%0], [at], db, %4, pt;\n\t"
+      "}" ::"r"(d_tmem),
+      "r"(a_tmem), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate_first), "n"(p_col(1)), "n"(p_col(2)), "n"(p_col(3)), "n"(p_col(4)),
+      "n"(p_col(5)), "n"(p_col(6)), "n"(p_col(7)), "n"(N)
+      : "memory");
+}
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -353,12 +380,14 @@ __host__ __device__ constexpr uint32_t instr_desc(bool b_mn_major) {
 // are read again; `valid` of them are real keys.  Per lane the reference moves up to the chunk's maximum if
 // that is larger (a lane that needs nothing gets the factor 1): the chunk's P is recomputed against the new
 // reference and stored, and everything accumulated under the old one is multiplied by f = 2^(old - new): the
-// running row sum, the P chunks 0 .. cc-1 already stored for this tile (16 columns each), and - once the
-// previous PV product of the tile has landed - the row's 128 columns of the O accumulator at o_addr.
+// running row sum, the P chunks p_first .. cc-1 stored for this tile that the tensor core has not been given yet
+// (16 columns each), and - once the product that `pv_bar` stands for has landed: the previous PV product of the
+// tile, or the early part of this one when its chunks have been handed over - the row's 128 columns of the O
+// accumulator at o_addr.
 // Everything goes in and out by value so that the caller's state stays in registers.
 struct Raised { float m, l, sum; int o_landed, ok; };
-__device__ __noinline__ Raised raise_reference(int valid, float c, float m, float l_run, uint32_t s_addr, int cc, uint32_t o_addr,
-                                               int with_o, int o_landed, uint32_t pv_bar, uint32_t pv_parity,
+__device__ __noinline__ Raised raise_reference(int valid, float c, float m, float l_run, uint32_t s_addr, int cc, int p_first,
+                                               uint32_t o_addr, int with_o, int o_landed, uint32_t pv_bar, uint32_t pv_parity,
                                                volatile int *abort_flag, int *status) {
   float x[32];
   tc_ld32(s_addr + cc * 32, x);
@@ -380,7 +409,7 @@ __device__ __noinline__ Raised raise_reference(int valid, float c, float m, floa
   }
   tc_st16(s_addr + cc * 16, pk);
 #pragma unroll 1
-  for (int e = 0; e < cc; ++e) {
+  for (int e = p_first; e < cc; ++e) {
     uint32_t r[16];
     tc_ld16(s_addr + e * 16, r);
     tc_wait_ld();
@@ -483,6 +512,8 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       mbar_init(bar(bSFull + s), 1);
       mbar_init(bar(bPFull + s), 4);      // one arrival per warp of the softmax warpgroup that serves the buffer
       mbar_init(bar(bPvDone + s), 1);
+      mbar_init(bar(bPEarly + s), 4);     // the same warps, once P of the tile's first kEarlyChunks chunks is stored
+      mbar_init(bar(bPvEarly + s), 1);    // the early part of a PV product has landed (only the rare path waits for it)
     }
     for (int s = 0; s < 2; ++s) mbar_init(bar(bFinal + s), 1);
     for (int s = 0; s < 2; ++s) mbar_init(bar(bOut + s), 4);
@@ -588,18 +619,61 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         return true;
       };
       if (!single) {
-        for (int j = 0; j < T && ok; ++j) {
-          ok = mbar_wait_warp(bar(bFull + (2 * j) % kStages), ((2 * j) / kStages) & 1, abort_flag, status);
-          if (!ok) break;
+        // A tile's chain is  sweep -> PV(j) -> S(j+1) -> sweep ..., so between the moment a tile's P is complete
+        // and the issue of its next S product this warp does nothing but issue: the operands of both products
+        // are waited for beforehand (they arrive long before P does), the two products go out back to back, and the
+        // commits follow them.
+        auto ring_full = [&](int t) { return mbar_wait_warp(bar(bFull + t % kStages), (t / kStages) & 1, abort_flag, status); };
+        auto mma_s = [&](int j, int qt) {
+          tc_mma_ss_x8(tmem + kColS + qt * 128, q_lo[qt], desc_lo(base + kOffRing + ((2 * j) % kStages) * kTileBytes, 16), dhi, idesc_qk);
+        };
+        constexpr int kEarlySteps = 2 * kEarlyChunks;      // a chunk of 32 keys is two steps of 16
+        auto mma_pv_early = [&](int j, int qt) {
+          tc_mma_ts_n<kEarlySteps>(tmem + kColO + qt * 128, tmem + kColS + qt * 128,
+                                   desc_lo(base + kOffRing + ((2 * j + 1) % kStages) * kTileBytes, kHalfBytes), dhi, idesc_pv,
+                                   j > 0 ? 1u : 0u);
+        };
+        auto mma_pv_rest = [&](int j, int qt) {
+          tc_mma_ts_n<8 - kEarlySteps>(tmem + kColO + qt * 128, tmem + kColS + qt * 128 + p_col(kEarlySteps),
+                                       desc_lo(base + kOffRing + ((2 * j + 1) % kStages) * kTileBytes, kHalfBytes) + 128 * kEarlySteps,
+                                       dhi, idesc_pv, 1u);
+        };
+        ok = ok && ring_full(0);
+        if (ok) {
           tc_fence_after();
-          issue_s(j, 0, 0);
-          if (j > 0) ok = issue_pv(j - 1, 1, 1, (j - 1) & 1, true);
-          if (!ok) break;
-          issue_s(j, 1, 1);
-          if (leader) tc_commit(bar(bEmpty + (2 * j) % kStages));
-          ok = issue_pv(j, 0, 0, j & 1, false);
+          mma_s(0, 0);
+          if (leader) tc_commit(bar(bSFull + 0));
+          __syncwarp();
+          mma_s(0, 1);
+          if (leader) { tc_commit(bar(bSFull + 1)); tc_commit(bar(bEmpty + 0)); }
+          __syncwarp();
         }
-        if (ok) ok = issue_pv(T - 1, 1, 1, (T - 1) & 1, true);
+        for (int j = 0; j < T && ok; ++j) {
+          const bool more = j + 1 < T;
+          ok = ring_full(2 * j + 1) && (!more || ring_full(2 * j + 2));
+          for (int qt = 0; qt < 2 && ok; ++qt) {
+            ok = mbar_wait_warp(bar(bPEarly + qt), j & 1, abort_flag, status);
+            if (!ok) break;
+            tc_fence_after();
+            mma_pv_early(j, qt);
+            if (leader) tc_commit(bar(bPvEarly + qt));
+            __syncwarp();
+            ok = mbar_wait_warp(bar(bPFull + qt), j & 1, abort_flag, status);
+            if (!ok) break;
+            tc_fence_after();
+            mma_pv_rest(j, qt);
+            if (more) mma_s(j + 1, qt);
+            if (leader) {
+              if (more) tc_commit(bar(bSFull + qt));
+              tc_commit(bar(bPvDone + qt));
+              if (qt == 1) {
+                tc_commit(bar(bEmpty + (2 * j + 1) % kStages));
+                if (more) tc_commit(bar(bEmpty + (2 * j + 2) % kStages));
+              }
+            }
+            __syncwarp();
+          }
+        }
         // one-shot barriers for the epilogue: everything issued so far has landed
         if (ok && leader) { tc_commit(bar(bFinal + 0)); tc_commit(bar(bFinal + 1)); }
       } else {
@@ -750,14 +824,26 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         unpack2(sum2b, s2, s3);
         float lt = (s0 + s1) + (s2 + s3);
         if (__any_sync(0xffffffffu, !(lt <= 8192.f))) {
-          const Raised r = raise_reference(vc, c, m, l, s_addr, cc, o_addr, j > 0 ? 1 : 0, o_landed, bar(bPvDone + qt),
-                                           (j - 1) & 1, abort_flag, status);
+          // Once the early chunks' P is with the tensor core, their product has to land before O is scaled, and only
+          // the later chunks' P is still this thread's to scale.
+          const bool late = !single && cc >= kEarlyChunks;
+          const Raised r = raise_reference(vc, c, m, l, s_addr, cc, late ? kEarlyChunks : 0, o_addr, (late || j > 0) ? 1 : 0,
+                                           late ? (o_landed == 2) : (o_landed >= 1), bar((late ? bPvEarly : bPvDone) + qt),
+                                           (late ? j : j - 1) & 1, abort_flag, status);
           ok = __all_sync(0xffffffffu, r.ok != 0);
           if (!ok) break;
-          m = r.m; l = r.l + r.sum; o_landed = r.o_landed;
+          m = r.m; l = r.l + r.sum;
+          if (r.o_landed) o_landed = late ? 2 : 1;
         } else {
           tc_st16(s_addr + cc * 16, pk);
           l += lt;
+        }
+        if (!single && cc == kEarlyChunks - 1) {
+          // P of the first chunks is complete: that part of the PV product may start under the rest of the sweep
+          tc_wait_st();
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar(bPEarly + buf));
         }
       }
       if (!ok) break;
