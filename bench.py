@@ -417,11 +417,47 @@ def run_scalekv(args):
     # compress of its last layers may still run on the side stream when the next scale-step starts)
     kv.scalekv_profile_enable(0)
     per_pass = []
+    per_scale_mode = "call by call (eager): at the small scales the host's launch rate, not the GPU, sets the time"
+    scale_graphs = None
+    if graph is not None:
+        # one CUDA graph per scale-step, captured while a pass runs (capture, then replay to execute it), each
+        # ending with a join of the side stream: what the events then bracket is GPU time
+        try:
+            kv.scalekv_reset()
+            kv.scalekv_sync()
+            scale_graphs = []
+            for k in range(wl.n_scales):
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=kv.stream_main, capture_error_mode="thread_local"):
+                    pipeline.scale_step(kv, inputs, windows, k, select=select)
+                    kv.scalekv_join()
+                with torch.cuda.stream(kv.stream_main):
+                    g.replay()
+                kv.scalekv_sync()
+                scale_graphs.append(g)
+            per_scale_mode = "one CUDA graph per scale-step, the side stream joined at every scale boundary"
+        except Exception:
+            scale_graphs = None
+            torch.cuda.synchronize()
+            kv.close()
+            kv = make_kv()
     for _ in range(args.steps):
-        marks = []
-        pipeline.run_pass(kv, inputs, windows, marks=marks, select=select)
+        if scale_graphs is None:
+            marks = []
+            pipeline.run_pass(kv, inputs, windows, marks=marks, select=select)
+        else:
+            marks = [torch.cuda.Event(enable_timing=True) for _ in range(wl.n_scales + 2)]
+            with torch.cuda.stream(kv.stream_main):
+                marks[0].record()
+            kv.scalekv_reset()
+            with torch.cuda.stream(kv.stream_main):
+                marks[1].record()
+                for k in range(wl.n_scales):
+                    scale_graphs[k].replay()
+                    marks[k + 2].record()
         kv.scalekv_sync()
         per_pass.append([marks[i].elapsed_time(marks[i + 1]) for i in range(len(marks) - 1)])
+    scale_graphs = None
     cols = list(zip(*per_pass))
     scale_flop = work["per_scale_flop"]
     per_scale = {"reset_ms_median": statistics.median(cols[0]),
@@ -429,6 +465,7 @@ def run_scalekv(args):
                                   "ms_min": min(cols[k + 1]),
                                   "attend_TFLOPps": scale_flop[k] / (statistics.median(cols[k + 1]) / 1e3) / 1e12}
                                  for k in range(wl.n_scales)],
+                 "mode": per_scale_mode,
                  "note": "CUDA events on stream_main at scale boundaries; one scale-step = append + attend + compress of "
                          "every layer at that scale; attend_TFLOPps = the scale's attention flop over the step's time"}
 

@@ -73,17 +73,43 @@ class PassInputs:
         return total
 
 
+def scale_step(kv: binding.ScaleKV, inputs: PassInputs, windows, k, compress_last=False, three_calls=False, select=None):
+    """One scale-step: append -> attend -> compress of every layer at scale k (one scalekv_step per layer, or
+    the three calls one by one with three_calls=True or a comparison policy in `select`: the same launches)."""
+    wl = inputs.wl
+    nk = wl.n_tokens[k]
+    O = inputs.O[:, :, :nk, :]
+    last = k + 1 == wl.n_scales
+    do_compress = not last or compress_last
+    wp = kv.window_array(windows[k]) if (do_compress and windows[k] is not None) else None
+    for l in range(wl.n_layers):
+        Q, K, V = inputs.data[(l, k)]
+        if select is not None:
+            kv.scalekv_append(l, k, K, V)
+            kv.scalekv_attend(l, Q, O)
+            if do_compress:
+                kv.scalekv_compress_ex(l, Q, windows[k], qw_is_full_map=True, **select)
+            continue
+        if not three_calls:
+            kv.scalekv_step(l, k, Q, K, V, O, window_pos=wp, whole_map=do_compress and wp is None)
+            continue
+        kv.scalekv_append(l, k, K, V)
+        kv.scalekv_attend(l, Q, O)
+        if do_compress:
+            if windows[k] is None:
+                kv.scalekv_compress(l, Q, None)
+            else:
+                kv.scalekv_compress(l, Q, windows[k], qw_is_full_map=True)
+
+
 def run_pass(kv: binding.ScaleKV, inputs: PassInputs, windows, compress_last=False, marks=None, three_calls=False, select=None):
-    """One pass: reset, then for every scale and layer append -> attend -> compress (one scalekv_step per
-    layer and scale, or the three calls one by one with three_calls=True: the same launches either way).
+    """One pass: reset, then scale_step for every scale.
 
     marks: a list that receives CUDA events recorded on stream_main before the reset, after it, and after
     every scale-step (2 + n_scales events), for per-scale-step latencies.
     select: options of scalekv_compress_ex (policy, pool_kernel, n_sink) for the comparison policies; the
     compress of every step then goes through that call.
     """
-    wl = inputs.wl
-
     def mark():
         if marks is not None:
             ev = torch.cuda.Event(enable_timing=True)
@@ -94,30 +120,8 @@ def run_pass(kv: binding.ScaleKV, inputs: PassInputs, windows, compress_last=Fal
     mark()
     kv.scalekv_reset()
     mark()
-    for k in range(wl.n_scales):
-        nk = wl.n_tokens[k]
-        O = inputs.O[:, :, :nk, :]
-        last = k + 1 == wl.n_scales
-        do_compress = not last or compress_last
-        wp = kv.window_array(windows[k]) if (do_compress and windows[k] is not None) else None
-        for l in range(wl.n_layers):
-            Q, K, V = inputs.data[(l, k)]
-            if select is not None:
-                kv.scalekv_append(l, k, K, V)
-                kv.scalekv_attend(l, Q, O)
-                if do_compress:
-                    kv.scalekv_compress_ex(l, Q, windows[k], qw_is_full_map=True, **select)
-                continue
-            if not three_calls:
-                kv.scalekv_step(l, k, Q, K, V, O, window_pos=wp, whole_map=do_compress and wp is None)
-                continue
-            kv.scalekv_append(l, k, K, V)
-            kv.scalekv_attend(l, Q, O)
-            if not last or compress_last:
-                if windows[k] is None:
-                    kv.scalekv_compress(l, Q, None)
-                else:
-                    kv.scalekv_compress(l, Q, windows[k], qw_is_full_map=True)
+    for k in range(inputs.wl.n_scales):
+        scale_step(kv, inputs, windows, k, compress_last=compress_last, three_calls=three_calls, select=select)
         mark()
 
 
