@@ -66,6 +66,7 @@ enum { bQFull = 0, bFull = 1, bEmpty = bFull + kStages, bSFull = bEmpty + kStage
        bFinal = bPvDone + 2, bOut = bFinal + 2, bPEarly = bOut + 2, bPvEarly = bPEarly + 2, bCount = bPvEarly + 2 };
 constexpr uint32_t kOffTmemSlot = 208;            // inside the barrier area, behind the barriers
 static_assert(bCount * 8 <= kOffTmemSlot, "barriers overlap the TMEM slot");
+static_assert(bCount <= 32, "one lane of the first warp initialises each barrier");
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColS = 0, kColO = 256;       // S/P buffers at 0 and 128, O accumulators at 256 and 384
 // Of every 4 pairs of exponentials, this many are computed on the FMA pipe (exp2_poly_pair) instead of the MUFU.
@@ -488,53 +489,51 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     return rest < 128 ? rest : 128;
   };
   int *status = lv.status;
-  {
-    // One thread decides for the whole CTA whether it runs at all (the status word may change between two
-    // threads' reads, and a CTA of which only a part left would go on with barriers and TMEM nobody set up):
-    // an earlier CTA gave up - do not pile on; swizzled tiles need the alignment, and a slice must not outgrow
-    // its page table - report, do not fault.
-    int leave = 0;
-    if (tid == 0) {
+  // Set-up, one rendezvous for everything.  Warp 0: its first lane decides for the whole CTA whether it runs at all
+  // (one thread, because the status word may change between two threads' reads, and a CTA of which only a part
+  // left would go on with barriers and TMEM nobody set up): an earlier CTA gave up - do not pile on; swizzled
+  // tiles need the alignment, and a slice must not outgrow its page table - report, do not fault.  Meanwhile the
+  // warp's lanes initialise one barrier each.  Warp 1 allocates the TMEM.  Everybody but warp 0 then waits on a
+  // named barrier for the barriers, the decision and the allocation; warp 0 (the TMA producer) needs neither the
+  // TMEM address nor anybody else: it only announces its part and goes on to issue the first loads while the
+  // allocation is still under way.
+  volatile int *leave_slot = reinterpret_cast<volatile int *>(base_ptr + kOffBar + kOffTmemSlot + 8);
+  int leave = 0;
+  if (warp == 0) {
+    if (lane == 0) {
       if (*reinterpret_cast<volatile int *>(status) != 0) leave = 1;
       else if ((base & 1023u) || L > (lv.pages_per_slice << lv.page_shift)) { atomicExch(status, kDevCheck); leave = 1; }
+      *abort_flag = 0;
+      *leave_slot = leave;
     }
-    if (__syncthreads_or(leave)) return;
-  }
-
-  if (tid == 0) {
-    *abort_flag = 0;
-    mbar_init(bar(bQFull), 1);
-    for (int s = 0; s < kStages; ++s) {
-      mbar_init(bar(bFull + s), 1);
-      mbar_init(bar(bEmpty + s), 3);      // the MMA warp's commit and the two append warps
+    if (lane < bCount) {
+      // arrivals per phase: a ring stage is released by the MMA warp's commit and the two append warps; P, early P and
+      // the staged output tile are announced by one lane of each of the four warps of a softmax warpgroup
+      const bool four = (lane >= bPFull && lane < bPFull + 2) || (lane >= bPEarly && lane < bPEarly + 2) ||
+                        (lane >= bOut && lane < bOut + 2);
+      const bool three = lane >= bEmpty && lane < bEmpty + kStages;
+      mbar_init(bar(lane), four ? 4u : (three ? 3u : 1u));
     }
-    for (int s = 0; s < 2; ++s) {
-      mbar_init(bar(bSFull + s), 1);
-      mbar_init(bar(bPFull + s), 4);      // one arrival per warp of the softmax warpgroup that serves the buffer
-      mbar_init(bar(bPvDone + s), 1);
-      mbar_init(bar(bPEarly + s), 4);     // the same warps, once P of the tile's first kEarlyChunks chunks is stored
-      mbar_init(bar(bPvEarly + s), 1);    // the early part of a PV product has landed (only the rare path waits for it)
-    }
-    for (int s = 0; s < 2; ++s) mbar_init(bar(bFinal + s), 1);
-    for (int s = 0; s < 2; ++s) mbar_init(bar(bOut + s), 4);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(base + kOffBar + kOffTmemSlot), "r"(kTmemCols)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-  }
-  // Everybody but the TMA warp waits here for the barriers (initialised by that warp's first thread) and for the
-  // TMEM allocation.  The TMA warp needs neither the TMEM address nor anybody else: it only announces that the
-  // barriers are ready and goes on to issue the first loads while the allocation is still under way.
-  tc_fence_before();
-  if (warp == 0) {
+    leave = __shfl_sync(0xffffffffu, leave, 0);
     __syncwarp();
+    __threadfence_block();
     asm volatile("bar.arrive 1, %0;" ::"n"(kThreads) : "memory");
   } else {
+    if (warp == 1) {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(base + kOffBar + kOffTmemSlot), "r"(kTmemCols)
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
     asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory");
+    tc_fence_after();
+    leave = *leave_slot;
   }
-  tc_fence_after();
+  if (leave) {
+    if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(*tmem_slot), "r"(kTmemCols) : "memory");
+    return;
+  }
   const uint32_t tmem = warp == 0 ? 0u : *tmem_slot;
 
   if (warp < 4) {
@@ -664,7 +663,9 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             mma_pv_rest(j, qt);
             if (more) mma_s(j + 1, qt);
             if (leader) {
-              if (more) tc_commit(bar(bSFull + qt));
+              // after the last key tile the tile's one-shot barrier for the epilogue instead of an S barrier:
+              // tile A normalises and stores its rows while tile B is still in its last sweep
+              tc_commit(bar((more ? bSFull : bFinal) + qt));
               tc_commit(bar(bPvDone + qt));
               if (qt == 1) {
                 tc_commit(bar(bEmpty + (2 * j + 1) % kStages));
@@ -674,8 +675,6 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             __syncwarp();
           }
         }
-        // one-shot barriers for the epilogue: everything issued so far has landed
-        if (ok && leader) { tc_commit(bar(bFinal + 0)); tc_commit(bar(bFinal + 1)); }
       } else {
         for (int j = 0; j < T && ok; ++j) {
           ok = mbar_wait_warp(bar(bFull + (2 * j) % kStages), ((2 * j) / kStages) & 1, abort_flag, status);
