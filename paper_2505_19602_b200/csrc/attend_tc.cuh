@@ -476,6 +476,28 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   const int n_k = prm.n_k;
   const int q_first = blockIdx.x * 256;                  // first query row of tile A
   const bool single = q_first + 128 >= n_k;              // tile B would be empty
+  // What needs no global memory comes first: the lanes of warp 0 initialise one barrier each, warp 1 allocates the
+  // TMEM.  When the launch allows it (programmatic stream serialisation) this part runs while the kernel before this
+  // one in the stream is still finishing; `griddepcontrol.wait` then holds every thread until that kernel's writes
+  // - cache lengths, page tables, pages, the status word - are visible.  The grid behind this one may come up as
+  // soon as all of this grid's CTAs are running.
+  if (warp == 0) {
+    if (lane < bCount) {
+      // arrivals per phase: a ring stage is released by the MMA warp's commit and the two append warps; P, early P and
+      // the staged output tile are announced by one lane of each of the four warps of a softmax warpgroup
+      const bool four = (lane >= bPFull && lane < bPFull + 2) || (lane >= bPEarly && lane < bPEarly + 2) ||
+                        (lane >= bOut && lane < bOut + 2);
+      const bool three = lane >= bEmpty && lane < bEmpty + kStages;
+      mbar_init(bar(lane), four ? 4u : (three ? 3u : 1u));
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  } else if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(base + kOffBar + kOffTmemSlot), "r"(kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const int hist = lv.hist_len[slice];
   const int L = hist + n_k;
   // key tiles: Th from the pages (all of them unless the current map still waits in the caller's
@@ -506,25 +528,11 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       *abort_flag = 0;
       *leave_slot = leave;
     }
-    if (lane < bCount) {
-      // arrivals per phase: a ring stage is released by the MMA warp's commit and the two append warps; P, early P and
-      // the staged output tile are announced by one lane of each of the four warps of a softmax warpgroup
-      const bool four = (lane >= bPFull && lane < bPFull + 2) || (lane >= bPEarly && lane < bPEarly + 2) ||
-                        (lane >= bOut && lane < bOut + 2);
-      const bool three = lane >= bEmpty && lane < bEmpty + kStages;
-      mbar_init(bar(lane), four ? 4u : (three ? 3u : 1u));
-    }
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     leave = __shfl_sync(0xffffffffu, leave, 0);
     __syncwarp();
     __threadfence_block();
     asm volatile("bar.arrive 1, %0;" ::"n"(kThreads) : "memory");
   } else {
-    if (warp == 1) {
-      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(base + kOffBar + kOffTmemSlot), "r"(kTmemCols)
-                   : "memory");
-      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
     tc_fence_before();
     asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory");
     tc_fence_after();
@@ -993,7 +1001,21 @@ struct AttendTc {
     prm.w = win_logits ? w : 0;
     for (int e = 0; e < kMaxWindow; ++e) prm.win_pos[e] = (win_logits && e < w) ? win_pos[e] : -1;
     dim3 grid((n_k + 255) / 256, lv.n_slices);
-    tc::attend_tc_kernel<<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(tmQ, tmK, tmV, tmKc, tmVc, tmO, prm);
+    // programmatic stream serialisation: the kernel's set-up may overlap the end of the kernel before it in the stream
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(tc::kThreads);
+    cfg.dynamicSmemBytes = tc::kSmemBytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, tc::attend_tc_kernel, tmQ, tmK, tmV, tmKc, tmVc, tmO, prm) != cudaSuccess) {
+      err = "attend: kernel launch failed";
+      return false;
+    }
     return true;
   }
 };
