@@ -16,13 +16,14 @@
 //                         thread per query row (TMEM lane), so that no row state is shared between threads and
 //                         the two tiles' chains  S -> softmax -> PV  run concurrently, each hiding the other's
 //                         hand-over latencies.  A thread sweeps its row of an S tile once, in four chunks of 32
-//                         columns (tcgen05.ld, the next chunk in flight): p = exp2(s * c - m) against a lazy
-//                         reference m with packed f32x2 arithmetic, the chunk's sum, and P as bf16 pairs written over the first 64 columns of the
-//                         row's S buffer (tcgen05.st; a chunk's P only covers columns already read), from
-//                         where the PV product takes its A operand.  Only when a chunk's sum shows that an
-//                         exponent left the lazy band (2^8) does the warp raise the reference: the chunk is
-//                         recomputed, the P chunks already stored for this tile, the running sum and the O
-//                         accumulator are scaled down.  Threads that own a row of the observation window also
+//                         columns (tcgen05.ld), software-pipelined: p = exp2(s * c - m) of chunk cc + 1 against
+//                         a lazy reference m (packed f32x2 arithmetic, in place) is issued before chunk cc is
+//                         summed, checked and written as bf16 pairs over the first 64 columns of the row's S
+//                         buffer (tcgen05.st; a chunk's P only covers columns already read), from where the PV
+//                         product takes its A operand.  Only when a chunk's sum shows that an exponent left
+//                         the lazy band (2^8) does the warp raise the reference: the chunk is recomputed, the
+//                         P chunks already stored for this tile, the running sum and the O accumulator are
+//                         scaled down, and the exponentials taken ahead for the next chunk are taken again.  Threads that own a row of the observation window also
 //                         store that row's raw products (16-byte stores, key tile j in columns 128 j ..) for
 //                         the compress that follows.  At the end each warpgroup normalises its O tile, stages
 //                         it in the query tile's shared memory and one thread sends it out with TMA stores.
@@ -39,6 +40,7 @@
 #include <cuda_runtime.h>
 
 #include <cstdlib>
+#include <type_traits>
 #include <string>
 
 #include "common.cuh"
@@ -69,10 +71,6 @@ static_assert(bCount * 8 <= kOffTmemSlot, "barriers overlap the TMEM slot");
 static_assert(bCount <= 32, "one lane of the first warp initialises each barrier");
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColS = 0, kColO = 256;       // S/P buffers at 0 and 128, O accumulators at 256 and 384
-// Of every 4 pairs of exponentials, this many are computed on the FMA pipe (exp2_poly_pair) instead of the MUFU.
-// 0: measured in whole passes under the power cap, every exponential on the MUFU is 2-3 % faster than one pair in
-// four on the FMA pipe (the polynomial costs seven times the instructions), although an isolated launch shows no difference.
-constexpr int kPolyPairs = 0;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -337,26 +335,6 @@ __device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
   uint64_t d;
   asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
   return d;
-}
-
-// 2^x for a pair of exponents on the FMA pipe instead of the transcendental unit: x = n + f with
-// n = round(x) (magic-number rounding) and f in [-0.5, 0.5], 2^f by a cubic fitted for minimal relative
-// error (7.5e-5, far below the bf16 rounding of P), 2^n by adding n to the exponent field.
-// x is clamped to [-126, 127]: below, the result is smaller than every normal number; above, the
-// exponent field would wrap (the caller's overflow check sees 2^127).
-__device__ __forceinline__ void exp2_poly_pair(float x0, float x1, float &p0, float &p1) {
-  const uint64_t x = pack2(fminf(fmaxf(x0, -126.f), 127.f), fminf(fmaxf(x1, -126.f), 127.f));
-  const uint64_t t = add2(x, pack2(12582912.f, 12582912.f));            // 1.5 * 2^23: integer part lands in the mantissa
-  const uint64_t n = add2(t, pack2(-12582912.f, -12582912.f));
-  const uint64_t f = fma2(n, pack2(-1.f, -1.f), x);
-  uint64_t q = fma2(f, pack2(0.05517147481441498f, 0.05517147481441498f), pack2(0.242610901594162f, 0.242610901594162f));
-  q = fma2(q, f, pack2(0.6932609677314758f, 0.6932609677314758f));
-  q = fma2(q, f, pack2(0.9999281167984009f, 0.9999281167984009f));
-  float t0, t1, q0, q1;
-  unpack2(t, t0, t1);
-  unpack2(q, q0, q1);
-  p0 = __uint_as_float(__float_as_uint(q0) + (__float_as_uint(t0) << 23));
-  p1 = __uint_as_float(__float_as_uint(q1) + (__float_as_uint(t1) << 23));
 }
 
 // Shared-memory matrix descriptor, 128-byte swizzle, operand tiles whose 8-row groups are 1024 B
@@ -746,6 +724,8 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         if (prm.win_pos[e] == qi) wrank = e;
       wwarp = __any_sync(0xffffffffu, wrank >= 0);
     }
+    // (the window row's address is taken once: inside the sweep it would cost 64-bit arithmetic in every chunk)
+    float *win_row = wrank >= 0 ? prm.win_logits + ((size_t)slice * prm.w + wrank) * prm.ld_l : nullptr;
     const uint32_t o_addr = lane_addr + kColO + qt * 128;
     bool ok = true;
     for (int j = 0; j < T && ok && active; ++j) {
@@ -757,79 +737,79 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       const uint32_t s_addr = lane_addr + kColS + buf * 128;
       const int valid = tile_valid(j);           // < 128 only in a ragged tile
       int o_landed = 0;                          // the previous PV product of this tile has been waited for
+      // The sweep is software-pipelined over the chunks: while chunk cc is summed, packed, checked and stored
+      // ("back"), the exponentials of chunk cc + 1 ("front": x = s c - m and 2^x, in place in the chunk's registers)
+      // are already issued, against the reference as it stands.  They are independent of chunk cc's check, so the
+      // transcendental unit stays busy across the vote and the stores; in the rare case that the check raises the
+      // reference, chunk cc + 1 is read again and redone.
       float v[2][32];
-      tc_ld32(s_addr, v[0]);
+      auto log_window = [&](const float *x, int cc) {
+        // The row's raw products go out as they are (the score kernel applies the softmax scale), 32
+        // columns as eight 16-byte stores, at column 128 j + ...: key tile j owns columns [128 j, 128 j + 128)
+        // of a logit row, so the current map starts at the next multiple of 128 behind the history and
+        // every store is aligned.  Columns of a ragged tile beyond its keys hold finite values nobody reads.
+        if (wrank >= 0) {
+          float4 *dst = reinterpret_cast<float4 *>(win_row + (j * 128 + cc * 32));
 #pragma unroll
-      for (int cc = 0; cc < kChunks; ++cc) {
-        tc_wait_ld();
-        if (cc + 1 < kChunks) tc_ld32(s_addr + (cc + 1) * 32, v[(cc + 1) & 1]);
-        float *x = v[cc & 1];
-        if (wwarp) {
-          if (wrank >= 0) {
-            // The row's raw products go out as they are (the score kernel applies the softmax scale), 32
-            // columns as eight 16-byte stores, at column 128 j + ...: key tile j owns columns [128 j, 128 j + 128)
-            // of a logit row, so the current map starts at the next multiple of 128 behind the history and
-            // every store is aligned.  Columns of a ragged tile beyond its keys hold finite values nobody reads.
-            const int col0 = j * 128 + cc * 32;
-            float4 *dst = reinterpret_cast<float4 *>(prm.win_logits + ((size_t)slice * prm.w + wrank) * prm.ld_l + col0);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) dst[i] = make_float4(x[4 * i], x[4 * i + 1], x[4 * i + 2], x[4 * i + 3]);
-          }
-          __syncwarp();   // the tcgen05 instructions that follow want the warp converged
+          for (int i = 0; i < 8; ++i) dst[i] = make_float4(x[4 * i], x[4 * i + 1], x[4 * i + 2], x[4 * i + 3]);
         }
-        if (j == 0 && cc == 0) {
-          // no reference yet: the largest of the row's first 32 products serves (column 0 of the first tile
-          // always holds a key, so it is finite); a later chunk that exceeds the band raises it like any other
-          float mt = -INFINITY;
-#pragma unroll
-          for (int i = 0; i < 32; i += 2) {
-            const float e0 = (i < valid) ? x[i] : -INFINITY;
-            const float e1 = (i + 1 < valid) ? x[i + 1] : -INFINITY;
-            mt = max3(mt, e0, e1);
-          }
-          m = mt * c;
-        }
-        // x = s * c - m, p = exp2(x), the chunk's sum.  32 values of at most 2^8 sum to at most 2^13; a larger,
-        // infinite or NaN sum means that some x exceeded 8.
+        __syncwarp();   // the tcgen05 instructions that follow want the warp converged
+      };
+      // (masked: a ragged tile, whose columns beyond the last key must not count)
+      auto front = [&](float *x, int vc, auto masked) {      // vc: real keys in this chunk (>= 32: all)
         const uint64_t negm2 = pack2(-m, -m);
-        uint64_t sum2a = pack2(0.f, 0.f), sum2b = sum2a;
-        uint32_t pk[16];
-        const int vc = valid - cc * 32;          // real keys in this chunk (>= 32: all)
 #pragma unroll
-        for (int i = 0; i < 16; i += 4) {
-          float a0, a1, a2, a3, a4, a5, a6, a7;
-          unpack2(fma2(pack2(x[2 * i + 0], x[2 * i + 1]), c2, negm2), a0, a1);
-          unpack2(fma2(pack2(x[2 * i + 2], x[2 * i + 3]), c2, negm2), a2, a3);
-          unpack2(fma2(pack2(x[2 * i + 4], x[2 * i + 5]), c2, negm2), a4, a5);
-          unpack2(fma2(pack2(x[2 * i + 6], x[2 * i + 7]), c2, negm2), a6, a7);
-          if (vc < 32) {
-            if (2 * i + 0 >= vc) a0 = -INFINITY;
+        for (int i = 0; i < 16; ++i) {
+          float a0, a1;
+          unpack2(fma2(pack2(x[2 * i], x[2 * i + 1]), c2, negm2), a0, a1);
+          if constexpr (decltype(masked)::value) {
+            if (2 * i >= vc) a0 = -INFINITY;
             if (2 * i + 1 >= vc) a1 = -INFINITY;
-            if (2 * i + 2 >= vc) a2 = -INFINITY;
-            if (2 * i + 3 >= vc) a3 = -INFINITY;
-            if (2 * i + 4 >= vc) a4 = -INFINITY;
-            if (2 * i + 5 >= vc) a5 = -INFINITY;
-            if (2 * i + 6 >= vc) a6 = -INFINITY;
-            if (2 * i + 7 >= vc) a7 = -INFINITY;
           }
-          float p0, p1, p2, p3, p4, p5, p6, p7;
-          if (kPolyPairs > 0) exp2_poly_pair(a0, a1, p0, p1); else { p0 = ex2(a0); p1 = ex2(a1); }
-          if (kPolyPairs > 1) exp2_poly_pair(a2, a3, p2, p3); else { p2 = ex2(a2); p3 = ex2(a3); }
-          if (kPolyPairs > 2) exp2_poly_pair(a4, a5, p4, p5); else { p4 = ex2(a4); p5 = ex2(a5); }
-          if (kPolyPairs > 3) exp2_poly_pair(a6, a7, p6, p7); else { p6 = ex2(a6); p7 = ex2(a7); }
-          sum2a = add2(sum2a, pack2(p0, p1));
-          sum2b = add2(sum2b, pack2(p2, p3));
-          sum2a = add2(sum2a, pack2(p4, p5));
-          sum2b = add2(sum2b, pack2(p6, p7));
-          pk[i + 0] = pack_bf16(p0, p1);
-          pk[i + 1] = pack_bf16(p2, p3);
-          pk[i + 2] = pack_bf16(p4, p5);
-          pk[i + 3] = pack_bf16(p6, p7);
+          x[2 * i] = ex2(a0);
+          x[2 * i + 1] = ex2(a1);
+        }
+      };
+      // 32 values of at most 2^8 sum to at most 2^13; a larger, infinite or NaN sum means that some x exceeded 8.
+      auto back = [&](const float *pv, uint32_t *pk) -> float {
+        uint64_t sum2a = pack2(0.f, 0.f), sum2b = sum2a;
+#pragma unroll
+        for (int i = 0; i < 16; i += 2) {
+          sum2a = add2(sum2a, pack2(pv[2 * i], pv[2 * i + 1]));
+          sum2b = add2(sum2b, pack2(pv[2 * i + 2], pv[2 * i + 3]));
+          pk[i] = pack_bf16(pv[2 * i], pv[2 * i + 1]);
+          pk[i + 1] = pack_bf16(pv[2 * i + 2], pv[2 * i + 3]);
         }
         float s0, s1, s2, s3;
         unpack2(sum2a, s0, s1);
         unpack2(sum2b, s2, s3);
-        float lt = (s0 + s1) + (s2 + s3);
+        return (s0 + s1) + (s2 + s3);
+      };
+      auto sweep = [&](auto masked) {
+      tc_ld32(s_addr, v[0]);
+      tc_ld32(s_addr + 32, v[1]);
+      tc_wait_ld();
+      if (wwarp) { log_window(v[0], 0); log_window(v[1], 1); }
+      if (j == 0) {
+        // no reference yet: the largest of the row's first 32 products serves (column 0 of the first tile
+        // always holds a key, so it is finite); a later chunk that exceeds the band raises it like any other
+        float mt = -INFINITY;
+#pragma unroll
+        for (int i = 0; i < 32; i += 2) {
+          const float e0 = (i < valid) ? v[0][i] : -INFINITY;
+          const float e1 = (i + 1 < valid) ? v[0][i + 1] : -INFINITY;
+          mt = max3(mt, e0, e1);
+        }
+        m = mt * c;
+      }
+      front(v[0], valid, masked);
+#pragma unroll
+      for (int cc = 0; cc < kChunks; ++cc) {
+        uint32_t pk[16];
+        const int vc = valid - cc * 32;
+        if (cc + 1 < kChunks) front(v[(cc + 1) & 1], vc - 32, masked);
+        const float lt = back(v[cc & 1], pk);
+        if (cc + 2 < kChunks) tc_ld32(s_addr + (cc + 2) * 32, v[cc & 1]);
         if (__any_sync(0xffffffffu, !(lt <= 8192.f))) {
           // Once the early chunks' P is with the tensor core, their product has to land before O is scaled, and only
           // the later chunks' P is still this thread's to scale.
@@ -838,9 +818,15 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                                            late ? (o_landed == 2) : (o_landed >= 1), bar((late ? bPvEarly : bPvDone) + qt),
                                            (late ? j : j - 1) & 1, abort_flag, status);
           ok = __all_sync(0xffffffffu, r.ok != 0);
-          if (!ok) break;
+          if (!ok) return;
           m = r.m; l = r.l + r.sum;
           if (r.o_landed) o_landed = late ? 2 : 1;
+          if (cc + 1 < kChunks) {
+            // the next chunk's exponentials were taken against the old reference: once more, from its raw products
+            tc_ld32(s_addr + (cc + 1) * 32, v[(cc + 1) & 1]);
+            tc_wait_ld();
+            front(v[(cc + 1) & 1], vc - 32, masked);
+          }
         } else {
           tc_st16(s_addr + cc * 16, pk);
           l += lt;
@@ -852,7 +838,13 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           __syncwarp();
           if (lane == 0) mbar_arrive(bar(bPEarly + buf));
         }
+        if (cc + 2 < kChunks) {
+          tc_wait_ld();
+          if (wwarp) log_window(v[cc & 1], cc + 2);
+        }
       }
+      };
+      if (valid < 128) sweep(std::true_type{}); else sweep(std::false_type{});
       if (!ok) break;
       tc_wait_st();
       tc_fence_before();
