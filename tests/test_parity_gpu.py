@@ -912,7 +912,7 @@ def test_one_call_step_equals_the_three_calls():
 @pytest.mark.parametrize("amp", [6.0, 12.0])
 def test_dominant_keys_anywhere_in_the_first_tiles(amp):
     """Rows whose logit towards one key is 70 or 140 nats above the rest, that key sitting in the first
-    columns of the first key tile, further inside it, in its second half, or in later tiles: whatever
+    columns of the first key tile, further inside it, in its second half, or in later tiles (a ragged one among them): whatever
     the kernel took as its first reference, the output is that key's value row (the second amplitude
     is beyond what exp2 can hold against a low reference)."""
     sides = (4, 20)
@@ -921,7 +921,8 @@ def test_dominant_keys_anywhere_in_the_first_tiles(amp):
     budgets = [[binding.KEEP_ALL] * 2]
     kv = binding.ScaleKV(1, 1, 2, d, "bf16", sides, sides, budgets, max_window=16)
     gen = torch.Generator().manual_seed(123)
-    hot_slots = [5, 40, 70, 100, 130, 300]            # cache slots: 5 lies in the first map, the others in the second
+    # cache slots: 5 lies in the first map, the others in the second; 405 in its ragged last key tile (16 keys)
+    hot_slots = [5, 40, 70, 100, 130, 300, 405]
     dirs = torch.randn(len(hot_slots), d, generator=gen)
     dirs = dirs / dirs.norm(dim=1, keepdim=True) * (d ** 0.5)      # |u|^2 = d: logit of a * u against u is a * sqrt(d)
 
