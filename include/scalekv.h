@@ -77,6 +77,9 @@ typedef struct {
                                  /* map (scalekv_window_centroids) while it computes them anyway, and a */
                                  /* scalekv_compress called with exactly that window scores the cache   */
                                  /* from them instead of reading K again.  Any other window still works.*/
+                                 /* Nothing is recorded at the last scale of the schedule (nothing is      */
+                                 /* generated after it, so the method prunes nothing there) nor by a        */
+                                 /* scalekv_step that names no window: a compress then scores from K.       */
   int32_t window_kind;           /* which rows window_patches = N stands for: SCALEKV_WINDOW_CENTROIDS (0, the   */
                                  /* paper's patch centroids) or SCALEKV_WINDOW_LAST (the last N rows of the map */
                                  /* in raster order, scalekv_window_last - the SnapKV-like comparison rule)     */

@@ -435,6 +435,9 @@ struct Params {
   int win_pos[kMaxWindow];   // ascending raster indices of the window rows inside the current map
 };
 
+// kWindow: the launch records the observation window's logits; the instance without that code serves the launches
+// that record nothing (its mere presence costs every warp's sweep 2-3 %).
+template <bool kWindow>
 __global__ void __launch_bounds__(kThreads, 1)
 attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                  const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmKc,
@@ -718,7 +721,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     // window row of this thread (rank in the window, or -1) and whether its warp has any
     int wrank = -1;
     bool wwarp = false;
-    if (prm.win_logits != nullptr && active) {
+    if (kWindow && prm.win_logits != nullptr && active) {
       const int qi = q_first + qt * 128 + row;
       for (int e = 0; e < prm.w; ++e)
         if (prm.win_pos[e] == qi) wrank = e;
@@ -789,7 +792,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       tc_ld32(s_addr, v[0]);
       tc_ld32(s_addr + 32, v[1]);
       tc_wait_ld();
-      if (wwarp) { log_window(v[0], 0); log_window(v[1], 1); }
+      if (kWindow && wwarp) { log_window(v[0], 0); log_window(v[1], 1); }
       if (j == 0) {
         // no reference yet: the largest of the row's first 32 products serves (column 0 of the first tile
         // always holds a key, so it is finite); a later chunk that exceeds the band raises it like any other
@@ -840,7 +843,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         }
         if (cc + 2 < kChunks) {
           tc_wait_ld();
-          if (wwarp) log_window(v[cc & 1], cc + 2);
+          if (kWindow && wwarp) log_window(v[cc & 1], cc + 2);
         }
       }
       };
@@ -897,7 +900,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         __syncwarp();
       }
       if (prm.lse != nullptr && qi < n_k) prm.lse[(size_t)slice * n_k + qi] = (m + log2f(l)) * 0.6931471805599453f;
-      if (wrank >= 0) prm.win_lse[(size_t)slice * prm.w + wrank] = m + log2f(l);
+      if (kWindow && wrank >= 0) prm.win_lse[(size_t)slice * prm.w + wrank] = m + log2f(l);
     }
     if (quarter == 0) tma_store_wait_read();   // (a lane that issued nothing has nothing to wait for)
     tc_fence_before();
@@ -942,7 +945,8 @@ struct AttendTc {
                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
       if (r != CUDA_SUCCESS) { err = "cuTensorMapEncodeTiled(pool) failed with code " + std::to_string((int)r); return false; }
     }
-    if (cudaFuncSetAttribute(tc::attend_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc::kSmemBytes) != cudaSuccess) {
+    if (cudaFuncSetAttribute(tc::attend_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc::kSmemBytes) != cudaSuccess ||
+        cudaFuncSetAttribute(tc::attend_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc::kSmemBytes) != cudaSuccess) {
       err = "cannot raise the dynamic shared memory limit";
       return false;
     }
@@ -1004,7 +1008,9 @@ struct AttendTc {
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, tc::attend_tc_kernel, tmQ, tmK, tmV, tmKc, tmVc, tmO, prm) != cudaSuccess) {
+    const cudaError_t launched = win_logits ? cudaLaunchKernelEx(&cfg, tc::attend_tc_kernel<true>, tmQ, tmK, tmV, tmKc, tmVc, tmO, prm)
+                                            : cudaLaunchKernelEx(&cfg, tc::attend_tc_kernel<false>, tmQ, tmK, tmV, tmKc, tmVc, tmO, prm);
+    if (launched != cudaSuccess) {
       err = "attend: kernel launch failed";
       return false;
     }

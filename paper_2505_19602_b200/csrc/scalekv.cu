@@ -602,7 +602,12 @@ scalekv_status scalekv_append(scalekv_ctx *ctx, int32_t layer, int32_t scale, sc
   return check_launch(ctx, "append");
 }
 
-scalekv_status scalekv_attend(scalekv_ctx *ctx, int32_t layer, scalekv_tensor Q, scalekv_tensor O, float *lse) {
+// record: whether the kernel should also record the logits of the scale's planned observation window for a compress
+// that follows.  Recording costs the kernel 3-13 % (the threads that own window rows store 512 bytes per key tile and
+// their tile waits for them), so it is left out where no compress can use it: after the last scale of the schedule
+// (Sec. 3.3: nothing is generated after it, so the method prunes nothing there; a compress called all the same takes
+// its logits from K) and in a one-call step that names no window.
+static scalekv_status attend_impl(scalekv_ctx *ctx, int32_t layer, scalekv_tensor Q, scalekv_tensor O, float *lse, bool record) {
   if (!ctx) return SCALEKV_ERR_INVALID_ARG;
   const Plan &p = ctx->plan;
   if (layer < 0 || layer >= p.n_layers) return fail(ctx, SCALEKV_ERR_INVALID_ARG, "layer %d out of range", layer);
@@ -623,7 +628,9 @@ scalekv_status scalekv_attend(scalekv_ctx *ctx, int32_t layer, scalekv_tensor Q,
       if (fused) { kc = tview(ctx->pend_k[layer]); vc = tview(ctx->pend_v[layer]); }
       const int k = ctx->next_scale[layer] - 1;
       const std::vector<int> &win = p.windows[k];
-      float *wl = win.empty() ? nullptr : reinterpret_cast<float *>(ctx->ws + p.off_logits) + (size_t)(layer % kSets) * p.logits_elems;
+      float *wl = (win.empty() || !record || k + 1 == p.K)
+                      ? nullptr
+                      : reinterpret_cast<float *>(ctx->ws + p.off_logits) + (size_t)(layer % kSets) * p.logits_elems;
       float *wlse = reinterpret_cast<float *>(ctx->ws + p.off_wlse) + (size_t)(layer % kSets) * p.n_slices * p.max_window;
       if (!ctx->tc.launch(lv, tview(Q), tview(O), lse, nk, fused ? &kc : nullptr, fused ? &vc : nullptr, p.N[k], ctx->scale, wl,
                           wlse, p.ld_l, win.data(), (int)win.size(), ctx->s_main, e))
@@ -644,6 +651,10 @@ scalekv_status scalekv_attend(scalekv_ctx *ctx, int32_t layer, scalekv_tensor Q,
   ctx->attended[layer] = 1;
   if (ctx->s_side != ctx->s_main) CU(cudaEventRecord(ctx->ev_attend[layer], ctx->s_main));
   return check_launch(ctx, "attend");
+}
+
+scalekv_status scalekv_attend(scalekv_ctx *ctx, int32_t layer, scalekv_tensor Q, scalekv_tensor O, float *lse) {
+  return attend_impl(ctx, layer, Q, O, lse, true);
 }
 
 scalekv_status scalekv_compress(scalekv_ctx *ctx, int32_t layer, scalekv_tensor Qw, int32_t w, const int32_t *window_pos,
@@ -882,7 +893,7 @@ scalekv_status scalekv_step(scalekv_ctx *ctx, int32_t layer, int32_t scale, scal
                             scalekv_tensor O, float *lse, int32_t w, const int32_t *window_pos) {
   scalekv_status st = scalekv_append(ctx, layer, scale, K, V);
   if (st != SCALEKV_OK) return st;
-  st = scalekv_attend(ctx, layer, Q, O, lse);
+  st = attend_impl(ctx, layer, Q, O, lse, w > 0);
   if (st != SCALEKV_OK) return st;
   if (w > 0) return scalekv_compress(ctx, layer, Q, w, window_pos, 1);
   if (w < 0) return scalekv_compress(ctx, layer, Q, 0, nullptr, 1);
