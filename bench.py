@@ -336,7 +336,8 @@ def run_scalekv(args):
 
     kv = make_kv()
     inputs = pipeline.PassInputs(wl, device=local_rank)
-    work = pipeline.pass_work(wl, budgets, windows, recent=select is not None and select["policy"] == "recent")
+    work = pipeline.pass_work(wl, budgets, windows, recent=select is not None and select["policy"] == "recent",
+                              one_call_steps=select is None)
     torch.cuda.synchronize()
 
     def barrier():

@@ -211,7 +211,14 @@ scalekv_status scalekv_compress_ex(scalekv_ctx *ctx, int32_t layer, scalekv_tens
 /* One whole step for one layer from DEVICE tensors, in one call: scalekv_append(K, V), scalekv_attend(Q -> O
  * [, lse]) and, with the window rows taken from Q (the full current map), scalekv_compress.
  * w > 0: window_pos holds w raster indices; w < 0: the whole current map is the window; w == 0: no
- * compress.  Same contracts as the three calls; saves two trips through the binding per step. */
+ * compress.  Same results as the three calls; saves two trips through the binding per step.
+ * Because the step knows what follows its attend, it does not write rows into the store that nothing will read: when
+ * its compress evicts, the attend leaves the current map in K and V and the compress (on stream_side) takes the
+ * surviving rows from there - in a layer with a 3 % budget 19 of 20 rows of a map would otherwise be written only to
+ * be dropped; after the last scale with w == 0 the map stays in K and V until a later call for the layer (export,
+ * layer_stats) copies it, if one comes.  K and V (and Q, which the compress may read) must therefore stay unmodified
+ * until the step's compress has completed: until stream_main has passed the layer's next append, or scalekv_join or
+ * scalekv_sync; after the last scale, until the layer's next call has passed on stream_main or scalekv_reset. */
 scalekv_status scalekv_step(scalekv_ctx *ctx, int32_t layer, int32_t scale, scalekv_tensor Q, scalekv_tensor K,
                             scalekv_tensor V, scalekv_tensor O, float *lse, int32_t w, const int32_t *window_pos);
 

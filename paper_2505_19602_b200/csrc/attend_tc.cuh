@@ -424,7 +424,8 @@ struct Params {
   int n_k;
   float scale_log2e;   // softmax scale * log2(e)
   int box_rows;        // rows per K/V TMA box = min(page_tokens, 128)
-  int fused_append;    // 1: the current map's K/V rows are still in the caller's tensors; read them there and copy them in
+  int fused_append;    // 1: the current map's K/V rows are still in the caller's tensors; read them there
+  int copy_in;         // 1: and copy them into the pages on the way
   int n_prev;          // original position of the current map's first token
   // observation window (Sec. 3.3): when win_logits is not null, the raw products <q, k> of the w window rows
   // against every cache entry are recorded in win_logits[slice][rank][column], column = 128 j + position in key tile j
@@ -690,7 +691,7 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       const int st = t % kStages, j = t >> 1;
       ok = mbar_wait_warp(bar(bFull + st), (t / kStages) & 1, abort_flag, status);
       if (!ok) break;
-      if (j >= Th && (j - Th) % (int)gridDim.x == (int)blockIdx.x) {
+      if (prm.copy_in && j >= Th && (j - Th) % (int)gridDim.x == (int)blockIdx.x) {
         const int first = (j - Th) * 128;
         const int nvalid = tile_valid(j);
         char *pool = (t & 1) ? lv.v_pool : lv.k_pool;
@@ -972,7 +973,7 @@ struct AttendTc {
   // reads them there and copies them in), else nullptr.
   // win_logits / win_pos / w: where to record the window rows' logits (nullptr: do not).
   bool launch(const LayerView &lv, const TensorView &Q, const TensorView &O, float *lse, int n_k, const TensorView *Kc,
-              const TensorView *Vc, int n_prev, float scale, float *win_logits, float *win_lse, int ld_l, const int *win_pos, int w,
+              const TensorView *Vc, bool copy_in, int n_prev, float scale, float *win_logits, float *win_lse, int ld_l, const int *win_pos, int w,
               cudaStream_t stream, std::string &err) {
     CUtensorMap tmQ, tmKc, tmVc, tmO;
     const int B = lv.n_slices / lv.n_heads;
@@ -990,6 +991,7 @@ struct AttendTc {
     prm.scale_log2e = scale * 1.4426950408889634f;
     prm.box_rows = box_rows;
     prm.fused_append = fused ? 1 : 0;
+    prm.copy_in = (fused && copy_in) ? 1 : 0;
     prm.n_prev = n_prev;
     prm.win_logits = win_logits;
     prm.win_lse = win_lse;

@@ -40,6 +40,15 @@ struct TensorView {
   long long sb, sh, st;   // in elements
 };
 
+// A current map that has not been copied into the pages: the caller's K and V tensors ([B][H][n_k][d] views,
+// strides in elements of esize bytes).  on == 0: the map is in the pages like every other entry.
+struct ExternalMap {
+  int on;
+  const char *k, *v;
+  long long sb, sh, st;
+  int esize;
+};
+
 template <typename T>
 __device__ __forceinline__ const T *row_ptr(const TensorView &t, int b, int h, int i) {
   return reinterpret_cast<const T *>(t.ptr) + (long long)b * t.sb + (long long)h * t.sh + (long long)i * t.st;

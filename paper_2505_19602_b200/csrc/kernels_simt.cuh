@@ -742,12 +742,15 @@ __global__ void __launch_bounds__(256) compact_kernel(LayerView lv, const int *k
 //   phase 2  select_and_emit: radix select in shared memory, ascending keep list in shared memory.
 //   phase 3  slot j <- old slot keep[j] for K, V and pos, in chunks: every thread loads its 8 16-byte pieces of
 //            the chunk, block barrier, stores them (keep[j] >= j, see compact_kernel); the untouched prefix is skipped.
+// ext.on: the current map has not been copied into the pages (a one-call step whose attend left it in the caller's
+// tensors): entries hist .. L-1 are rows of those tensors, phase 3 reads the survivors among them there and every kept
+// row of the map is written, whatever its index.
 // Dynamic shared memory: 4 * (2 * ld_s + pages_per_slice) bytes.  grid = n_slices.
 // ------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(1024) compress_fused_kernel(LayerView lv, WindowArg wa, int policy, int n_sink,
                                                               const float *logits, const float *lse, int ld_l, float logit_scale,
                                                               int tile_padded, int budget, const int *slice_budget, int pool,
-                                                              float *scores, int ld_s, int *kept_count) {
+                                                              float *scores, int ld_s, int *kept_count, ExternalMap ext) {
   extern __shared__ uint32_t fsm[];
   uint32_t *key = fsm;                                   // [ld_s]
   int *list = reinterpret_cast<int *>(fsm + ld_s);       // [ld_s]
@@ -765,6 +768,10 @@ __global__ void __launch_bounds__(1024) compress_fused_kernel(LayerView lv, Wind
   if (policy == 0 && tid < w) lse_row[tid] = lse[(size_t)slice * w + tid];
   __syncthreads();
   auto row_of = [&](int slot) { return ((size_t)pt[slot >> lv.page_shift] << lv.page_shift) + (size_t)(slot & lv.page_mask); };
+  // With ext.on the current map (entries hist .. L-1) is not in the pages: entry i is row i - hist of the caller's
+  // tensors and its original position follows from its index.
+  auto pos_of = [&](int i) { return (ext.on && i >= hist) ? wa.n_prev + (i - hist) : lv.pos_pool[row_of(i)]; };
+  const long long ext_base = ext.on ? (long long)(slice / lv.n_heads) * ext.sb + (long long)(slice % lv.n_heads) * ext.sh : 0;
 
   // ---- phase 1: keys
   float *sc_out = scores + (size_t)slice * ld_s;
@@ -785,7 +792,7 @@ __global__ void __launch_bounds__(1024) compress_fused_kernel(LayerView lv, Wind
       for (; j < w; ++j) sc += exp2f(fmaf(__ldg(y + (size_t)j * ld_l), logit_scale, -lse_row[j]));
       sc *= inv_w;
       sc_out[i] = sc;
-      const bool win = is_window_pos(wa, lv.pos_pool[row_of(i)]);
+      const bool win = is_window_pos(wa, pos_of(i));
       key[i] = win ? kWindowKey : (__float_as_uint(sc) & 0x7FFFFFFFu);
     }
     if (pool > 1) {
@@ -798,7 +805,7 @@ __global__ void __launch_bounds__(1024) compress_fused_kernel(LayerView lv, Wind
     }
   } else {
     for (int i = tid; i < L; i += 1024) {
-      const int pos = lv.pos_pool[row_of(i)];
+      const int pos = pos_of(i);
       key[i] = pos < n_sink ? kWindowKey : (uint32_t)pos + 1u;
     }
   }
@@ -824,7 +831,9 @@ __global__ void __launch_bounds__(1024) compress_fused_kernel(LayerView lv, Wind
     const int mid = (lo + hi) >> 1;
     if (list[mid] == mid) lo = mid + 1; else hi = mid;
   }
+  if (ext.on && lo > hist) lo = hist;          // kept rows of the current map are not where they belong yet, whatever their index
   const int r_in = tid / per_row, c = tid % per_row;
+  const char *ext_ptr = c < ppr ? ext.k : ext.v;
   char *pool_ptr = c < ppr ? lv.k_pool : lv.v_pool;
   const int piece = c < ppr ? c : c - ppr;
   const bool pos_thread = c == 0;
@@ -836,9 +845,16 @@ __global__ void __launch_bounds__(1024) compress_fused_kernel(LayerView lv, Wind
       for (int u = 0; u < 8; ++u) {
         const int j = c0 + r_in + u * r_step;
         if (j < kept) {
-          const size_t row = row_of(list[j]);
-          buf[u] = reinterpret_cast<const uint4 *>(pool_ptr + row * lv.row_bytes)[piece];
-          if (pos_thread) pv[u] = lv.pos_pool[row];
+          const int src = list[j];
+          if (ext.on && src >= hist) {
+            const long long e = (ext_base + (long long)(src - hist) * ext.st) * ext.esize;
+            buf[u] = __ldg(reinterpret_cast<const uint4 *>(ext_ptr + e) + piece);
+            if (pos_thread) pv[u] = wa.n_prev + (src - hist);
+          } else {
+            const size_t row = row_of(src);
+            buf[u] = reinterpret_cast<const uint4 *>(pool_ptr + row * lv.row_bytes)[piece];
+            if (pos_thread) pv[u] = lv.pos_pool[row];
+          }
         }
       }
       __syncthreads();

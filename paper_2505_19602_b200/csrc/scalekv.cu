@@ -607,7 +607,13 @@ scalekv_status scalekv_append(scalekv_ctx *ctx, int32_t layer, int32_t scale, sc
 // their tile waits for them), so it is left out where no compress can use it: after the last scale of the schedule
 // (Sec. 3.3: nothing is generated after it, so the method prunes nothing there; a compress called all the same takes
 // its logits from K) and in a one-call step that names no window.
-static scalekv_status attend_impl(scalekv_ctx *ctx, int32_t layer, scalekv_tensor Q, scalekv_tensor O, float *lse, bool record) {
+// copy: whether a current map that is still in the caller's tensors is also copied into the pages while the kernel
+// streams it.  A one-call step leaves the copy out when its own compress will evict (the compress then takes the
+// surviving rows of the map straight from the caller's tensors: in a refiner layer 19 of 20 rows of a map would be
+// written to the pages only to be dropped) and after the last scale without a compress (the rows are copied by
+// whichever later call needs them, if any does).
+static scalekv_status attend_impl(scalekv_ctx *ctx, int32_t layer, scalekv_tensor Q, scalekv_tensor O, float *lse, bool record,
+                                  bool copy) {
   if (!ctx) return SCALEKV_ERR_INVALID_ARG;
   const Plan &p = ctx->plan;
   if (layer < 0 || layer >= p.n_layers) return fail(ctx, SCALEKV_ERR_INVALID_ARG, "layer %d out of range", layer);
@@ -632,10 +638,10 @@ static scalekv_status attend_impl(scalekv_ctx *ctx, int32_t layer, scalekv_tenso
                       ? nullptr
                       : reinterpret_cast<float *>(ctx->ws + p.off_logits) + (size_t)(layer % kSets) * p.logits_elems;
       float *wlse = reinterpret_cast<float *>(ctx->ws + p.off_wlse) + (size_t)(layer % kSets) * p.n_slices * p.max_window;
-      if (!ctx->tc.launch(lv, tview(Q), tview(O), lse, nk, fused ? &kc : nullptr, fused ? &vc : nullptr, p.N[k], ctx->scale, wl,
-                          wlse, p.ld_l, win.data(), (int)win.size(), ctx->s_main, e))
+      if (!ctx->tc.launch(lv, tview(Q), tview(O), lse, nk, fused ? &kc : nullptr, fused ? &vc : nullptr, fused && copy, p.N[k],
+                          ctx->scale, wl, wlse, p.ld_l, win.data(), (int)win.size(), ctx->s_main, e))
         return fail(ctx, SCALEKV_ERR_CUDA, "attend launch: %s", e.c_str());
-      ctx->in_store[layer] = 1;
+      if (copy) ctx->in_store[layer] = 1;
       ctx->logits_of[layer] = wl ? k : -1;
       ctx->logits_padded[layer] = fused ? 1 : 0;
     } else {
@@ -654,7 +660,7 @@ static scalekv_status attend_impl(scalekv_ctx *ctx, int32_t layer, scalekv_tenso
 }
 
 scalekv_status scalekv_attend(scalekv_ctx *ctx, int32_t layer, scalekv_tensor Q, scalekv_tensor O, float *lse) {
-  return attend_impl(ctx, layer, Q, O, lse, true);
+  return attend_impl(ctx, layer, Q, O, lse, true, true);
 }
 
 scalekv_status scalekv_compress(scalekv_ctx *ctx, int32_t layer, scalekv_tensor Qw, int32_t w, const int32_t *window_pos,
@@ -729,9 +735,18 @@ scalekv_status scalekv_compress_ex(scalekv_ctx *ctx, int32_t layer, scalekv_tens
   const bool evict = budget != SCALEKV_KEEP_ALL && (budget < cand || hb_on);
   // while per-kernel timing is on, compress runs on stream_main too, so that every kernel is timed alone
   cudaStream_t s = ctx->serialize ? ctx->s_main : ctx->s_side;
-  const bool copy_now = !ctx->in_store[layer];
-  st = materialize(ctx, layer);
-  if (st != SCALEKV_OK) return st;
+  // the logits of exactly this window may already be there, recorded by attend
+  bool recorded = recent || (ctx->logits_of[layer] == k && (int)p.windows[k].size() == wa.w);
+  for (int j = 0; !recent && recorded && j < wa.w; ++j) recorded = p.windows[k][j] == wa.pos[j];
+  const bool fused = ctx->fused_ok && !head_shared && !(opts && opts->separate_kernels);
+  // A map that attend left in the caller's tensors stays there when the one-launch compress can do without the pages:
+  // it needs no K (the logits are recorded) and takes the surviving rows from the tensors.  Everything else copies first.
+  const bool external = !ctx->in_store[layer] && ctx->attended[layer] && evict && fused && recorded;
+  const bool copy_now = !ctx->in_store[layer] && !external;
+  if (!external) {
+    st = materialize(ctx, layer);
+    if (st != SCALEKV_OK) return st;
+  }
   if (s != ctx->s_main) {
     if (!ctx->attended[layer] || copy_now) CU(cudaEventRecord(ctx->ev_attend[layer], ctx->s_main));
     CU(cudaStreamWaitEvent(s, ctx->ev_attend[layer], 0));
@@ -746,14 +761,10 @@ scalekv_status scalekv_compress_ex(scalekv_ctx *ctx, int32_t layer, scalekv_tens
     int *keep = reinterpret_cast<int *>(ctx->ws + p.off_keep);
     int *kept = reinterpret_cast<int *>(ctx->ws + p.off_kept);
     uint32_t *keys = reinterpret_cast<uint32_t *>(ctx->ws + p.off_keys);
-    const bool fused = ctx->fused_ok && !head_shared && !(opts && opts->separate_kernels);
     if (recent && !fused) {
       Scope sc(ctx, s, kScore);
       recent_keys_kernel<<<dim3((L + 255) / 256, p.n_slices), 256, 0, s>>>(lv, wa.n_k, n_sink, keys, p.ld_s);
     }
-    // the logits of exactly this window may already be there, recorded by attend
-    bool recorded = recent || (ctx->logits_of[layer] == k && (int)p.windows[k].size() == wa.w);
-    for (int j = 0; !recent && recorded && j < wa.w; ++j) recorded = p.windows[k][j] == wa.pos[j];
     if (!recorded) {
       // this writes the logit buffer of the layer's set: if another layer of that set has appended since, what
       // its attend recorded there is lost (its compress scores from K too), and its attend must be through first
@@ -791,8 +802,15 @@ scalekv_status scalekv_compress_ex(scalekv_ctx *ctx, int32_t layer, scalekv_tens
     if (fused) {
       // importance, selection and pruning of a slice by one CTA, in one launch
       Scope sc(ctx, s, kCompress);
+      ExternalMap ext{};
+      if (external) {
+        const TensorView kc = tview(ctx->pend_k[layer]), vc = tview(ctx->pend_v[layer]);
+        ext.on = 1; ext.k = kc.ptr; ext.v = vc.ptr; ext.sb = kc.sb; ext.sh = kc.sh; ext.st = kc.st; ext.esize = p.esize;
+        if (vc.sb != kc.sb || vc.sh != kc.sh || vc.st != kc.st) return fail(ctx, SCALEKV_ERR_INVALID_ARG, "K and V of a map must have the same strides");
+      }
       compress_fused_kernel<<<p.n_slices, 1024, ctx->fused_smem, s>>>(lv, wa, recent ? 1 : 0, n_sink, logits, wlse, p.ld_l, logit_scale,
-                                                                     tile_padded, budget, slice_budget, pool, scores, p.ld_s, kept);
+                                                                     tile_padded, budget, slice_budget, pool, scores, p.ld_s, kept, ext);
+      if (external) ctx->in_store[layer] = 1;
     } else {
       if (!recent) {
         Scope sc(ctx, s, kScore);
@@ -893,7 +911,23 @@ scalekv_status scalekv_step(scalekv_ctx *ctx, int32_t layer, int32_t scale, scal
                             scalekv_tensor O, float *lse, int32_t w, const int32_t *window_pos) {
   scalekv_status st = scalekv_append(ctx, layer, scale, K, V);
   if (st != SCALEKV_OK) return st;
-  st = attend_impl(ctx, layer, Q, O, lse, w > 0);
+  // whether the step's own compress will evict (the test scalekv_compress makes) and so can take the map's surviving
+  // rows from K and V itself; after the last scale without a compress nothing may ever need the rows
+  bool copy = true;
+  if (ctx && ctx->tc.enabled() && layer >= 0 && layer < ctx->plan.n_layers && scale >= 0 && scale < ctx->plan.K) {
+    const Plan &p = ctx->plan;
+    const int table = p.budgets[(size_t)layer * p.K + scale];
+    const int L = ctx->hist[layer] + p.n[scale];
+    if (w > 0) {
+      // ... and will find the logits of exactly its window recorded (else it needs K in the pages)
+      bool planned = ctx->fused_ok && scale + 1 != p.K && window_pos && (int)p.windows[scale].size() == w;
+      for (int j = 0; planned && j < w; ++j) planned = p.windows[scale][j] == window_pos[j];
+      copy = !(planned && table != SCALEKV_KEEP_ALL && table < L - w);
+    } else if (w == 0) {
+      copy = scale + 1 != p.K;
+    }
+  }
+  st = attend_impl(ctx, layer, Q, O, lse, w > 0, copy);
   if (st != SCALEKV_OK) return st;
   if (w > 0) return scalekv_compress(ctx, layer, Q, w, window_pos, 1);
   if (w < 0) return scalekv_compress(ctx, layer, Q, 0, nullptr, 1);

@@ -125,13 +125,15 @@ def run_pass(kv: binding.ScaleKV, inputs: PassInputs, windows, compress_last=Fal
         mark()
 
 
-def pass_work(wl: synth.Workload, budgets, windows, recent=False):
+def pass_work(wl: synth.Workload, budgets, windows, recent=False, one_call_steps=True):
     """Algorithmic work of one pass, from the schedule alone.
 
     attend_flop       4 n_k L d per slice-step.
-    attend_min_bytes  what attend must move: K and V of the L entries once, Q and O, plus - since it also
+    attend_min_bytes  what attend must move: K and V of the L entries once, Q and O, plus - where it also
                       appends - the write of the current map's K/V rows and positions into the pages, and
-                      the write of the w x L window logits.
+                      the write of the w x L window logits where it records them (not after the last scale).
+                      one_call_steps: the pass is made of scalekv_step calls, whose attend leaves the map in the
+                      caller's tensors when the step's compress evicts and after the last scale.
     score_bytes       the score kernel: w x L logits and L positions in, L scores and L keys out (plus K read
                       by the stand-alone logits kernel when attend did not record the logits).
     select_bytes      the select kernel: L keys in, the keep list out.
@@ -158,8 +160,13 @@ def pass_work(wl: synth.Workload, budgets, windows, recent=False):
             out["attend_flop"] += f
             per_scale_flop[k] += f
             out["attend_min_bytes"] += (2 * L + 2 * n[k]) * d * esz * slices
+            last = k + 1 == wl.n_scales
+            evicts = (not last) and budgets[l][k] != binding.KEEP_ALL and budgets[l][k] < L - wk
             if fused:
-                out["attend_min_bytes"] += (2 * n[k] * d * esz + 4 * n[k] + 4 * w * L) * slices
+                if not (one_call_steps and (last or evicts)):
+                    out["attend_min_bytes"] += (2 * n[k] * d * esz + 4 * n[k]) * slices
+                if not last:
+                    out["attend_min_bytes"] += 4 * w * L * slices
             else:
                 out["append_bytes"] += 2 * 2 * n[k] * d * esz * slices
             out["attend_launches"] += 1
