@@ -909,6 +909,51 @@ def test_one_call_step_equals_the_three_calls():
         assert all(torch.equal(x, y) for x, y in zip(a, b))
 
 
+def test_step_takes_surviving_rows_from_strided_caller_tensors():
+    """A one-call step whose compress evicts leaves the current map in the caller's K and V and gathers the survivors
+    from there: with K and V as strided views (token stride 3 d, head-major storage) it must keep exactly the rows, values
+    and positions that the same step keeps from dense tensors, and what three separate calls (attend copies) keep."""
+    from paper_2505_19602_b200 import pipeline
+    sides = (3, 6, 10, 15)
+    n = orc.scale_token_counts(sides)
+    B, H, d = 2, 2, 128
+    budgets = [[30] * len(sides)]
+    windows = pipeline.windows_for(sides, 16)
+    gen = torch.Generator().manual_seed(77)
+    data = [[torch.randn(B, H, nk, d, generator=gen).to(torch.bfloat16).cuda() for _ in range(3)] for nk in n]
+
+    def strided(t):
+        big = torch.zeros(t.shape[1], t.shape[0], t.shape[2], 3 * d, dtype=t.dtype, device="cuda")
+        big[..., d:2 * d] = t.permute(1, 0, 2, 3)
+        return big[..., d:2 * d].permute(1, 0, 2, 3)          # [B, H, n, d] view: strides (n 3d, B n 3d, 3d, 1)
+
+    kept = []
+    for mode in ("dense", "strided", "three"):
+        kv = binding.ScaleKV(1, B, H, d, "bf16", sides, sides, budgets, max_window=16)
+        hold = []
+        for k, nk in enumerate(n):
+            Q, K, V = data[k]
+            if mode == "strided":
+                K, V = strided(K), strided(V)
+                assert not K.is_contiguous()
+            hold.append((K, V))
+            O = torch.empty_like(Q)
+            last = k + 1 == len(n)
+            if mode == "three":
+                kv.scalekv_append(0, k, K, V)
+                kv.scalekv_attend(0, Q, O)
+                if not last:
+                    kv.scalekv_compress(0, Q, windows[k], qw_is_full_map=True)
+            else:
+                kv.scalekv_step(0, k, Q, K, V, O, window_pos=None if last else windows[k])
+        kv.scalekv_sync()
+        kept.append([kv.scalekv_export_slice(0, b, h, with_kv=True) for b in range(B) for h in range(H)])
+        kv.close()
+    for other in kept[1:]:
+        for a, b in zip(kept[0], other):
+            assert all(torch.equal(x, y) for x, y in zip(a, b))
+
+
 @pytest.mark.parametrize("amp", [6.0, 12.0])
 def test_dominant_keys_anywhere_in_the_first_tiles(amp):
     """Rows whose logit towards one key is 70 or 140 nats above the rest, that key sitting in the first
