@@ -337,7 +337,7 @@ def run_scalekv(args):
     kv = make_kv()
     inputs = pipeline.PassInputs(wl, device=local_rank)
     work = pipeline.pass_work(wl, budgets, windows, recent=select is not None and select["policy"] == "recent",
-                              one_call_steps=select is None)
+                              one_call_steps=True)
     torch.cuda.synchronize()
 
     def barrier():

@@ -222,6 +222,14 @@ scalekv_status scalekv_compress_ex(scalekv_ctx *ctx, int32_t layer, scalekv_tens
 scalekv_status scalekv_step(scalekv_ctx *ctx, int32_t layer, int32_t scale, scalekv_tensor Q, scalekv_tensor K,
                             scalekv_tensor V, scalekv_tensor O, float *lse, int32_t w, const int32_t *window_pos);
 
+/* scalekv_step with a selection variant: compress == 0: no compress; otherwise the step ends with
+ * scalekv_compress_ex(layer, Q as the full current map, w, window_pos, opts) - Sec. 4.1's comparison rules as one-call
+ * steps (w and window_pos as scalekv_compress_ex takes them: ignored by SCALEKV_SELECT_RECENT, window_pos == NULL for the
+ * whole map).  Same results and the same contract as scalekv_step. */
+scalekv_status scalekv_step_ex(scalekv_ctx *ctx, int32_t layer, int32_t scale, scalekv_tensor Q, scalekv_tensor K,
+                               scalekv_tensor V, scalekv_tensor O, float *lse, int32_t compress, int32_t w,
+                               const int32_t *window_pos, const scalekv_select_opts *opts);
+
 /* One whole step for one layer from HOST memory (pinned memory recommended): copies Q, K, V
  * (dense [B][H][n_k][d]) to `staging`, runs append, attend and compress with the window rows
  * taken from Q (w > 0: explicit window_pos; w < 0: the whole map is the window; w == 0: no

@@ -96,6 +96,7 @@ def load_library():
         "scalekv_compress": [ctx_p, i32, T, i32, P(i32), i32],
         "scalekv_compress_ex": [ctx_p, i32, T, i32, P(i32), i32, P(scalekv_select_opts)],
         "scalekv_step": [ctx_p, i32, i32, T, T, T, T, P(C.c_float), i32, P(i32)],
+        "scalekv_step_ex": [ctx_p, i32, i32, T, T, T, T, P(C.c_float), i32, i32, P(i32), P(scalekv_select_opts)],
         "scalekv_step_host": [ctx_p, i32, i32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, i32, P(i32)],
         "scalekv_layer_stats": [ctx_p, i32, T, i32, i32, P(f64), P(f64)],
         "scalekv_layer_stats_ex": [ctx_p, i32, T, i32, i32, P(f64), P(f64), P(f64), P(f64), P(f64)],
@@ -352,6 +353,21 @@ class ScaleKV:
     def window_array(window_pos):
         """The window as the ctypes array the calls take, so that a loop need not rebuild it."""
         return _i32_array(window_pos)
+
+    def scalekv_step_ex(self, layer, scale, Q, K, V, O, compress=True, window_pos=None, lse=None, policy="score", pool_kernel=1,
+                        n_sink=0, head_shared=False, head_budgets=None, separate_kernels=False):
+        """append + attend + scalekv_compress_ex (Q as the full current map) in one call; compress=False: no compress."""
+        hb = _i32_array(head_budgets) if head_budgets is not None else None
+        opts = scalekv_select_opts({"score": 0, "recent": 1}[policy], pool_kernel, n_sink, int(head_shared), hb,
+                                   int(separate_kernels))
+        if window_pos is None:
+            wp, w = None, 0
+        else:
+            wp = window_pos if isinstance(window_pos, C.Array) else _i32_array(window_pos)
+            w = len(wp)
+        lp = C.cast(lse.data_ptr(), C.POINTER(C.c_float)) if lse is not None else None
+        self._check(self.lib.scalekv_step_ex(self.ctx, layer, scale, tensor_arg(Q), tensor_arg(K), tensor_arg(V), tensor_arg(O),
+                                             lp, int(bool(compress)), w, wp, C.byref(opts)))
 
     def scalekv_step_host(self, layer, scale, Qh, Kh, Vh, Oh, staging, window_pos=None, whole_map=False):
         if whole_map:

@@ -907,31 +907,52 @@ scalekv_status scalekv_step_host(scalekv_ctx *ctx, int32_t layer, int32_t scale,
   return SCALEKV_OK;
 }
 
+// Whether the attend of a one-call step copies the current map into the pages (see attend_impl).  It does not when
+// the step's own compress will evict - the test scalekv_compress_ex makes - and will find what it needs without K in
+// the pages (the logits of exactly its window recorded, or a positional rule), so that it can take the map's
+// surviving rows from K and V itself; nor after the last scale without a compress, when nothing may ever need the rows.
+// A wrong guess costs a copy kernel, never a result.
+static bool step_copies(const scalekv_ctx *ctx, int layer, int scale, bool compress, int w, const int32_t *window_pos,
+                        const scalekv_select_opts *opts) {
+  if (!ctx || !ctx->tc.enabled() || layer < 0 || layer >= ctx->plan.n_layers || scale < 0 || scale >= ctx->plan.K) return true;
+  const Plan &p = ctx->plan;
+  if (!compress) return scale + 1 != p.K;
+  if (!ctx->fused_ok || (opts && (opts->head_shared || opts->separate_kernels || opts->head_budgets))) return true;
+  const int table = p.budgets[(size_t)layer * p.K + scale];
+  if (table == SCALEKV_KEEP_ALL) return true;
+  const int L = ctx->hist[layer] + p.n[scale];
+  if (opts && opts->policy == SCALEKV_SELECT_RECENT) {
+    const int sinks = std::min(std::max(opts->n_sink, 0), p.N[scale + 1]);
+    return !(std::max(table - sinks, 0) < L - sinks);
+  }
+  if (w <= 0) return true;
+  bool planned = scale + 1 != p.K && window_pos && (int)p.windows[scale].size() == w;
+  for (int j = 0; planned && j < w; ++j) planned = p.windows[scale][j] == window_pos[j];
+  return !(planned && table < L - w);
+}
+
 scalekv_status scalekv_step(scalekv_ctx *ctx, int32_t layer, int32_t scale, scalekv_tensor Q, scalekv_tensor K, scalekv_tensor V,
                             scalekv_tensor O, float *lse, int32_t w, const int32_t *window_pos) {
   scalekv_status st = scalekv_append(ctx, layer, scale, K, V);
   if (st != SCALEKV_OK) return st;
-  // whether the step's own compress will evict (the test scalekv_compress makes) and so can take the map's surviving
-  // rows from K and V itself; after the last scale without a compress nothing may ever need the rows
-  bool copy = true;
-  if (ctx && ctx->tc.enabled() && layer >= 0 && layer < ctx->plan.n_layers && scale >= 0 && scale < ctx->plan.K) {
-    const Plan &p = ctx->plan;
-    const int table = p.budgets[(size_t)layer * p.K + scale];
-    const int L = ctx->hist[layer] + p.n[scale];
-    if (w > 0) {
-      // ... and will find the logits of exactly its window recorded (else it needs K in the pages)
-      bool planned = ctx->fused_ok && scale + 1 != p.K && window_pos && (int)p.windows[scale].size() == w;
-      for (int j = 0; planned && j < w; ++j) planned = p.windows[scale][j] == window_pos[j];
-      copy = !(planned && table != SCALEKV_KEEP_ALL && table < L - w);
-    } else if (w == 0) {
-      copy = scale + 1 != p.K;
-    }
-  }
-  st = attend_impl(ctx, layer, Q, O, lse, w > 0, copy);
+  st = attend_impl(ctx, layer, Q, O, lse, w > 0, step_copies(ctx, layer, scale, w != 0, w, window_pos, nullptr));
   if (st != SCALEKV_OK) return st;
   if (w > 0) return scalekv_compress(ctx, layer, Q, w, window_pos, 1);
   if (w < 0) return scalekv_compress(ctx, layer, Q, 0, nullptr, 1);
   return SCALEKV_OK;
+}
+
+scalekv_status scalekv_step_ex(scalekv_ctx *ctx, int32_t layer, int32_t scale, scalekv_tensor Q, scalekv_tensor K, scalekv_tensor V,
+                               scalekv_tensor O, float *lse, int32_t compress, int32_t w, const int32_t *window_pos,
+                               const scalekv_select_opts *opts) {
+  scalekv_status st = scalekv_append(ctx, layer, scale, K, V);
+  if (st != SCALEKV_OK) return st;
+  const bool score = !opts || opts->policy == SCALEKV_SELECT_SCORE;
+  st = attend_impl(ctx, layer, Q, O, lse, compress != 0 && score && w > 0,
+                   step_copies(ctx, layer, scale, compress != 0, w, window_pos, opts));
+  if (st != SCALEKV_OK) return st;
+  if (!compress) return SCALEKV_OK;
+  return scalekv_compress_ex(ctx, layer, Q, w, window_pos, 1, opts);
 }
 
 scalekv_status scalekv_layer_stats(scalekv_ctx *ctx, int32_t layer, scalekv_tensor Q, int32_t topk_prime,

@@ -75,7 +75,8 @@ class PassInputs:
 
 def scale_step(kv: binding.ScaleKV, inputs: PassInputs, windows, k, compress_last=False, three_calls=False, select=None):
     """One scale-step: append -> attend -> compress of every layer at scale k (one scalekv_step per layer, or
-    the three calls one by one with three_calls=True or a comparison policy in `select`: the same launches)."""
+    the three calls one by one with three_calls=True: the same launches; `select`: the options of a comparison policy,
+    through scalekv_step_ex or, with three_calls, scalekv_compress_ex)."""
     wl = inputs.wl
     nk = wl.n_tokens[k]
     O = inputs.O[:, :, :nk, :]
@@ -84,6 +85,9 @@ def scale_step(kv: binding.ScaleKV, inputs: PassInputs, windows, k, compress_las
     wp = kv.window_array(windows[k]) if (do_compress and windows[k] is not None) else None
     for l in range(wl.n_layers):
         Q, K, V = inputs.data[(l, k)]
+        if select is not None and not three_calls:
+            kv.scalekv_step_ex(l, k, Q, K, V, O, compress=do_compress, window_pos=windows[k], **select)
+            continue
         if select is not None:
             kv.scalekv_append(l, k, K, V)
             kv.scalekv_attend(l, Q, O)

@@ -909,6 +909,34 @@ def test_one_call_step_equals_the_three_calls():
         assert all(torch.equal(x, y) for x, y in zip(a, b))
 
 
+@pytest.mark.parametrize("rule", ["sinks", "snapkv"])
+def test_step_ex_equals_the_three_calls_for_the_comparison_rules(rule):
+    """scalekv_step_ex (one call per step, the attend leaving out the copies nothing reads) leaves exactly what
+    append, attend and scalekv_compress_ex leave: outputs, kept rows, values and positions."""
+    from paper_2505_19602_b200 import pipeline
+    sides = (2, 4, 7, 11, 16)
+    wl = synth.Workload("sx", 2, 2, 2, 128, "bf16", sides, seed=43)
+    budgets = [[60] * len(sides), [25] * len(sides)]
+    if rule == "sinks":
+        select, kind, windows = {"policy": "recent", "n_sink": 4}, "centroids", pipeline.windows_for(sides, 16)
+    else:
+        select, kind = {"policy": "score", "pool_kernel": 7}, "last"
+        windows = [binding.scalekv_window_last(a, a, 16) for a in sides]
+    results = []
+    for three in (True, False):
+        kv = binding.ScaleKV(2, 2, 2, 128, "bf16", sides, sides, budgets, max_window=16, window_kind=kind)
+        inputs = pipeline.PassInputs(wl)
+        pipeline.run_pass(kv, inputs, windows, three_calls=three, select=select)
+        kv.scalekv_sync()
+        kept = [kv.scalekv_export_slice(l, b, h, with_kv=True) for l in range(2) for b in range(2) for h in range(2)]
+        results.append((inputs.O.clone(), kept))
+        kv.close()
+    (O3, kept3), (O1, kept1) = results
+    assert torch.equal(O3, O1)
+    for a, b in zip(kept3, kept1):
+        assert all(torch.equal(x, y) for x, y in zip(a, b))
+
+
 def test_step_takes_surviving_rows_from_strided_caller_tensors():
     """A one-call step whose compress evicts leaves the current map in the caller's K and V and gathers the survivors
     from there: with K and V as strided views (token stride 3 d, head-major storage) it must keep exactly the rows, values
