@@ -842,10 +842,17 @@ attend_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           __syncwarp();
           if (lane == 0) mbar_arrive(bar(bPEarly + buf));
         }
-        if (cc + 2 < kChunks) {
-          tc_wait_ld();
-          if (kWindow && wwarp) log_window(v[cc & 1], cc + 2);
-        }
+        if (cc + 2 < kChunks) tc_wait_ld();
+      }
+      // The window rows' products of the tile's second half are recorded here, not between the chunks (a branch
+      // there costs every warp's schedule 2-3 %): columns 64-127 of the S buffer still hold them, P only covers
+      // columns 0-63, and the buffer is not written again before this warp has arrived below.
+      if (kWindow && wwarp && ok) {
+        tc_ld32(s_addr + 64, v[0]);
+        tc_ld32(s_addr + 96, v[1]);
+        tc_wait_ld();
+        log_window(v[0], 2);
+        log_window(v[1], 3);
       }
       };
       if (valid < 128) sweep(std::true_type{}); else sweep(std::false_type{});
