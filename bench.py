@@ -33,8 +33,8 @@ METRIC = "scale_steps_per_sec"
 # one layer of the workload; traffic grows in proportion to the bytes a launch must move, so the roofline object reports
 # this ratio times the average algorithmic bytes per launch.  Captured on the kernel as of the commit named below
 # (profiles/attend_tc_kernel_pass2b_1layer.md); set ATTEND_TRAFFIC_RATIO to None when attend_tc.cuh changes after it.
-ATTEND_TRAFFIC_RATIO = 1112.6 / 1128.4
-ATTEND_TRAFFIC_SOURCE = ("ncu capture of attend_tc_kernel at commit 32d9126 (one layer, scales 12 and 13), scaled to the "
+ATTEND_TRAFFIC_RATIO = 1110.5 / 1128.4
+ATTEND_TRAFFIC_SOURCE = ("ncu capture of attend_tc_kernel at commit 319ec61 (one layer, scales 12 and 13), scaled to the "
                          "average launch by algorithmic bytes")
 UNIT = "scale-steps/s"
 E2E_HOST_LAYERS = 4
