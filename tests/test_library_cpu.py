@@ -112,3 +112,24 @@ def test_comparison_policy_helpers_match_oracle(lib):
         for L, b, beta in ((32, 627, 20.0), (40, 1300.5, 20.0), (5, 100, 4.0), (1, 77, 20.0), (6, 50, 1.0)):
             assert np.array_equal(binding.scalekv_policy_budgets(shape, L, 4, b, beta), orc.policy_budgets(shape, L, 4, b, beta))
 
+
+
+def test_pass_work_counts_what_a_one_call_step_leaves_out():
+    """The algorithmic byte count of attend (the bench's roofline traffic comes from it): same flop either way; with
+    one-call steps the appended rows of evicting steps and of the last scale are not counted, and nobody records window
+    logits after the last scale.  Checked against a count written out here for a two-scale, one-layer schedule."""
+    from paper_2505_19602_b200 import pipeline, synth
+    sides = (4, 12)                      # 16 and 144 tokens
+    wl = synth.Workload("pw", 1, 1, 2, 128, "bf16", sides, seed=1)
+    windows = [[0, 5], [3, 77]]          # two window rows per scale
+    budgets = [[6, 6]]                   # scale 0: 16 - 2 candidates > 6: evicts; scale 1 is the last
+    full = pipeline.pass_work(wl, budgets, windows, one_call_steps=False)
+    step = pipeline.pass_work(wl, budgets, windows, one_call_steps=True)
+    assert full["attend_flop"] == step["attend_flop"] == 4 * 128 * 2 * (16 * 16 + 144 * (8 + 144))
+    row = 128 * 2
+    kv_q_o = 2 * ((2 * 16 + 2 * 16) + (2 * (8 + 144) + 2 * 144)) * row          # K, V of L entries, Q and O, both slices
+    logits = 2 * 4 * 2 * 16                                                   # w x L floats at scale 0 only
+    appended = 2 * ((2 * 16 * row + 4 * 16) + (2 * 144 * row + 4 * 144))
+    assert full["attend_min_bytes"] == kv_q_o + logits + appended
+    assert step["attend_min_bytes"] == kv_q_o + logits                        # scale 0 evicts, scale 1 is the last
+    assert full["compress_bytes"] == step["compress_bytes"] and step["compress_launches"] == 1
